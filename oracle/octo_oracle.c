@@ -1,0 +1,350 @@
+/*
+ * CPU oracle for the per-batch tensor work of a cascade pipeline stage.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA library is
+ * checked against.  It shares no code with the CUDA path and must never be linked into,
+ * imported by or called from it; only the tests, the smoke check and the benchmark's CPU
+ * baseline leg may use it.
+ *
+ * What the paper fixes and what it does not.  The paper (OctopInf) describes pipelines as
+ * cascades of DNNs such as [Object Detect -> Vehicle Classify, Plate Detect] (Section I),
+ * whose models map an image to bounding boxes (Table II, In_m / Out_m), run in batches of
+ * size bz (Eq. 1, Algorithm 1) and hand their detections to downstream models
+ * (Section III-B, Observation 1).  It gives no formula for the tensor work around the
+ * model.  Every numeric rule below is therefore a stated reading (labelled R1..R8 in the
+ * comments), chosen so that exactly one result is correct:
+ *
+ *   R1 letterbox geometry      integer, round-half-up of the scaled short side, centred
+ *   R2 bilinear resize core    half-pixel centres, edge clamp, no antialias; double here
+ *   R3 decode / score          best class by raw value, score = sigma(obj)*sigma(cls) in a
+ *                              fixed sequence of binary32 operations
+ *   R4 ordering                score descending, ties by lower anchor index
+ *   R5 greedy class-aware NMS  IoU in a fixed binary32 formula, strict thresholds
+ *   R6 scale-back              letterbox pixels -> frame pixels, binary32, clamped
+ *   R7 crop rectangle + resize outward-rounded integer rectangle, stretched by R2
+ *   R8 batch assembler         exclusive prefix sum of per-frame masked counts
+ *
+ * Floating point that decides an index (R3, R5, R6) is binary32 with every operation
+ * rounded on its own (build with -ffp-contract=off); pixel values (R2) are double.
+ * Parity pins live in tests/test_oracle_*.py; no function here is unpinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------------------ */
+/* R1: letterbox geometry.  The longer side maps to S; the other side is h*S/w rounded   */
+/* half-up in exact integer arithmetic; the image is centred, an odd remainder puts the  */
+/* extra canvas pixel on the right / bottom.                                             */
+/* ------------------------------------------------------------------------------------ */
+void orc_letterbox_geometry(int32_t w, int32_t h, int32_t S, int32_t* nw, int32_t* nh,
+                            int32_t* pad_l, int32_t* pad_t) {
+    int64_t W = w, H = h, s = S, a, b;
+    if (W >= H) {
+        a = s;
+        b = (2 * H * s + W) / (2 * W);
+        if (b < 1) b = 1;
+    } else {
+        b = s;
+        a = (2 * W * s + H) / (2 * H);
+        if (a < 1) a = 1;
+    }
+    *nw = (int32_t)a;
+    *nh = (int32_t)b;
+    *pad_l = (int32_t)((s - a) / 2);
+    *pad_t = (int32_t)((s - b) / 2);
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* R2: bilinear resize of the rectangle [rx0, rx0+cw) x [ry0, ry0+ch) of an interleaved   */
+/* 3-channel uint8 image to nw x nh.  Destination pixel centre (dx+0.5, dy+0.5) maps to   */
+/* source coordinate (dx+0.5)*cw/nw - 0.5, clamped to [0, cw-1]; the four taps are        */
+/* clamped inside the rectangle; raw 0..255 values, no intermediate rounding.             */
+/* out: [3][nh][nw] doubles in the image's own channel order.                             */
+/* ------------------------------------------------------------------------------------ */
+static double resize_tap(const uint8_t* img, int32_t pitch, int32_t rx0, int32_t ry0,
+                         int32_t x, int32_t y, int c) {
+    return (double)img[(size_t)(ry0 + y) * (size_t)pitch + (size_t)(rx0 + x) * 3 + (size_t)c];
+}
+
+void orc_resize_f64(const uint8_t* img, int32_t pitch, int32_t rx0, int32_t ry0, int32_t cw,
+                    int32_t ch, int32_t nw, int32_t nh, double* out) {
+    for (int dy = 0; dy < nh; ++dy) {
+        double sy = ((double)dy + 0.5) * ((double)ch / (double)nh) - 0.5;
+        if (sy < 0.0) sy = 0.0;
+        if (sy > (double)(ch - 1)) sy = (double)(ch - 1);
+        int y0 = (int)floor(sy);
+        int y1 = y0 + 1 < ch - 1 ? y0 + 1 : ch - 1;
+        double fy = sy - (double)y0;
+        for (int dx = 0; dx < nw; ++dx) {
+            double sx = ((double)dx + 0.5) * ((double)cw / (double)nw) - 0.5;
+            if (sx < 0.0) sx = 0.0;
+            if (sx > (double)(cw - 1)) sx = (double)(cw - 1);
+            int x0 = (int)floor(sx);
+            int x1 = x0 + 1 < cw - 1 ? x0 + 1 : cw - 1;
+            double fx = sx - (double)x0;
+            for (int c = 0; c < 3; ++c) {
+                double p00 = resize_tap(img, pitch, rx0, ry0, x0, y0, c);
+                double p01 = resize_tap(img, pitch, rx0, ry0, x1, y0, c);
+                double p10 = resize_tap(img, pitch, rx0, ry0, x0, y1, c);
+                double p11 = resize_tap(img, pitch, rx0, ry0, x1, y1, c);
+                double top = (1.0 - fx) * p00 + fx * p01;
+                double bot = (1.0 - fx) * p10 + fx * p11;
+                out[((size_t)c * (size_t)nh + (size_t)dy) * (size_t)nw + (size_t)dx] =
+                    (1.0 - fy) * top + fy * bot;
+            }
+        }
+    }
+}
+
+/* double -> IEEE binary16 bits, round to nearest even, one rounding (no float detour). */
+uint16_t orc_f64_to_half(double v) {
+    uint16_t sign = 0;
+    if (v != v) return 0x7E00;
+    if (v < 0.0) { sign = 0x8000; v = -v; }
+    if (v == 0.0) return sign;
+    if (v >= 65520.0) return (uint16_t)(sign | 0x7C00);
+    int e;
+    (void)frexp(v, &e); /* v = m * 2^e, m in [0.5, 1) */
+    int E = e - 1;      /* v = 1.f * 2^E */
+    if (E < -14) {
+        double q = rint(ldexp(v, 24)); /* units of 2^-24 */
+        return (uint16_t)(sign | (uint16_t)q);
+    }
+    double q = rint(ldexp(v, 10 - E)); /* in [1024, 2048] */
+    if (q >= 2048.0) { q = 1024.0; E += 1; }
+    if (E > 15) return (uint16_t)(sign | 0x7C00);
+    return (uint16_t)(sign | (uint16_t)((E + 15) << 10) | (uint16_t)((int)q - 1024));
+}
+
+/* R1 + R2: one frame -> [3][S][S] half bits.  Plane p holds input channel (swap_rb ? 2-p : p);
+ * value = half(v / 255); canvas outside the image = half(pad_value / 255). */
+void orc_letterbox(const uint8_t* img, int32_t w, int32_t h, int32_t pitch, int32_t S,
+                   int32_t pad_value, int32_t swap_rb, uint16_t* out) {
+    int32_t nw, nh, pl, pt;
+    orc_letterbox_geometry(w, h, S, &nw, &nh, &pl, &pt);
+    double* tmp = (double*)malloc(sizeof(double) * 3 * (size_t)nw * (size_t)nh);
+    orc_resize_f64(img, pitch, 0, 0, w, h, nw, nh, tmp);
+    uint16_t fill = orc_f64_to_half((double)pad_value / 255.0);
+    for (size_t i = 0; i < (size_t)3 * (size_t)S * (size_t)S; ++i) out[i] = fill;
+    for (int p = 0; p < 3; ++p) {
+        int c = swap_rb ? 2 - p : p;
+        for (int y = 0; y < nh; ++y)
+            for (int x = 0; x < nw; ++x)
+                out[((size_t)p * (size_t)S + (size_t)(pt + y)) * (size_t)S + (size_t)(pl + x)] =
+                    orc_f64_to_half(tmp[((size_t)c * (size_t)nh + (size_t)y) * (size_t)nw + (size_t)x] / 255.0);
+    }
+    free(tmp);
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* R3: logistic function as a fixed sequence of binary32 operations (each rounded to      */
+/* nearest even; the only fused operations are the ones written as fmaf):                 */
+/*   t = clamp(x, -30, 30); z = -t; n = rint(z * log2(e));                                */
+/*   r = z - n*ln2 (two-constant split, two fmaf); p = sum_{k<=7} r^k/k! by Horner;       */
+/*   e = p * 2^n (exact scaling); sigma = 1 / (1 + e).                                    */
+/* The platform expf is deliberately not used: its last bits differ between machines and  */
+/* would flip threshold tests and the score order.                                        */
+/* ------------------------------------------------------------------------------------ */
+float orc_sigmoid(float x) {
+    float t = fminf(fmaxf(x, -30.0f), 30.0f);
+    float z = -t;
+    float n = rintf(z * 0x1.715476p+0f);
+    float r = fmaf(n, -0x1.62e4p-1f, z);
+    r = fmaf(n, -0x1.7f7d1cp-20f, r);
+    float p = 0x1.a01a02p-13f;          /* 1/7! */
+    p = fmaf(p, r, 0x1.6c16c2p-10f);    /* 1/6! */
+    p = fmaf(p, r, 0x1.111112p-7f);     /* 1/5! */
+    p = fmaf(p, r, 0x1.555556p-5f);     /* 1/4! */
+    p = fmaf(p, r, 0x1.555556p-3f);     /* 1/3! */
+    p = fmaf(p, r, 0.5f);
+    p = fmaf(p, r, 1.0f);
+    p = fmaf(p, r, 1.0f);
+    union { uint32_t u; float f; } two_n;
+    two_n.u = (uint32_t)((int32_t)n + 127) << 23;
+    float e = p * two_n.f;
+    return 1.0f / (1.0f + e);
+}
+
+typedef struct {
+    float x1, y1, x2, y2, score;
+    int32_t cls, anchor, _pad;
+} orc_det_t; /* 32 bytes; same field order as the library's detection record */
+
+static int finite_f(float v) { return v == v && v - v == 0.0f; }
+
+/* R3: decode one image's head [A][5+C].  A row is a candidate iff every value in it is
+ * finite, w > 0, h > 0 and score > conf (strict), with k* = first maximal class value and
+ * score = fl(sigma(obj) * sigma(c_k*)) for logits, fl(obj * c_k*) for probabilities.
+ * Corners: x1 = fl(cx - fl(0.5*w)), x2 = fl(cx + fl(0.5*w)), same in y (letterbox pixels).
+ * Output in anchor order; returns the count.  out must hold A records. */
+int32_t orc_decode(const float* head, int32_t A, int32_t C, int32_t logits, float conf,
+                   orc_det_t* out) {
+    int32_t n = 0;
+    const int row = 5 + C;
+    for (int32_t a = 0; a < A; ++a) {
+        const float* p = head + (size_t)a * (size_t)row;
+        int ok = 1;
+        for (int k = 0; k < row; ++k) ok &= finite_f(p[k]);
+        if (!ok) continue;
+        if (!(p[2] > 0.0f) || !(p[3] > 0.0f)) continue;
+        int best = 0;
+        float bv = p[5];
+        for (int k = 1; k < C; ++k)
+            if (p[5 + k] > bv) { bv = p[5 + k]; best = k; }
+        float score;
+        if (logits) {
+            float so = orc_sigmoid(p[4]);
+            float sc = orc_sigmoid(bv);
+            score = so * sc;
+        } else {
+            score = p[4] * bv;
+        }
+        if (!(score > conf)) continue;
+        float hw = 0.5f * p[2], hh = 0.5f * p[3];
+        orc_det_t d;
+        d.x1 = p[0] - hw; d.y1 = p[1] - hh; d.x2 = p[0] + hw; d.y2 = p[1] + hh;
+        d.score = score; d.cls = best; d.anchor = a; d._pad = 0;
+        out[n++] = d;
+    }
+    return n;
+}
+
+/* R4: total order -- score descending, then anchor ascending. */
+static int cand_cmp(const void* pa, const void* pb) {
+    const orc_det_t* a = (const orc_det_t*)pa;
+    const orc_det_t* b = (const orc_det_t*)pb;
+    if (a->score > b->score) return -1;
+    if (a->score < b->score) return 1;
+    return (a->anchor > b->anchor) - (a->anchor < b->anchor);
+}
+void orc_sort(orc_det_t* c, int32_t n) { qsort(c, (size_t)n, sizeof(orc_det_t), cand_cmp); }
+
+/* R5: IoU in binary32, operation by operation. */
+float orc_iou(const orc_det_t* a, const orc_det_t* b) {
+    float iw = fminf(a->x2, b->x2) - fmaxf(a->x1, b->x1);
+    float ih = fminf(a->y2, b->y2) - fmaxf(a->y1, b->y1);
+    iw = fmaxf(iw, 0.0f);
+    ih = fmaxf(ih, 0.0f);
+    float inter = iw * ih;
+    float aw = a->x2 - a->x1, ah = a->y2 - a->y1;
+    float bw = b->x2 - b->x1, bh = b->y2 - b->y1;
+    float area_a = aw * ah, area_b = bw * bh;
+    float sum = area_a + area_b;
+    float uni = sum - inter;
+    return uni > 0.0f ? inter / uni : 0.0f;
+}
+
+/* R5: greedy class-aware NMS over a list already in R4 order.  Element i is kept iff no
+ * earlier KEPT element of the same class has IoU(j, i) > thr (strict); stops after max_det
+ * kept.  keep[] receives the kept positions in order; returns their number. */
+int32_t orc_nms(const orc_det_t* c, int32_t n, float thr, int32_t max_det, int32_t* keep) {
+    int32_t k = 0;
+    for (int32_t i = 0; i < n && k < max_det; ++i) {
+        int alive = 1;
+        for (int32_t t = 0; t < k; ++t) {
+            const orc_det_t* j = &c[keep[t]];
+            if (j->cls == c[i].cls && orc_iou(j, &c[i]) > thr) { alive = 0; break; }
+        }
+        if (alive) keep[k++] = i;
+    }
+    return k;
+}
+
+/* R6: letterbox pixels -> frame pixels in binary32: X = fl(fl(x - pad) * g), g = fl(w / nw),
+ * clamped to [0, w] (and [0, h]). */
+void orc_scale_back(orc_det_t* d, int32_t w, int32_t h, int32_t S) {
+    int32_t nw, nh, pl, pt;
+    orc_letterbox_geometry(w, h, S, &nw, &nh, &pl, &pt);
+    float gx = (float)w / (float)nw, gy = (float)h / (float)nh;
+    float fw = (float)w, fh = (float)h, fpl = (float)pl, fpt = (float)pt;
+    float X1 = (d->x1 - fpl) * gx, X2 = (d->x2 - fpl) * gx;
+    float Y1 = (d->y1 - fpt) * gy, Y2 = (d->y2 - fpt) * gy;
+    d->x1 = fminf(fmaxf(X1, 0.0f), fw);
+    d->x2 = fminf(fmaxf(X2, 0.0f), fw);
+    d->y1 = fminf(fmaxf(Y1, 0.0f), fh);
+    d->y2 = fminf(fmaxf(Y2, 0.0f), fh);
+}
+
+/* R3..R6 for one image: head -> dets[<= max_det] in frame pixels.  Returns kept count;
+ * *n_cand receives the candidate count before NMS. */
+int32_t orc_postprocess_image(const float* head, int32_t A, int32_t C, int32_t logits,
+                              float conf, float iou_thr, int32_t max_det, int32_t w, int32_t h,
+                              int32_t S, orc_det_t* dets, int32_t* n_cand) {
+    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * (size_t)(A > 0 ? A : 1));
+    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
+    int32_t n = orc_decode(head, A, C, logits, conf, cand);
+    orc_sort(cand, n);
+    int32_t k = orc_nms(cand, n, iou_thr, max_det, keep);
+    for (int32_t t = 0; t < k; ++t) {
+        dets[t] = cand[keep[t]];
+        orc_scale_back(&dets[t], w, h, S);
+    }
+    if (n_cand) *n_cand = n;
+    free(cand);
+    free(keep);
+    return k;
+}
+
+/* R7: integer crop rectangle of a frame-space box: rx0 = clamp(floor(X1), 0, w-1),
+ * rx1 = clamp(ceil(X2), rx0+1, w), same in y.  rect = {rx0, ry0, rx1, ry1}. */
+void orc_crop_rect(const orc_det_t* d, int32_t w, int32_t h, int32_t* rect) {
+    int64_t x0 = (int64_t)floorf(d->x1), y0 = (int64_t)floorf(d->y1);
+    int64_t x1 = (int64_t)ceilf(d->x2), y1 = (int64_t)ceilf(d->y2);
+    if (x0 < 0) x0 = 0;
+    if (x0 > w - 1) x0 = w - 1;
+    if (y0 < 0) y0 = 0;
+    if (y0 > h - 1) y0 = h - 1;
+    if (x1 < x0 + 1) x1 = x0 + 1;
+    if (x1 > w) x1 = w;
+    if (y1 < y0 + 1) y1 = y0 + 1;
+    if (y1 > h) y1 = h;
+    rect[0] = (int32_t)x0; rect[1] = (int32_t)y0; rect[2] = (int32_t)x1; rect[3] = (int32_t)y1;
+}
+
+/* R7: cut the rectangle, stretch it to ow x oh by R2, same plane order and /255 as the
+ * letterbox.  out: [3][oh][ow] half bits. */
+void orc_crop(const uint8_t* img, int32_t w, int32_t h, int32_t pitch, const orc_det_t* d,
+              int32_t ow, int32_t oh, int32_t swap_rb, uint16_t* out) {
+    int32_t r[4];
+    orc_crop_rect(d, w, h, r);
+    double* tmp = (double*)malloc(sizeof(double) * 3 * (size_t)ow * (size_t)oh);
+    orc_resize_f64(img, pitch, r[0], r[1], r[2] - r[0], r[3] - r[1], ow, oh, tmp);
+    size_t plane = (size_t)ow * (size_t)oh;
+    for (int p = 0; p < 3; ++p) {
+        int c = swap_rb ? 2 - p : p;
+        for (size_t i = 0; i < plane; ++i)
+            out[(size_t)p * plane + i] = orc_f64_to_half(tmp[(size_t)c * plane + i] / 255.0);
+    }
+    free(tmp);
+}
+
+/* R8: batch assembler for one branch.  m_n = number of frame n's kept detections whose
+ * class bit is set in class_mask (128 bits, bit k of word k/32); offsets = exclusive prefix
+ * sum, offsets[N] = total.  Item offsets[n]+j is the j-th such detection of frame n in NMS
+ * output order.  items receives (frame, det) pairs for the window
+ * [first_item, first_item + max_items); n_items = {packed, total}. */
+void orc_assemble(const orc_det_t* dets, const int32_t* counts, int32_t N, int32_t max_det,
+                  const uint32_t* class_mask, int32_t first_item, int32_t max_items,
+                  int32_t* offsets, int32_t* items, int32_t* n_items) {
+    int32_t run = 0, packed = 0;
+    offsets[0] = 0;
+    for (int32_t n = 0; n < N; ++n) {
+        for (int32_t j = 0; j < counts[n]; ++j) {
+            const orc_det_t* d = &dets[(size_t)n * (size_t)max_det + (size_t)j];
+            uint32_t k = (uint32_t)d->cls;
+            if (k < 128u && ((class_mask[k >> 5] >> (k & 31u)) & 1u)) {
+                if (run >= first_item && run - first_item < max_items) {
+                    items[2 * (size_t)(run - first_item)] = n;
+                    items[2 * (size_t)(run - first_item) + 1] = j;
+                    ++packed;
+                }
+                ++run;
+            }
+        }
+        offsets[n + 1] = run;
+    }
+    n_items[0] = packed;
+    n_items[1] = run;
+}
