@@ -1,0 +1,235 @@
+/*
+ * octo.h -- C ABI of the cascade-stage tensor library (CUDA, sm_100a).
+ *
+ * A "stage" is one model instance of a DNN cascade as the paper states it: it receives a
+ * batch of bz inputs, runs on an assigned execution stream and emits outputs that become
+ * the inputs of its downstream models (Section II, Eq. 1 and Table II: In_m / Out_m =
+ * "image - bounding box"; Section III-C "Inference Stream"; the traffic pipeline
+ * [Object Detect -> Vehicle Classify, Plate Detect] of Section I).  This library is the
+ * per-batch tensor work around the detector of such a stage:
+ *
+ *   octo_preprocess_batch   frames (BGR uint8)  -> letterboxed fp16 NCHW detector batch
+ *   [the caller runs the detector]
+ *   octo_postprocess_batch  detector head       -> per-frame detections (decode, confidence
+ *                                                  filter, class-aware NMS, frame pixels)
+ *   octo_crop_batch         detections + frames -> one downstream branch's fp16 batch
+ *                                                  (batch assembler + ROI crop-resize)
+ *
+ * The paper gives no formula for this work; the numeric rules are fixed in the comments
+ * below, and each has exactly one correct result.
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; everything else is host
+ *     memory.  The library never frees or retains caller buffers, except that the frames
+ *     passed to octo_preprocess_batch are read again by octo_crop_batch (see there).
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).  The three
+ *     batch calls only enqueue work on it and return; they never synchronise.
+ *   - A stage is not re-entrant: use it from one host thread and one stream at a time.
+ *   - Every function returns OCTO_OK (0) or a negative octo_status_t.  No exception
+ *     crosses the boundary and nothing aborts the process.  Conditions detected on the
+ *     device (non-finite head values, a wait that ran out) set bits in a status word read
+ *     with octo_stage_status.
+ */
+#ifndef OCTO_H_
+#define OCTO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define OCTO_API __attribute__((visibility("default")))
+#else
+#define OCTO_API
+#endif
+
+#define OCTO_MAX_BRANCHES 4
+#define OCTO_MAX_CLASSES 128
+#define OCTO_MAX_BATCH 512
+
+typedef enum {
+    OCTO_OK = 0,
+    OCTO_E_INVALID_ARG = -1,   /* null pointer, size out of range, bad configuration      */
+    OCTO_E_CAPACITY = -2,      /* n > max_batch, frame wider than the stage supports      */
+    OCTO_E_ALIGNMENT = -3,     /* pointer or pitch not a multiple of 16 bytes             */
+    OCTO_E_NO_PREPROCESS = -4, /* post/crop called before any octo_preprocess_batch       */
+    OCTO_E_CUDA = -5,          /* a CUDA runtime call failed (octo_last_cuda_error)       */
+    OCTO_E_DEVICE_TIMEOUT = -6,/* a bounded device-side wait gave up (status word)        */
+    OCTO_E_NO_POSTPROCESS = -7 /* crop called before octo_postprocess_batch of this batch */
+} octo_status_t;
+
+/* Bits of the device status word. */
+#define OCTO_STATUS_NONFINITE 0x1u      /* an examined head row held NaN/Inf and was dropped */
+#define OCTO_STATUS_TRUNCATED 0x2u      /* a crop window held fewer slots than items         */
+#define OCTO_STATUS_COPY_TIMEOUT 0x4u   /* a bulk-copy wait ran out; that tile was skipped    */
+#define OCTO_STATUS_BIG_NMS 0x8u        /* an image had more candidates than fit on chip and   */
+                                        /* took the slower global-memory path (informational)  */
+
+typedef struct octo_stage octo_stage_t; /* opaque; owned by the library */
+
+/* One downstream branch (e.g. vehicle classifier 224x224, plate detector 256x256).
+ * class_mask: bit k (word k/32, bit k%32) set => detections of class k feed this branch. */
+typedef struct {
+    int32_t out_w, out_h;   /* crop size; out_w must be a multiple of 8 */
+    uint32_t class_mask[4];
+} octo_branch_cfg_t;
+
+typedef struct {
+    int32_t device;         /* CUDA device ordinal                                          */
+    int32_t net_size;       /* S: side of the square detector input, multiple of 8 (640)    */
+    int32_t max_batch;      /* upper bound on n; sizes the workspace (<= OCTO_MAX_BATCH)    */
+    int32_t num_anchors;    /* A: rows of the head per image (25200 at S = 640)             */
+    int32_t num_classes;    /* C <= OCTO_MAX_CLASSES; a head row is 5 + C floats            */
+    int32_t head_is_logits; /* 1: obj / class values are logits; 0: probabilities           */
+    float conf_thresh;      /* candidate iff score > conf_thresh (strict)                   */
+    float iou_thresh;       /* suppress iff IoU > iou_thresh (strict)                       */
+    int32_t max_det;        /* detections kept per frame                                    */
+    int32_t pad_value;      /* canvas fill, 0..255 (114)                                    */
+    int32_t swap_rb;        /* 1: output plane 0 = input channel 2 (BGR -> RGB)             */
+    int32_t num_branches;   /* 1..OCTO_MAX_BRANCHES                                         */
+    octo_branch_cfg_t branch[OCTO_MAX_BRANCHES];
+} octo_stage_config_t;
+
+/* One source frame: interleaved 3-channel uint8 rows, pixel (y, x) at
+ * d_data + y * pitch_bytes + 3 * x.  d_data must be 16-byte aligned, pitch_bytes a multiple
+ * of 16 and >= 3 * width (rows are fetched with 16-byte bulk copies). */
+typedef struct {
+    const uint8_t* d_data;
+    int32_t width, height, pitch_bytes;
+    int32_t _pad;
+} octo_frame_t;
+
+/* One detection, 32 bytes.  Box in source-frame pixels, clamped to the frame. */
+typedef struct {
+    float x1, y1, x2, y2, score;
+    int32_t cls, anchor, _pad;
+} octo_det_t;
+
+/* One packed item of a branch batch: which detection it is and the integer source
+ * rectangle [rx0, rx1) x [ry0, ry1) that was resized into the slot. */
+typedef struct {
+    int32_t frame, det, rx0, ry0, rx1, ry1, _pad[2];
+} octo_item_t;
+
+typedef struct {
+    int64_t candidates;   /* rows that passed the confidence filter since the last get_stats */
+    int64_t kept;         /* detections after NMS since the last get_stats                   */
+    int64_t packed;       /* items written by the last crop call                            */
+    int64_t total_items;  /* items the last crop call's branch holds in total               */
+    uint32_t status_word; /* same as octo_stage_status                                      */
+    int32_t max_candidates_per_image;
+} octo_stage_stats_t;
+
+/*
+ * Create a stage on cfg->device and allocate its workspace (candidate keys
+ * max_batch * A * 8 bytes, per-branch item tables, counters).  Arguments are validated
+ * before any CUDA call, so OCTO_E_INVALID_ARG is reported even on a machine without a GPU.
+ * On success *out owns the workspace until octo_stage_destroy.
+ */
+OCTO_API int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** out);
+
+/* Free the workspace.  The caller must have synchronised the streams that used it. */
+OCTO_API int octo_stage_destroy(octo_stage_t* st);
+
+/*
+ * Letterbox n frames into the detector batch (stage input In_m of Table II).
+ *   frames          host array of n descriptors; device pixels stay owned by the caller and
+ *                   must remain valid and unchanged until the last octo_crop_batch of this
+ *                   batch has run.
+ *   d_out_f16_nchw  device, [n, 3, S, S] binary16, 16-byte aligned, fully overwritten.
+ * Rule: the longer side maps to S, the other to round-half-up(h*S/w) in integer arithmetic
+ * (at least 1); the image is centred, an odd remainder goes right/bottom; canvas =
+ * pad_value/255.  Bilinear, half-pixel centres: source x = (dx + 0.5) * w/nw - 0.5 clamped
+ * to [0, w-1], no antialiasing, raw 0..255 values; output = half(v / 255).  Plane order per
+ * swap_rb.  Also records the frame table used by the next two calls.
+ * Errors: OCTO_E_INVALID_ARG (null, n < 1, non-positive size, pitch < 3*width),
+ * OCTO_E_CAPACITY (n > max_batch), OCTO_E_ALIGNMENT, OCTO_E_CUDA.
+ */
+OCTO_API int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frames, int32_t n,
+                          void* d_out_f16_nchw, void* cuda_stream);
+
+/*
+ * Decode the detector head of the batch last given to octo_preprocess_batch (n must match)
+ * into detections (stage output Out_m of Table II; the per-frame count is what drives the
+ * downstream request rate, Section III-B Observation 1).
+ *   d_head    device, [n, A, 5 + C] float32 contiguous, rows (cx, cy, w, h, obj, class_0..)
+ *             with the box in letterbox pixels; 4-byte aligned.
+ *   d_dets    device, [n, max_det] records; entries [0, d_counts[i]) of frame i are written.
+ *   d_counts  device, [n] int32.
+ * Rules.  Candidate: every value of the row finite, w > 0, h > 0, k* = first maximal class
+ * value, score = fl(sigma(obj) * sigma(c_k*)) (or fl(obj * c_k*) for probabilities),
+ * score > conf_thresh.  sigma is a fixed sequence of binary32 operations (see the kernel
+ * source), not the platform expf, so scores are reproducible bit for bit.  Order: score
+ * descending, ties by lower anchor index.  NMS: walking that order, a candidate is kept iff
+ * no earlier KEPT candidate of the same class has IoU > iou_thresh, IoU evaluated in
+ * binary32 as inter / (area_a + area_b - inter) on letterbox-pixel corners
+ * x1 = cx - w/2 ...; at most max_det are kept.  Kept boxes are mapped to frame pixels,
+ * X = (x - pad_left) * fl(w / nw), clamped to [0, w] x [0, h].
+ * Errors: OCTO_E_INVALID_ARG, OCTO_E_NO_PREPROCESS, OCTO_E_CUDA.
+ */
+OCTO_API int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int32_t n,
+                           octo_det_t* d_dets, int32_t* d_counts, void* cuda_stream);
+
+/*
+ * Pack one branch's downstream batch (the model input that the scheduler's batch size bz of
+ * Algorithm 1 cuts into batches): batch assembler, then ROI crop-resize.
+ *   branch      index into cfg.branch.
+ *   first_item, max_items  window [first_item, first_item + max_items) of the branch's item
+ *               list; lets the caller cut the list into batches of bz.
+ *   d_out_f16   device, [max_items, 3, out_h, out_w] binary16, 16-byte aligned.  Item i of
+ *               the window is written to slot i - first_item; slots >= packed are untouched.
+ *   d_offsets   device, [n + 1] int32: exclusive prefix sum of the per-frame number of kept
+ *               detections whose class is in the branch's mask; d_offsets[n] = total.
+ *   d_n_items   device, [2] int32: {packed, total}.  total > first_item + max_items is not
+ *               an error (OCTO_STATUS_TRUNCATED is set).
+ * Item offsets[f] + j is the j-th masked detection of frame f in NMS output order.  Its
+ * rectangle is rx0 = clamp(floor(x1), 0, w-1), rx1 = clamp(ceil(x2), rx0 + 1, w), likewise
+ * in y; the rectangle is stretched to out_w x out_h with the same bilinear rule as the
+ * letterbox (taps clamped inside the rectangle), same plane order, /255, binary16.
+ * Uses the detections written by the last octo_postprocess_batch (d_dets must still be
+ * valid) and the frames of the last octo_preprocess_batch.
+ * Errors: OCTO_E_INVALID_ARG, OCTO_E_NO_PREPROCESS, OCTO_E_NO_POSTPROCESS, OCTO_E_CUDA.
+ */
+OCTO_API int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_item, int32_t max_items,
+                    void* d_out_f16, int32_t* d_offsets, int32_t* d_n_items, void* cuda_stream);
+
+/* Synchronise `cuda_stream`, then read (and keep) the device status word. */
+OCTO_API int octo_stage_status(octo_stage_t* st, uint32_t* status_word, void* cuda_stream);
+
+/* Clear the device status word (enqueued on the stream). */
+OCTO_API int octo_stage_clear_status(octo_stage_t* st, void* cuda_stream);
+
+/* Synchronise `cuda_stream`, then fill *stats from the stage's device counters; the
+ * candidate / kept / max counters restart from zero afterwards. */
+OCTO_API int octo_stage_get_stats(octo_stage_t* st, octo_stage_stats_t* stats, void* cuda_stream);
+
+/* Device pointer to the item table the last octo_crop_batch of `branch` built (entries
+ * [0, packed)); stage-owned, valid until the next crop call on that branch. */
+OCTO_API int octo_stage_item_table(octo_stage_t* st, int32_t branch, const octo_item_t** d_items);
+
+/* Synchronise `cuda_stream`, then copy the first `count` entries of that table to host
+ * memory (count <= max_batch * max_det). */
+OCTO_API int octo_stage_copy_items(octo_stage_t* st, int32_t branch, octo_item_t* items_out, int32_t count,
+                                   void* cuda_stream);
+
+/* Bytes of device memory the stage holds. */
+OCTO_API int64_t octo_stage_workspace_bytes(const octo_stage_t* st);
+
+/* Number of kernels the stage has launched since creation (for launch accounting). */
+OCTO_API int64_t octo_stage_launch_count(const octo_stage_t* st);
+
+/* Text of a status code; never NULL. */
+OCTO_API const char* octo_strerror(int code);
+
+/* Text of the last CUDA error a call on this thread reported as OCTO_E_CUDA. */
+OCTO_API const char* octo_last_cuda_error(void);
+
+/* Library version, "major.minor". */
+OCTO_API const char* octo_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OCTO_H_ */

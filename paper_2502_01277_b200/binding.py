@@ -1,0 +1,304 @@
+"""ctypes binding of the C-ABI library (include/octo.h).  Argument marshalling only: every
+step of the stage runs in the CUDA kernels of liboctostage.so.  There is no CPU fallback;
+importing the library fails loudly if the shared object has not been built.
+
+Function names match the C ABI: octo_stage_create, octo_preprocess_batch,
+octo_postprocess_batch, octo_crop_batch, ...  `Stage` is a thin convenience object over
+them for callers that hold torch tensors (torch provides device memory and streams only).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liboctostage.so")
+
+OCTO_MAX_BRANCHES = 4
+OCTO_MAX_BATCH = 512
+
+OCTO_OK = 0
+OCTO_E_INVALID_ARG = -1
+OCTO_E_CAPACITY = -2
+OCTO_E_ALIGNMENT = -3
+OCTO_E_NO_PREPROCESS = -4
+OCTO_E_CUDA = -5
+OCTO_E_DEVICE_TIMEOUT = -6
+OCTO_E_NO_POSTPROCESS = -7
+
+OCTO_STATUS_NONFINITE = 0x1
+OCTO_STATUS_TRUNCATED = 0x2
+OCTO_STATUS_COPY_TIMEOUT = 0x4
+OCTO_STATUS_BIG_NMS = 0x8
+
+EXPORTS = (
+    "octo_stage_create", "octo_stage_destroy", "octo_preprocess_batch", "octo_postprocess_batch",
+    "octo_crop_batch", "octo_stage_status", "octo_stage_clear_status", "octo_stage_get_stats",
+    "octo_stage_item_table", "octo_stage_copy_items", "octo_stage_workspace_bytes", "octo_stage_launch_count",
+    "octo_strerror", "octo_last_cuda_error", "octo_version",
+)
+
+
+class BranchCfg(ctypes.Structure):
+    _fields_ = [("out_w", ctypes.c_int32), ("out_h", ctypes.c_int32), ("class_mask", ctypes.c_uint32 * 4)]
+
+
+class StageConfig(ctypes.Structure):
+    _fields_ = [
+        ("device", ctypes.c_int32), ("net_size", ctypes.c_int32), ("max_batch", ctypes.c_int32),
+        ("num_anchors", ctypes.c_int32), ("num_classes", ctypes.c_int32),
+        ("head_is_logits", ctypes.c_int32), ("conf_thresh", ctypes.c_float),
+        ("iou_thresh", ctypes.c_float), ("max_det", ctypes.c_int32), ("pad_value", ctypes.c_int32),
+        ("swap_rb", ctypes.c_int32), ("num_branches", ctypes.c_int32),
+        ("branch", BranchCfg * OCTO_MAX_BRANCHES),
+    ]
+
+
+class Frame(ctypes.Structure):
+    _fields_ = [("d_data", ctypes.c_void_p), ("width", ctypes.c_int32), ("height", ctypes.c_int32),
+                ("pitch_bytes", ctypes.c_int32), ("_pad", ctypes.c_int32)]
+
+
+class StageStats(ctypes.Structure):
+    _fields_ = [("candidates", ctypes.c_int64), ("kept", ctypes.c_int64), ("packed", ctypes.c_int64),
+                ("total_items", ctypes.c_int64), ("status_word", ctypes.c_uint32),
+                ("max_candidates_per_image", ctypes.c_int32)]
+
+
+DET_DTYPE = np.dtype([("x1", "<f4"), ("y1", "<f4"), ("x2", "<f4"), ("y2", "<f4"), ("score", "<f4"),
+                      ("cls", "<i4"), ("anchor", "<i4"), ("pad", "<i4")])
+ITEM_DTYPE = np.dtype([("frame", "<i4"), ("det", "<i4"), ("rx0", "<i4"), ("ry0", "<i4"),
+                       ("rx1", "<i4"), ("ry1", "<i4"), ("pad0", "<i4"), ("pad1", "<i4")])
+
+_lib = None
+
+
+class OctoError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        detail = ""
+        if _lib is not None:
+            detail = _lib.octo_strerror(code).decode()
+            if code == OCTO_E_CUDA:
+                detail += " (" + _lib.octo_last_cuda_error().decode() + ")"
+        super().__init__(f"{where} failed with status {code}: {detail}")
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """dlopen liboctostage.so and declare the prototypes.  Raises if it is missing."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise ImportError(
+            f"{p} not found: build the CUDA library first (python -m paper_2502_01277_b200.build). "
+            "There is no fallback path.")
+    lib = ctypes.CDLL(p)
+    vp, i32 = ctypes.c_void_p, ctypes.c_int32
+    lib.octo_stage_create.argtypes = [ctypes.POINTER(StageConfig), ctypes.POINTER(vp)]
+    lib.octo_stage_destroy.argtypes = [vp]
+    lib.octo_preprocess_batch.argtypes = [vp, ctypes.POINTER(Frame), i32, vp, vp]
+    lib.octo_postprocess_batch.argtypes = [vp, vp, i32, vp, vp, vp]
+    lib.octo_crop_batch.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.octo_stage_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+    lib.octo_stage_clear_status.argtypes = [vp, vp]
+    lib.octo_stage_get_stats.argtypes = [vp, ctypes.POINTER(StageStats), vp]
+    lib.octo_stage_item_table.argtypes = [vp, i32, ctypes.POINTER(vp)]
+    lib.octo_stage_copy_items.argtypes = [vp, i32, vp, i32, vp]
+    lib.octo_stage_copy_items.restype = ctypes.c_int
+    lib.octo_stage_workspace_bytes.argtypes = [vp]
+    lib.octo_stage_workspace_bytes.restype = ctypes.c_int64
+    lib.octo_stage_launch_count.argtypes = [vp]
+    lib.octo_stage_launch_count.restype = ctypes.c_int64
+    for name in ("octo_strerror", "octo_last_cuda_error", "octo_version"):
+        getattr(lib, name).restype = ctypes.c_char_p
+    lib.octo_strerror.argtypes = [ctypes.c_int]
+    for name in ("octo_stage_create", "octo_stage_destroy", "octo_preprocess_batch",
+                 "octo_postprocess_batch", "octo_crop_batch", "octo_stage_status",
+                 "octo_stage_clear_status", "octo_stage_get_stats", "octo_stage_item_table"):
+        getattr(lib, name).restype = ctypes.c_int
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def make_config(*, device: int = 0, net_size: int = 640, max_batch: int = 8, num_anchors: int = 25200,
+                num_classes: int = 80, head_is_logits: bool = True, conf_thresh: float = 0.25,
+                iou_thresh: float = 0.45, max_det: int = 300, pad_value: int = 114, swap_rb: bool = True,
+                branches: Sequence[Tuple[int, int]] = ((224, 224),),
+                class_masks: Optional[Sequence[Sequence[int]]] = None) -> StageConfig:
+    cfg = StageConfig()
+    cfg.device, cfg.net_size, cfg.max_batch = device, net_size, max_batch
+    cfg.num_anchors, cfg.num_classes = num_anchors, num_classes
+    cfg.head_is_logits = 1 if head_is_logits else 0
+    cfg.conf_thresh, cfg.iou_thresh = conf_thresh, iou_thresh
+    cfg.max_det, cfg.pad_value, cfg.swap_rb = max_det, pad_value, 1 if swap_rb else 0
+    cfg.num_branches = len(branches)
+    for b, (ow, oh) in enumerate(branches[:OCTO_MAX_BRANCHES]):
+        cfg.branch[b].out_w, cfg.branch[b].out_h = ow, oh
+        mask = class_masks[b] if class_masks is not None else (0xFFFFFFFF,) * 4
+        for k in range(4):
+            cfg.branch[b].class_mask[k] = int(mask[k]) & 0xFFFFFFFF
+    return cfg
+
+
+# ---- thin functional layer: same names as the C ABI ------------------------------------------
+
+def octo_stage_create(cfg: StageConfig) -> ctypes.c_void_p:
+    lib = load_library()
+    h = ctypes.c_void_p()
+    rc = lib.octo_stage_create(ctypes.byref(cfg), ctypes.byref(h))
+    if rc != OCTO_OK:
+        raise OctoError(rc, "octo_stage_create")
+    return h
+
+
+def octo_stage_destroy(handle) -> None:
+    load_library().octo_stage_destroy(handle)
+
+
+def octo_preprocess_batch(handle, frames: Sequence[Tuple[int, int, int, int]], d_out: int, stream: int = 0) -> None:
+    """frames: (device_ptr, width, height, pitch_bytes) per frame."""
+    n = len(frames)
+    arr = (Frame * max(n, 1))()
+    for i, (ptr, w, h, pitch) in enumerate(frames):
+        arr[i].d_data, arr[i].width, arr[i].height, arr[i].pitch_bytes = ptr, w, h, pitch
+    rc = load_library().octo_preprocess_batch(handle, arr, n, d_out, stream)
+    if rc != OCTO_OK:
+        raise OctoError(rc, "octo_preprocess_batch")
+
+
+def octo_postprocess_batch(handle, d_head: int, n: int, d_dets: int, d_counts: int, stream: int = 0) -> None:
+    rc = load_library().octo_postprocess_batch(handle, d_head, n, d_dets, d_counts, stream)
+    if rc != OCTO_OK:
+        raise OctoError(rc, "octo_postprocess_batch")
+
+
+def octo_crop_batch(handle, branch: int, first_item: int, max_items: int, d_out: int, d_offsets: int,
+                    d_n_items: int, stream: int = 0) -> None:
+    rc = load_library().octo_crop_batch(handle, branch, first_item, max_items, d_out, d_offsets, d_n_items, stream)
+    if rc != OCTO_OK:
+        raise OctoError(rc, "octo_crop_batch")
+
+
+def octo_stage_status(handle, stream: int = 0) -> int:
+    w = ctypes.c_uint32(0)
+    rc = load_library().octo_stage_status(handle, ctypes.byref(w), stream)
+    if rc not in (OCTO_OK, OCTO_E_DEVICE_TIMEOUT):
+        raise OctoError(rc, "octo_stage_status")
+    return int(w.value)
+
+
+def octo_stage_get_stats(handle, stream: int = 0) -> dict:
+    s = StageStats()
+    rc = load_library().octo_stage_get_stats(handle, ctypes.byref(s), stream)
+    if rc != OCTO_OK:
+        raise OctoError(rc, "octo_stage_get_stats")
+    return {k: int(getattr(s, k)) for k, _ in StageStats._fields_}
+
+
+# ---- convenience object for torch callers ----------------------------------------------------
+
+class Stage:
+    """Owns one octo_stage_t and the torch tensors a caller usually wants around it."""
+
+    def __init__(self, **cfg_kwargs):
+        import torch  # device memory and streams only
+        self._torch = torch
+        self.cfg = make_config(**cfg_kwargs)
+        self.handle = octo_stage_create(self.cfg)
+        self.device = torch.device("cuda", self.cfg.device)
+        self.n = 0
+        self._frames_keepalive: List = []
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            octo_stage_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _stream(self, stream) -> int:
+        if stream is None:
+            stream = self._torch.cuda.current_stream(self.device)
+        return int(stream.cuda_stream)
+
+    def preprocess(self, frames, sizes, out=None, stream=None):
+        """frames: list of uint8 CUDA tensors [h, pitch]; sizes: (w, h) per frame.
+        Returns the fp16 [n, 3, S, S] batch."""
+        t = self._torch
+        n, s = len(frames), self.cfg.net_size
+        if out is None:
+            out = t.empty((n, 3, s, s), dtype=t.float16, device=self.device)
+        desc = [(f.data_ptr(), w, h, f.stride(0)) for f, (w, h) in zip(frames, sizes)]
+        octo_preprocess_batch(self.handle, desc, out.data_ptr(), self._stream(stream))
+        self._frames_keepalive = list(frames)
+        self.n = n
+        return out
+
+    def postprocess(self, head, dets=None, counts=None, stream=None):
+        """head: float32 CUDA tensor [n, A, 5+C].  Returns (dets uint8 [n, max_det, 32], counts int32 [n])."""
+        t = self._torch
+        n = head.shape[0]
+        if dets is None:
+            dets = t.empty((n, self.cfg.max_det, 32), dtype=t.uint8, device=self.device)
+        if counts is None:
+            counts = t.empty((n,), dtype=t.int32, device=self.device)
+        octo_postprocess_batch(self.handle, head.data_ptr(), n, dets.data_ptr(), counts.data_ptr(),
+                               self._stream(stream))
+        self._dets_keepalive = dets
+        return dets, counts
+
+    def crop(self, branch, max_items, first_item=0, out=None, offsets=None, n_items=None, stream=None):
+        """Returns (crops fp16 [max_items, 3, oh, ow], offsets int32 [n+1], n_items int32 [2])."""
+        t = self._torch
+        ow, oh = self.cfg.branch[branch].out_w, self.cfg.branch[branch].out_h
+        if out is None:
+            out = t.empty((max(max_items, 1), 3, oh, ow), dtype=t.float16, device=self.device)
+        if offsets is None:
+            offsets = t.empty((self.n + 1,), dtype=t.int32, device=self.device)
+        if n_items is None:
+            n_items = t.empty((2,), dtype=t.int32, device=self.device)
+        octo_crop_batch(self.handle, branch, first_item, max_items, out.data_ptr(), offsets.data_ptr(),
+                        n_items.data_ptr(), self._stream(stream))
+        return out, offsets, n_items
+
+    def item_table(self, branch: int, count: int) -> np.ndarray:
+        """Host copy of the first `count` entries of the branch's item table (synchronises)."""
+        host = np.zeros(max(count, 1), dtype=ITEM_DTYPE)
+        rc = load_library().octo_stage_copy_items(self.handle, branch, host.ctypes.data, count, self._stream(None))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_stage_copy_items")
+        return host[:count]
+
+    def status(self, stream=None) -> int:
+        return octo_stage_status(self.handle, self._stream(stream))
+
+    def clear_status(self, stream=None) -> None:
+        load_library().octo_stage_clear_status(self.handle, self._stream(stream))
+
+    def stats(self, stream=None) -> dict:
+        return octo_stage_get_stats(self.handle, self._stream(stream))
+
+    @property
+    def launch_count(self) -> int:
+        return int(load_library().octo_stage_launch_count(self.handle))
+
+    @property
+    def workspace_bytes(self) -> int:
+        return int(load_library().octo_stage_workspace_bytes(self.handle))
+
+
+def dets_to_numpy(dets, counts) -> Tuple[np.ndarray, np.ndarray]:
+    """Device (dets uint8 [n, max_det, 32], counts) -> host structured array + counts."""
+    d = dets.cpu().numpy().view(DET_DTYPE).reshape(dets.shape[0], dets.shape[1])
+    return d, counts.cpu().numpy()

@@ -1,0 +1,192 @@
+// Shared device-side definitions of the cascade-stage kernels (sm_100a).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace octo {
+
+// One frame of the current batch plus its letterbox geometry (computed on the host in exact
+// integer arithmetic).  Passed to kernels BY VALUE inside a FrameTable (kernel parameter
+// space), so no host->device table copy sits on the critical path of a batch.
+struct FrameDesc {
+    const uint8_t* data;
+    int32_t w, h, pitch;
+    int32_t nw, nh, pad_l, pad_t;
+    float gx, gy;  // fl(w / nw), fl(h / nh): scale-back gains
+    int32_t _pad;
+};
+static_assert(sizeof(FrameDesc) == 48, "FrameDesc layout");
+
+template <int CAP>
+struct FrameTable {
+    FrameDesc f[CAP];
+};
+
+struct BranchDesc {
+    int32_t out_w, out_h;
+    uint32_t class_mask[4];
+};
+
+// Device counters of a stage (one allocation, zeroed at creation).
+struct StageCounters {
+    unsigned long long candidates;
+    unsigned long long kept;
+    unsigned int status;
+    int max_cand;
+    int packed;
+    int total_items;
+};
+
+constexpr int kKeyAnchorBits = 25;  // anchor index field of a candidate key
+constexpr unsigned long long kKeySentinel = ~0ull;
+
+// ---------------------------------------------------------------------------------------
+// Exact source coordinate of destination index d when `src` samples are resized to `dst`
+// (half-pixel centres): s = ((2d + 1) * src - dst) / (2 * dst), clamped to [0, src - 1].
+// Returns i0 = floor(s) and the remainder r in [0, 2*dst) with frac = r / (2*dst); r == 0
+// when clamped.  The quotient comes from a float estimate corrected in integers, which is
+// exact for every value that fits 31 bits.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void src_coord(int d, int src, int dst, float inv_den, int& i0, int& rem) {
+    const int den = 2 * dst;
+    int num = (2 * d + 1) * src - dst;
+    if (num <= 0) { i0 = 0; rem = 0; return; }
+    int q = __float2int_rz(__int2float_rn(num) * inv_den);
+    int r = num - q * den;
+    if (r < 0) { q -= 1; r += den; }
+    else if (r >= den) { q += 1; r -= den; }
+    if (q >= src - 1) { i0 = src - 1; rem = 0; return; }
+    i0 = q; rem = r;
+}
+
+// Six consecutive bytes (two BGR pixels) starting at byte offset `o` of a 4-byte aligned
+// row of 32-bit words; `last_word` bounds the word index so nothing past the row is read.
+__device__ __forceinline__ void load6(const uint32_t* __restrict__ row, int o, int last_word,
+                                      uint32_t& lo, uint32_t& hi) {
+    const int wi = o >> 2;
+    const int sh = (o & 3) * 8;
+    const uint32_t a = row[wi];
+    const uint32_t b = row[min(wi + 1, last_word)];
+    const uint32_t c = row[min(wi + 2, last_word)];
+    lo = __funnelshift_r(a, b, sh);  // bytes o .. o+3
+    hi = __funnelshift_r(b, c, sh);  // bytes o+4 .. o+7
+}
+
+__device__ __forceinline__ float byte_f(uint32_t w, int i) {
+    return __uint2float_rn((w >> (8 * i)) & 0xffu);
+}
+
+// Horizontal lerp of one row's two taps for the three channels; fx == 0 skips the second tap.
+__device__ __forceinline__ void row_taps(uint32_t lo, uint32_t hi, float fx, bool lerp_x,
+                                         float& c0, float& c1, float& c2) {
+    c0 = byte_f(lo, 0);
+    c1 = byte_f(lo, 1);
+    c2 = byte_f(lo, 2);
+    if (lerp_x) {
+        const float d0 = byte_f(lo, 3), d1 = byte_f(hi, 0), d2 = byte_f(hi, 1);
+        c0 = fmaf(fx, d0 - c0, c0);
+        c1 = fmaf(fx, d1 - c1, c1);
+        c2 = fmaf(fx, d2 - c2, c2);
+    }
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
+    __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// ---------------------------------------------------------------------------------------
+// mbarrier + bulk-copy (TMA engine, untiled) helpers.  Every wait is bounded.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Returns false if the phase did not complete within the iteration limit.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, int limit = 1 << 22) {
+    for (int i = 0; i < limit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// Global -> shared bulk copy; both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(dst_smem)),
+        "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// ---------------------------------------------------------------------------------------
+// Fixed binary32 arithmetic shared by decode and NMS.  Every operation is an explicitly
+// rounded intrinsic so that compiler contraction cannot change a bit.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ bool finite_f(float v) { return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u; }
+
+// Logistic function: clamp to [-30, 30]; n = rint(z*log2 e); r = z - n*ln2 (two fused steps
+// with a hi/lo split of ln2); degree-7 Taylor polynomial of exp(r) by Horner; scale by 2^n
+// through the exponent field; 1 / (1 + e) with IEEE add and divide.
+__device__ __forceinline__ float sigmoid_fixed(float x) {
+    const float t = fminf(fmaxf(x, -30.0f), 30.0f);
+    const float z = -t;
+    const float n = rintf(__fmul_rn(z, 0x1.715476p+0f));
+    float r = __fmaf_rn(n, -0x1.62e4p-1f, z);
+    r = __fmaf_rn(n, -0x1.7f7d1cp-20f, r);
+    float p = 0x1.a01a02p-13f;
+    p = __fmaf_rn(p, r, 0x1.6c16c2p-10f);
+    p = __fmaf_rn(p, r, 0x1.111112p-7f);
+    p = __fmaf_rn(p, r, 0x1.555556p-5f);
+    p = __fmaf_rn(p, r, 0x1.555556p-3f);
+    p = __fmaf_rn(p, r, 0.5f);
+    p = __fmaf_rn(p, r, 1.0f);
+    p = __fmaf_rn(p, r, 1.0f);
+    const float two_n = __int_as_float((__float2int_rn(n) + 127) << 23);
+    const float e = __fmul_rn(p, two_n);
+    return __fdiv_rn(1.0f, __fadd_rn(1.0f, e));
+}
+
+// Corners of a head row's box: x1 = cx - 0.5*w, x2 = cx + 0.5*w (0.5*w is exact).
+__device__ __forceinline__ float4 box_corners(float cx, float cy, float bw, float bh) {
+    const float hw = __fmul_rn(0.5f, bw), hh = __fmul_rn(0.5f, bh);
+    return make_float4(__fsub_rn(cx, hw), __fsub_rn(cy, hh), __fadd_rn(cx, hw), __fadd_rn(cy, hh));
+}
+
+// IoU, operation by operation: inter / ((area_a + area_b) - inter), 0 if the union is empty.
+__device__ __forceinline__ float iou_fixed(const float4 a, const float4 b) {
+    float iw = __fsub_rn(fminf(a.z, b.z), fmaxf(a.x, b.x));
+    float ih = __fsub_rn(fminf(a.w, b.w), fmaxf(a.y, b.y));
+    iw = fmaxf(iw, 0.0f);
+    ih = fmaxf(ih, 0.0f);
+    const float inter = __fmul_rn(iw, ih);
+    const float area_a = __fmul_rn(__fsub_rn(a.z, a.x), __fsub_rn(a.w, a.y));
+    const float area_b = __fmul_rn(__fsub_rn(b.z, b.x), __fsub_rn(b.w, b.y));
+    const float uni = __fsub_rn(__fadd_rn(area_a, area_b), inter);
+    return uni > 0.0f ? __fdiv_rn(inter, uni) : 0.0f;
+}
+
+}  // namespace octo

@@ -1,0 +1,109 @@
+// Decode + confidence filter + compaction of a YOLOv5-layout head [n, A, 5 + C] fp32.
+//
+// HBM-bound scan.  For logit heads sigma <= 1 makes sigma(obj) > conf a necessary condition
+// for score = fl(sigma(obj) * sigma(cls)) > conf, so the scan reads only the obj value of
+// each 340-byte row (one DRAM sector) and fetches the whole row, coalesced across the warp,
+// for the few anchors that pass.  Probability heads are read densely.  A passing row is
+// reduced by the warp (finite check, first-maximum class), scored in the fixed binary32
+// sequence and appended to the image's key list with one atomic; the key carries class,
+// inverted score bits and anchor, so later steps need nothing else from this kernel and the
+// nondeterministic append order is erased by the sort.
+#include "octo_common.cuh"
+#include "octo_kernels.h"
+
+namespace octo {
+
+constexpr int kDecThreads = 256;
+constexpr int kDecPerThread = 4;  // anchors per thread
+constexpr int kDecPerCta = kDecThreads * kDecPerThread;
+
+__global__ void __launch_bounds__(kDecThreads)
+decode_kernel(const float* __restrict__ head, int A, int C, int logits, float conf, int key_stride,
+              unsigned long long* __restrict__ keys, int* __restrict__ cand_count,
+              unsigned int* __restrict__ status) {
+    const int img = blockIdx.y;
+    const int row_len = 5 + C;
+    const float* __restrict__ hbase = head + (size_t)img * (size_t)A * (size_t)row_len;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    // each warp owns kDecPerThread consecutive groups of 32 anchors
+    const int a_warp = blockIdx.x * kDecPerCta + warp * (32 * kDecPerThread);
+
+    float obj[kDecPerThread];
+#pragma unroll
+    for (int u = 0; u < kDecPerThread; ++u) {
+        const int a = a_warp + u * 32 + lane;
+        obj[u] = (logits && a < A) ? __ldg(hbase + (size_t)a * row_len + 4) : 0.0f;
+    }
+    bool nonfinite_seen = false;
+#pragma unroll
+    for (int u = 0; u < kDecPerThread; ++u) {
+        const int a = a_warp + u * 32 + lane;
+        bool pass = a < A;
+        if (logits && pass) {
+            const bool fin = finite_f(obj[u]);
+            nonfinite_seen |= !fin;
+            pass = fin && sigmoid_fixed(obj[u]) > conf;
+        }
+        unsigned todo = __ballot_sync(0xffffffffu, pass);
+        while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const int ra = a_warp + u * 32 + src;
+            const float* __restrict__ row = hbase + (size_t)ra * row_len;
+            // the warp reads the row; lane l holds elements l, l+32, l+64, ...
+            bool fin = true;
+            float best = -INFINITY;
+            int best_k = 0x7fffffff;
+            float e0 = 0.0f;
+#pragma unroll
+            for (int j = 0; j < (5 + 128 + 31) / 32; ++j) {
+                const int e = lane + 32 * j;
+                if (e < row_len) {
+                    const float v = __ldg(row + e);
+                    if (j == 0) e0 = v;
+                    fin &= finite_f(v);
+                    if (e >= 5 && v > best) { best = v; best_k = e - 5; }
+                }
+            }
+            fin = __all_sync(0xffffffffu, fin);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+                const int ok = __shfl_xor_sync(0xffffffffu, best_k, off);
+                if (ov > best || (ov == best && ok < best_k)) { best = ov; best_k = ok; }
+            }
+            const float cx = __shfl_sync(0xffffffffu, e0, 0);
+            const float cy = __shfl_sync(0xffffffffu, e0, 1);
+            const float bw = __shfl_sync(0xffffffffu, e0, 2);
+            const float bh = __shfl_sync(0xffffffffu, e0, 3);
+            const float ob = __shfl_sync(0xffffffffu, e0, 4);
+            (void)cx; (void)cy;
+            if (!fin) { nonfinite_seen = true; continue; }
+            if (lane == 0 && bw > 0.0f && bh > 0.0f) {
+                const float score = logits ? __fmul_rn(sigmoid_fixed(ob), sigmoid_fixed(best))
+                                           : __fmul_rn(ob, best);
+                if (score > conf) {
+                    const int slot = atomicAdd(cand_count + img, 1);
+                    const unsigned long long key = ((unsigned long long)(unsigned)best_k << 57) |
+                                                   ((unsigned long long)(~__float_as_uint(score)) << kKeyAnchorBits) |
+                                                   (unsigned long long)(unsigned)ra;
+                    if (slot < key_stride) keys[(size_t)img * key_stride + slot] = key;
+                }
+            }
+        }
+    }
+    if (__any_sync(0xffffffffu, nonfinite_seen) && lane == 0) atomicOr(status, 0x1u);
+}
+
+cudaError_t launch_decode(const float* d_head, int n, int A, int C, int logits, float conf, int key_stride,
+                          unsigned long long* d_keys, int* d_cand_count, unsigned int* d_status,
+                          cudaStream_t stream) {
+    // d_cand_count is zero on entry: zeroed at stage creation and re-zeroed by the NMS kernel.
+    dim3 grid((A + kDecPerCta - 1) / kDecPerCta, n);
+    decode_kernel<<<grid, kDecThreads, 0, stream>>>(d_head, A, C, logits, conf, key_stride, d_keys, d_cand_count,
+                                                   d_status);
+    return cudaGetLastError();
+}
+
+}  // namespace octo

@@ -1,0 +1,67 @@
+// Internal launcher interface between the stage object (octo_stage.cu) and the kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "octo.h"
+#include "octo_common.cuh"
+
+namespace octo {
+
+typedef octo_det_t octo_det_rec;
+
+struct BranchMasks {
+    uint32_t m[OCTO_MAX_BRANCHES][4];
+};
+
+struct NmsArgs {
+    const FrameDesc* frames;  // host
+    int n;
+    const float* d_head;
+    int A, C;
+    float iou_thr;
+    int max_det, key_stride;
+    unsigned long long* d_keys;
+    float4* d_boxes;
+    int* d_cand_count;
+    octo_det_t* d_dets;
+    int* d_counts;
+    int num_branches;
+    BranchMasks masks;
+    int* d_bcount;
+    int* d_bidx;
+    int max_batch;
+    StageCounters* d_ctr;
+};
+
+struct CropArgs {
+    const FrameDesc* frames;  // host
+    int n;
+    int max_det, first_item, max_items;
+    const int* d_bcount;  // this branch's [max_batch]
+    const int* d_bidx;    // this branch's [max_batch][max_det]
+    const octo_det_t* d_dets;
+    int* d_offsets;
+    int* d_n_items;
+    octo_item_t* d_items;
+    void* d_out;
+    int out_w, out_h, swap_rb, sm_count;
+    StageCounters* d_ctr;
+};
+
+// Opt the kernels of every table capacity into the shared memory they need (current device).
+cudaError_t prepare_letterbox();
+cudaError_t prepare_nms();
+
+cudaError_t launch_letterbox(const FrameDesc* frames, int n, void* d_out, int S, int max_w, int pad_value,
+                             int swap_rb, unsigned int* d_status, cudaStream_t stream);
+cudaError_t launch_decode(const float* d_head, int n, int A, int C, int logits, float conf, int key_stride,
+                          unsigned long long* d_keys, int* d_cand_count, unsigned int* d_status,
+                          cudaStream_t stream);
+cudaError_t launch_nms(const NmsArgs& a, cudaStream_t stream);
+cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream);
+
+constexpr int kLetterboxMaxWidth = 8192;  // widest frame the row staging supports
+
+}  // namespace octo

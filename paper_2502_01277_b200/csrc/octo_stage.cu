@@ -1,0 +1,353 @@
+// Stage object and the extern "C" boundary (see include/octo.h for the contract).
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "octo.h"
+#include "octo_kernels.h"
+
+using namespace octo;
+
+struct octo_stage {
+    octo_stage_config_t cfg;
+    int sm_count;
+    int key_stride;  // candidate slots per image: next power of two >= A
+    // device workspace
+    unsigned long long* d_keys;
+    float4* d_boxes;
+    int* d_cand_count;
+    int* d_bcount;  // [branches][max_batch]
+    int* d_bidx;    // [branches][max_batch][max_det]
+    octo_item_t* d_items[OCTO_MAX_BRANCHES];
+    StageCounters* d_ctr;
+    int64_t workspace_bytes;
+    // host state of the current batch
+    FrameDesc frames[OCTO_MAX_BATCH];
+    int n_frames;
+    int max_w;
+    bool have_dets;
+    const octo_det_t* d_dets;
+    int64_t launches;
+};
+
+static thread_local char g_cuda_err[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+    return OCTO_E_CUDA;
+}
+#define OCTO_CUDA(call)                                     \
+    do {                                                    \
+        cudaError_t e__ = (call);                           \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+    } while (0)
+
+static int validate_config(const octo_stage_config_t* c) {
+    if (!c) return OCTO_E_INVALID_ARG;
+    if (c->device < 0) return OCTO_E_INVALID_ARG;
+    if (c->net_size < 8 || c->net_size > 4096 || (c->net_size & 7)) return OCTO_E_INVALID_ARG;
+    if (c->max_batch < 1 || c->max_batch > OCTO_MAX_BATCH) return OCTO_E_INVALID_ARG;
+    if (c->num_anchors < 1 || c->num_anchors > (1 << 24)) return OCTO_E_INVALID_ARG;
+    if (c->num_classes < 1 || c->num_classes > OCTO_MAX_CLASSES) return OCTO_E_INVALID_ARG;
+    if (c->head_is_logits != 0 && c->head_is_logits != 1) return OCTO_E_INVALID_ARG;
+    if (!(c->conf_thresh >= 0.0f) || !(c->conf_thresh <= 1.0f)) return OCTO_E_INVALID_ARG;
+    if (!(c->iou_thresh >= 0.0f) || !(c->iou_thresh <= 1.0f)) return OCTO_E_INVALID_ARG;
+    if (c->max_det < 1 || c->max_det > 65536) return OCTO_E_INVALID_ARG;
+    if (c->pad_value < 0 || c->pad_value > 255) return OCTO_E_INVALID_ARG;
+    if (c->swap_rb != 0 && c->swap_rb != 1) return OCTO_E_INVALID_ARG;
+    if (c->num_branches < 1 || c->num_branches > OCTO_MAX_BRANCHES) return OCTO_E_INVALID_ARG;
+    for (int b = 0; b < c->num_branches; ++b) {
+        const octo_branch_cfg_t& br = c->branch[b];
+        if (br.out_w < 8 || br.out_w > 2048 || (br.out_w & 7)) return OCTO_E_INVALID_ARG;
+        if (br.out_h < 1 || br.out_h > 2048) return OCTO_E_INVALID_ARG;
+    }
+    return OCTO_OK;
+}
+
+template <typename T>
+static cudaError_t dev_alloc(T** p, size_t count, int64_t* total) {
+    const size_t bytes = sizeof(T) * (count ? count : 1);
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes);
+    if (e == cudaSuccess) {
+        *total += (int64_t)bytes;
+        e = cudaMemset(*p, 0, bytes);
+    }
+    return e;
+}
+
+static void free_all(octo_stage* st) {
+    cudaFree(st->d_keys);
+    cudaFree(st->d_boxes);
+    cudaFree(st->d_cand_count);
+    cudaFree(st->d_bcount);
+    cudaFree(st->d_bidx);
+    for (int b = 0; b < OCTO_MAX_BRANCHES; ++b) cudaFree(st->d_items[b]);
+    cudaFree(st->d_ctr);
+}
+
+extern "C" int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** out) {
+    if (!out) return OCTO_E_INVALID_ARG;
+    *out = nullptr;
+    int rc = validate_config(cfg);
+    if (rc != OCTO_OK) return rc;
+
+    int ndev = 0;
+    OCTO_CUDA(cudaGetDeviceCount(&ndev));
+    if (cfg->device >= ndev) return OCTO_E_INVALID_ARG;
+    OCTO_CUDA(cudaSetDevice(cfg->device));
+
+    octo_stage* st = new (std::nothrow) octo_stage();
+    if (!st) return OCTO_E_INVALID_ARG;
+    memset(st, 0, sizeof(*st));
+    st->cfg = *cfg;
+    OCTO_CUDA(cudaDeviceGetAttribute(&st->sm_count, cudaDevAttrMultiProcessorCount, cfg->device));
+    int ks = 2;
+    while (ks < cfg->num_anchors) ks <<= 1;
+    st->key_stride = ks;
+
+    const size_t mb = (size_t)cfg->max_batch;
+    cudaError_t e = cudaSuccess;
+    if (e == cudaSuccess) e = dev_alloc(&st->d_keys, mb * ks, &st->workspace_bytes);
+    if (e == cudaSuccess) e = dev_alloc(&st->d_boxes, mb * ks, &st->workspace_bytes);
+    if (e == cudaSuccess) e = dev_alloc(&st->d_cand_count, mb, &st->workspace_bytes);
+    if (e == cudaSuccess) e = dev_alloc(&st->d_bcount, (size_t)OCTO_MAX_BRANCHES * mb, &st->workspace_bytes);
+    if (e == cudaSuccess)
+        e = dev_alloc(&st->d_bidx, (size_t)OCTO_MAX_BRANCHES * mb * cfg->max_det, &st->workspace_bytes);
+    for (int b = 0; b < cfg->num_branches && e == cudaSuccess; ++b)
+        e = dev_alloc(&st->d_items[b], mb * cfg->max_det, &st->workspace_bytes);
+    if (e == cudaSuccess) e = dev_alloc(&st->d_ctr, 1, &st->workspace_bytes);
+    if (e == cudaSuccess) e = prepare_letterbox();
+    if (e == cudaSuccess) e = prepare_nms();
+    if (e != cudaSuccess) {
+        free_all(st);
+        delete st;
+        return cuda_fail(e, "octo_stage_create");
+    }
+    *out = st;
+    return OCTO_OK;
+}
+
+extern "C" int octo_stage_destroy(octo_stage_t* st) {
+    if (!st) return OCTO_E_INVALID_ARG;
+    cudaSetDevice(st->cfg.device);
+    free_all(st);
+    delete st;
+    return OCTO_OK;
+}
+
+// Letterbox geometry in exact integer arithmetic: the longer side maps to S, the other to
+// round-half-up(short * S / long), at least 1; centred, odd remainder right/bottom.
+static void letterbox_geometry(int w, int h, int S, FrameDesc* fd) {
+    long long nw, nh;
+    if (w >= h) {
+        nw = S;
+        nh = (2LL * h * S + w) / (2LL * w);
+        if (nh < 1) nh = 1;
+    } else {
+        nh = S;
+        nw = (2LL * w * S + h) / (2LL * h);
+        if (nw < 1) nw = 1;
+    }
+    fd->nw = (int)nw;
+    fd->nh = (int)nh;
+    fd->pad_l = (int)((S - nw) / 2);
+    fd->pad_t = (int)((S - nh) / 2);
+    fd->gx = (float)w / (float)fd->nw;
+    fd->gy = (float)h / (float)fd->nh;
+}
+
+extern "C" int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frames, int32_t n,
+                                     void* d_out_f16_nchw, void* cuda_stream) {
+    if (!st || !frames || !d_out_f16_nchw || n < 1) return OCTO_E_INVALID_ARG;
+    if (n > st->cfg.max_batch) return OCTO_E_CAPACITY;
+    if (reinterpret_cast<uintptr_t>(d_out_f16_nchw) & 15) return OCTO_E_ALIGNMENT;
+    int max_w = 0;
+    for (int i = 0; i < n; ++i) {
+        const octo_frame_t& f = frames[i];
+        if (!f.d_data || f.width < 1 || f.height < 1) return OCTO_E_INVALID_ARG;
+        if (f.width > 16384 || f.height > 16384) return OCTO_E_CAPACITY;
+        if (f.width > kLetterboxMaxWidth) return OCTO_E_CAPACITY;
+        if ((long long)f.pitch_bytes < 3LL * f.width) return OCTO_E_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(f.d_data) & 15) || (f.pitch_bytes & 15)) return OCTO_E_ALIGNMENT;
+        if (f.width > max_w) max_w = f.width;
+    }
+    st->n_frames = 0;
+    st->have_dets = false;
+    for (int i = 0; i < n; ++i) {
+        FrameDesc& fd = st->frames[i];
+        fd.data = frames[i].d_data;
+        fd.w = frames[i].width;
+        fd.h = frames[i].height;
+        fd.pitch = frames[i].pitch_bytes;
+        fd._pad = 0;
+        letterbox_geometry(fd.w, fd.h, st->cfg.net_size, &fd);
+    }
+    st->max_w = max_w;
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    OCTO_CUDA(launch_letterbox(st->frames, n, d_out_f16_nchw, st->cfg.net_size, max_w, st->cfg.pad_value,
+                               st->cfg.swap_rb, &st->d_ctr->status, static_cast<cudaStream_t>(cuda_stream)));
+    st->launches += 1;
+    st->n_frames = n;
+    return OCTO_OK;
+}
+
+extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int32_t n, octo_det_t* d_dets,
+                                      int32_t* d_counts, void* cuda_stream) {
+    if (!st || !d_head || !d_dets || !d_counts) return OCTO_E_INVALID_ARG;
+    if (st->n_frames < 1) return OCTO_E_NO_PREPROCESS;
+    if (n != st->n_frames) return OCTO_E_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_head) & 3) || (reinterpret_cast<uintptr_t>(d_dets) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_counts) & 3))
+        return OCTO_E_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const octo_stage_config_t& c = st->cfg;
+    st->have_dets = false;
+    OCTO_CUDA(cudaSetDevice(c.device));
+    OCTO_CUDA(launch_decode(d_head, n, c.num_anchors, c.num_classes, c.head_is_logits, c.conf_thresh,
+                            st->key_stride, st->d_keys, st->d_cand_count, &st->d_ctr->status, stream));
+    st->launches += 1;
+    NmsArgs a;
+    a.frames = st->frames;
+    a.n = n;
+    a.d_head = d_head;
+    a.A = c.num_anchors;
+    a.C = c.num_classes;
+    a.iou_thr = c.iou_thresh;
+    a.max_det = c.max_det;
+    a.key_stride = st->key_stride;
+    a.d_keys = st->d_keys;
+    a.d_boxes = st->d_boxes;
+    a.d_cand_count = st->d_cand_count;
+    a.d_dets = d_dets;
+    a.d_counts = d_counts;
+    a.num_branches = c.num_branches;
+    memset(&a.masks, 0, sizeof(a.masks));
+    for (int b = 0; b < c.num_branches; ++b) memcpy(a.masks.m[b], c.branch[b].class_mask, sizeof(uint32_t) * 4);
+    a.d_bcount = st->d_bcount;
+    a.d_bidx = st->d_bidx;
+    a.max_batch = c.max_batch;
+    a.d_ctr = st->d_ctr;
+    cudaError_t e = launch_nms(a, stream);
+    if (e != cudaSuccess) {
+        // keep the "candidate counters are zero on entry" invariant after a failed launch
+        cudaMemsetAsync(st->d_cand_count, 0, sizeof(int) * (size_t)c.max_batch, stream);
+        return cuda_fail(e, "launch_nms");
+    }
+    st->launches += 1;
+    st->have_dets = true;
+    st->d_dets = d_dets;
+    return OCTO_OK;
+}
+
+extern "C" int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_item, int32_t max_items,
+                               void* d_out_f16, int32_t* d_offsets, int32_t* d_n_items, void* cuda_stream) {
+    if (!st || !d_offsets || !d_n_items) return OCTO_E_INVALID_ARG;
+    if (branch < 0 || branch >= st->cfg.num_branches) return OCTO_E_INVALID_ARG;
+    if (first_item < 0 || max_items < 0) return OCTO_E_INVALID_ARG;
+    if (max_items > 0 && !d_out_f16) return OCTO_E_INVALID_ARG;
+    if (st->n_frames < 1) return OCTO_E_NO_PREPROCESS;
+    if (!st->have_dets) return OCTO_E_NO_POSTPROCESS;
+    if ((reinterpret_cast<uintptr_t>(d_out_f16) & 15) || (reinterpret_cast<uintptr_t>(d_offsets) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_n_items) & 3))
+        return OCTO_E_ALIGNMENT;
+    const octo_stage_config_t& c = st->cfg;
+    const long long cap = (long long)c.max_batch * c.max_det;
+    if (max_items > cap) max_items = (int32_t)cap;  // a branch can never hold more items
+    CropArgs a;
+    a.frames = st->frames;
+    a.n = st->n_frames;
+    a.max_det = c.max_det;
+    a.first_item = first_item;
+    a.max_items = max_items;
+    a.d_bcount = st->d_bcount + (size_t)branch * c.max_batch;
+    a.d_bidx = st->d_bidx + (size_t)branch * c.max_batch * c.max_det;
+    a.d_dets = st->d_dets;
+    a.d_offsets = d_offsets;
+    a.d_n_items = d_n_items;
+    a.d_items = st->d_items[branch];
+    a.d_out = d_out_f16;
+    a.out_w = c.branch[branch].out_w;
+    a.out_h = c.branch[branch].out_h;
+    a.swap_rb = c.swap_rb;
+    a.sm_count = st->sm_count;
+    a.d_ctr = st->d_ctr;
+    OCTO_CUDA(cudaSetDevice(c.device));
+    OCTO_CUDA(launch_crop(a, static_cast<cudaStream_t>(cuda_stream)));
+    st->launches += max_items > 0 ? 2 : 1;
+    return OCTO_OK;
+}
+
+extern "C" int octo_stage_status(octo_stage_t* st, uint32_t* status_word, void* cuda_stream) {
+    if (!st || !status_word) return OCTO_E_INVALID_ARG;
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    OCTO_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+    unsigned int w = 0;
+    OCTO_CUDA(cudaMemcpy(&w, &st->d_ctr->status, sizeof(w), cudaMemcpyDeviceToHost));
+    *status_word = w;
+    return (w & OCTO_STATUS_COPY_TIMEOUT) ? OCTO_E_DEVICE_TIMEOUT : OCTO_OK;
+}
+
+extern "C" int octo_stage_clear_status(octo_stage_t* st, void* cuda_stream) {
+    if (!st) return OCTO_E_INVALID_ARG;
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    OCTO_CUDA(cudaMemsetAsync(&st->d_ctr->status, 0, sizeof(unsigned int), static_cast<cudaStream_t>(cuda_stream)));
+    return OCTO_OK;
+}
+
+extern "C" int octo_stage_get_stats(octo_stage_t* st, octo_stage_stats_t* stats, void* cuda_stream) {
+    if (!st || !stats) return OCTO_E_INVALID_ARG;
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    OCTO_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+    StageCounters h;
+    OCTO_CUDA(cudaMemcpy(&h, st->d_ctr, sizeof(h), cudaMemcpyDeviceToHost));
+    stats->candidates = (int64_t)h.candidates;
+    stats->kept = (int64_t)h.kept;
+    stats->packed = h.packed;
+    stats->total_items = h.total_items;
+    stats->status_word = h.status;
+    stats->max_candidates_per_image = h.max_cand;
+    // candidates / kept accumulate over one postprocess call only: reset for the next one
+    OCTO_CUDA(cudaMemset(st->d_ctr, 0, offsetof(StageCounters, status)));
+    OCTO_CUDA(cudaMemset(&st->d_ctr->max_cand, 0, sizeof(int)));
+    return OCTO_OK;
+}
+
+extern "C" int octo_stage_item_table(octo_stage_t* st, int32_t branch, const octo_item_t** d_items) {
+    if (!st || !d_items || branch < 0 || branch >= st->cfg.num_branches) return OCTO_E_INVALID_ARG;
+    *d_items = st->d_items[branch];
+    return OCTO_OK;
+}
+
+extern "C" int octo_stage_copy_items(octo_stage_t* st, int32_t branch, octo_item_t* items_out, int32_t count,
+                                     void* cuda_stream) {
+    if (!st || branch < 0 || branch >= st->cfg.num_branches || count < 0) return OCTO_E_INVALID_ARG;
+    if ((long long)count > (long long)st->cfg.max_batch * st->cfg.max_det) return OCTO_E_CAPACITY;
+    if (count > 0 && !items_out) return OCTO_E_INVALID_ARG;
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    OCTO_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+    if (count > 0)
+        OCTO_CUDA(cudaMemcpy(items_out, st->d_items[branch], sizeof(octo_item_t) * (size_t)count,
+                             cudaMemcpyDeviceToHost));
+    return OCTO_OK;
+}
+
+extern "C" int64_t octo_stage_workspace_bytes(const octo_stage_t* st) { return st ? st->workspace_bytes : 0; }
+extern "C" int64_t octo_stage_launch_count(const octo_stage_t* st) { return st ? st->launches : 0; }
+
+extern "C" const char* octo_strerror(int code) {
+    switch (code) {
+        case OCTO_OK: return "ok";
+        case OCTO_E_INVALID_ARG: return "invalid argument";
+        case OCTO_E_CAPACITY: return "capacity exceeded";
+        case OCTO_E_ALIGNMENT: return "pointer or pitch not 16-byte aligned";
+        case OCTO_E_NO_PREPROCESS: return "no batch has been preprocessed on this stage";
+        case OCTO_E_CUDA: return "CUDA runtime error";
+        case OCTO_E_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+        case OCTO_E_NO_POSTPROCESS: return "the current batch has not been postprocessed";
+        default: return "unknown status code";
+    }
+}
+
+extern "C" const char* octo_last_cuda_error(void) { return g_cuda_err; }
+extern "C" const char* octo_version(void) { return "0.1"; }
