@@ -1,0 +1,460 @@
+#!/usr/bin/env python
+"""Benchmark of the cascade-stage hot path (letterbox -> decode/NMS -> assemble -> crop).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload sweep] [--batch 256]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores
+
+A step is one pass of the whole stage over one batch of synthetic frames and detector
+heads.  `value` is frames/s with the inputs resident in device memory; `e2e` is the same
+pass driven from pinned host buffers with the host<->device copies inside the timed region.
+With N > 1 (torchrun) every rank runs the same stage on its own frames (replicas, no
+collective on the data path); the time is the maximum over ranks.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "stage_frames_per_s"
+UNIT = "frames/s"
+
+# DRAM traffic from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum) per unit of
+# work, so that it can be scaled to the benchmarked launch, with the hash of the kernel
+# source the capture was taken from.  An entry whose hash no longer matches the source is
+# reported as null.
+NCU_TRAFFIC = {
+    # kernel: (source file, sha256[:16] of that file at capture time, bytes per unit, unit)
+}
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=30)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--workload", default="sweep", choices=sorted(workloads.WORKLOADS))
+    p.add_argument("--batch", type=int, default=None, help="frames per GPU per step")
+    p.add_argument("--impl", default="octo", choices=["octo", "reference"])
+    p.add_argument("--e2e-steps", type=int, default=None)
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-e2e", action="store_true")
+    return p.parse_args()
+
+
+def default_batch(name: str) -> int:
+    return 256 if name == "sweep" else workloads.WORKLOADS[name].batch
+
+
+# ---- algorithmic bytes (what the method must move; numerators of the roofline) --------------
+
+def letterbox_bytes(sizes, s: int) -> int:
+    """Source rows that carry weight (as 16-byte-granular row copies) + the fp16 output."""
+    total = 0
+    cache = {}
+    for (w, h) in sizes:
+        if (w, h) not in cache:
+            nh = max(1, (2 * h * s + w) // (2 * w)) if w >= h else s
+            rows = 0
+            for dy in range(nh):
+                num = (2 * dy + 1) * h - nh
+                if num <= 0 or num // (2 * nh) >= h - 1:
+                    rows += 1
+                else:
+                    rows += 1 if num % (2 * nh) == 0 else 2
+            cache[(w, h)] = rows * ((3 * w + 15) // 16 * 16) + 3 * s * s * 2
+        total += cache[(w, h)]
+    return total
+
+
+def crop_bytes(items: np.ndarray, ow: int, oh: int) -> int:
+    """fp16 output of every packed crop + its source rectangle, each counted once."""
+    cw = (items["rx1"] - items["rx0"]).astype(np.int64)
+    ch = (items["ry1"] - items["ry0"]).astype(np.int64)
+    return int(len(items) * 3 * ow * oh * 2 + int((cw * ch * 3).sum()))
+
+
+def decode_bytes(n: int, a: int, c: int, candidates: int, logits: bool) -> int:
+    """One 32-byte sector per head row for the obj scan (logit heads) or the whole row
+    (probability heads), plus the full row and the 8-byte key of each candidate."""
+    row = 4 * (5 + c)
+    scan = 32 * a * n if logits else row * a * n
+    return int(scan + candidates * (row + 8))
+
+
+def file_hash(path: str) -> str:
+    return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
+
+
+def traffic_for(kernel: str, units: float):
+    ent = NCU_TRAFFIC.get(kernel)
+    if not ent:
+        return None
+    src, digest, per_unit, _unit = ent
+    if file_hash(os.path.join(ROOT, src)) != digest:
+        return None
+    return per_unit * units
+
+
+# ---- clocks ---------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm), reasons=sorted(reasons))
+        return out
+
+
+# ---- the reference arm: the CPU oracle ------------------------------------------------------
+
+def oracle_pass(batch, frames_used: int, threads: int) -> float:
+    """Seconds the oracle needs for the whole stage on the first `frames_used` frames."""
+    import oracle
+    wl = batch.workload
+    t0 = time.perf_counter()
+    oracle.run_stage(batch.frames[:frames_used], batch.sizes[:frames_used], batch.head[:frames_used],
+                     wl.net_size, wl.branches, logits=wl.logits, conf=wl.conf_thresh, iou_thr=wl.iou_thresh,
+                     max_det=wl.max_det, threads=threads)
+    return time.perf_counter() - t0
+
+
+def cpu_sample_frames(batch_n: int, cores: int) -> int:
+    # about 0.25 s of single-core work per 1080p frame -> roughly 5-20 s of wall time
+    return max(1, min(batch_n, 64 * cores))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    name = args.workload
+    bsz = args.batch or default_batch(name)
+    cores = len(os.sched_getaffinity(0))
+    sample = cpu_sample_frames(bsz, cores)
+    batch = workloads.make_batch(name, batch=sample)
+    warm = min(args.warmup, 1)
+    for _ in range(warm):
+        oracle_pass(batch, min(sample, cores), cores)
+    steps = max(1, min(args.steps, 3))
+    times = [oracle_pass(batch, sample, cores) for _ in range(steps)]
+    t = sum(times) / len(times)
+    value = sample / t
+    wl = batch.workload
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": 1e3 * t, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{name} B={bsz}", "frames_per_step": sample, "net_size": wl.net_size,
+                   "note": "CPU oracle; each step is a bounded sample of the batch"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"first {sample} of {bsz} frames, whole stage, {cores} threads"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---- the CUDA arm ---------------------------------------------------------------------------
+
+def run_octo(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2502_01277_b200 as octo
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    name = args.workload
+    bsz = args.batch or default_batch(name)
+    batch = workloads.make_batch(name, batch=bsz, first_frame=rank * bsz)
+    wl = batch.workload
+    n, s = batch.n, wl.net_size
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured" if "hbm_gbs" in peaks else "fallback"
+
+    stage = octo.Stage(device=local_rank, net_size=s, max_batch=n, num_anchors=wl.num_anchors,
+                       num_classes=wl.num_classes, head_is_logits=wl.logits, conf_thresh=wl.conf_thresh,
+                       iou_thresh=wl.iou_thresh, max_det=wl.max_det, branches=wl.branches)
+    stream = torch.cuda.Stream(dev)
+    cap = n * wl.items_per_frame
+
+    # Input sets: a single set once it exceeds 512 MB, else enough rotating copies that the
+    # working set is larger than L2 several times over.
+    h_frames = [torch.from_numpy(f).pin_memory() for f in batch.frames]
+    h_head = torch.from_numpy(batch.head).pin_memory()
+    in_bytes = sum(f.numel() for f in h_frames) + h_head.numel() * 4
+    out_bytes = n * 3 * s * s * 2 + sum(cap * 3 * ow * oh * 2 for ow, oh in wl.branches)
+    n_sets = max(1, min(64, -(-(512 << 20) // (in_bytes + n * 3 * s * s * 2))))
+
+    class Set:
+        pass
+
+    sets = []
+    with torch.cuda.stream(stream):
+        for _ in range(n_sets):
+            z = Set()
+            z.frames = [f.to(dev, non_blocking=True) for f in h_frames]
+            z.head = h_head.to(dev, non_blocking=True)
+            z.det_in = torch.empty((n, 3, s, s), dtype=torch.float16, device=dev)
+            z.dets = torch.zeros((n, wl.max_det, 32), dtype=torch.uint8, device=dev)
+            z.counts = torch.zeros((n,), dtype=torch.int32, device=dev)
+            z.crops = [torch.empty((cap, 3, oh, ow), dtype=torch.float16, device=dev) for ow, oh in wl.branches]
+            z.offsets = [torch.zeros((n + 1,), dtype=torch.int32, device=dev) for _ in wl.branches]
+            z.n_items = [torch.zeros((2,), dtype=torch.int32, device=dev) for _ in wl.branches]
+            z.desc = stage.frame_array(z.frames, batch.sizes)
+            sets.append(z)
+    stream.synchronize()
+
+    def step(z):
+        stage.preprocess_array(z.desc, n, z.det_in, stream=stream, keepalive=z.frames)
+        stage.postprocess(z.head, dets=z.dets, counts=z.counts, stream=stream)
+        for b in range(len(wl.branches)):
+            stage.crop(b, cap, out=z.crops[b], offsets=z.offsets[b], n_items=z.n_items[b], stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def timed(nsteps, fn):
+        barrier()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(nsteps):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    # ---- resident-input throughput ----
+    warm = max(args.warmup, 3)
+    for i in range(warm):
+        step(sets[i % n_sets])
+    torch.cuda.synchronize(dev)
+    launches0 = stage.launch_count
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ms_total = timed(args.steps, lambda i: step(sets[i % n_sets]))
+    gpu_launches = stage.launch_count - launches0
+    ms_per_step = ms_total / args.steps
+    value = world * n / (ms_per_step * 1e-3)
+
+    # sanity of the run + sizes for the byte accounting (outside the timed region)
+    z0 = sets[0]
+    totals = [tuple(int(v) for v in t.cpu()) for t in z0.n_items]
+    for b, (packed, total) in enumerate(totals):
+        if packed != total:
+            raise SystemExit(f"branch {b}: provisioned {cap} crop slots but the batch holds {total} items")
+    stage.stats(stream)
+    status = stage.status(stream)
+    if status & ~0x8:
+        raise SystemExit(f"device status word {status:#x}")
+    items = [stage.item_table(b, totals[b][0]) for b in range(len(wl.branches))]
+
+    # ---- per-kernel device times: the same steps with an event pair around every launch ----
+    stage.set_timing(True)
+    stage.kernel_times(stream)
+    ms_ev_total = timed(args.steps, lambda i: step(sets[i % n_sets]))
+    kt = stage.kernel_times(stream)
+    stage.set_timing(False)
+    clocks = sampler.stop() if rank == 0 else {}
+    stats = stage.stats(stream)
+    cand_per_step = stats["candidates"] / args.steps
+    kern = {}
+    alg = {
+        "letterbox": letterbox_bytes(batch.sizes, s),
+        "decode": decode_bytes(n, wl.num_anchors, wl.num_classes, int(cand_per_step), wl.logits),
+        "crop": sum(crop_bytes(items[b], *wl.branches[b]) for b in range(len(wl.branches))) / len(wl.branches),
+    }
+    names = octo.binding.KERNEL_NAMES
+    for k in names:
+        ms_sum, cnt = kt[k]
+        if cnt == 0:
+            continue
+        avg = ms_sum / cnt
+        kern[k] = {"launches_per_step": cnt / args.steps, "ms_per_launch": avg, "share": None}
+        if k in alg:
+            kern[k]["alg_bytes_per_launch"] = alg[k]
+            kern[k]["gbs"] = alg[k] / (avg * 1e-3) / 1e9
+            kern[k]["frac_of_hbm_peak"] = kern[k]["gbs"] / hbm_peak
+    tot_ms = sum(kt[k][0] for k in names)
+    for k in kern:
+        kern[k]["share"] = kt[k][0] / tot_ms if tot_ms > 0 else None
+    dominant = max((k for k in kern if k in alg), key=lambda k: kt[k][0])
+    units = {"letterbox": n, "decode": n, "crop": len(items[0])}[dominant]
+    roofline = {
+        "kernel": dominant, "bound": "hbm", "achieved": kern[dominant]["gbs"], "peak": hbm_peak,
+        "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})", "unit": "GB/s",
+        "frac": kern[dominant]["gbs"] / hbm_peak, "frac_of_nominal_8TBs": kern[dominant]["gbs"] / 8000.0,
+        "alg_bytes_per_launch": alg[dominant], "ms_per_launch": kern[dominant]["ms_per_launch"],
+        "traffic": traffic_for(dominant, units),
+    }
+
+    # ---- end to end from pinned host buffers ----
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = args.e2e_steps or max(3, min(args.steps, 10))
+        z = sets[0]
+        h_dets = torch.empty((n, wl.max_det, 32), dtype=torch.uint8).pin_memory()
+        h_counts = torch.empty((n,), dtype=torch.int32).pin_memory()
+        h_off = [torch.empty((n + 1,), dtype=torch.int32).pin_memory() for _ in wl.branches]
+        h_ni = [torch.empty((2,), dtype=torch.int32).pin_memory() for _ in wl.branches]
+        h_crops = [torch.empty((max(totals[b][1], 1), 3, oh, ow), dtype=torch.float16).pin_memory()
+                   for b, (ow, oh) in enumerate(wl.branches)]
+        d2h = [0]
+
+        def e2e_step(_i):
+            with torch.cuda.stream(stream):
+                for hf, df in zip(h_frames, z.frames):
+                    df.copy_(hf, non_blocking=True)
+                z.head.copy_(h_head, non_blocking=True)
+                step(z)
+                h_dets.copy_(z.dets, non_blocking=True)
+                h_counts.copy_(z.counts, non_blocking=True)
+                for b in range(len(wl.branches)):
+                    h_off[b].copy_(z.offsets[b], non_blocking=True)
+                    h_ni[b].copy_(z.n_items[b], non_blocking=True)
+            stream.synchronize()  # the caller needs the packed counts to size the crop read-back
+            nb = h_dets.numel() + h_counts.numel() * 4
+            with torch.cuda.stream(stream):
+                for b in range(len(wl.branches)):
+                    packed = min(int(h_ni[b][0]), h_crops[b].shape[0])
+                    h_crops[b][:packed].copy_(z.crops[b][:packed], non_blocking=True)
+                    nb += packed * h_crops[b][0].numel() * 2 + h_off[b].numel() * 4 + 8
+            stream.synchronize()
+            d2h[0] = nb
+
+        for i in range(3):
+            e2e_step(i)
+        ms_e2e = timed(e2e_steps, e2e_step) / e2e_steps
+        e2e = {"value": world * n / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
+               "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(d2h[0])}
+
+    # ---- CPU baseline (rank 0, single-GPU runs only) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cores = len(os.sched_getaffinity(0))
+        sample = cpu_sample_frames(n, cores)
+        t = oracle_pass(batch, sample, cores)
+        cpu = {"value": sample / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {sample} of {n} frames, whole stage, {cores} threads, {t:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": f"{name} B={n}" + (" per GPU" if world > 1 else ""),
+                "frames": "x".join(str(v) for v in batch.sizes[0]) + (" (mixed)" if len(set(batch.sizes)) > 1 else ""),
+                "net_size": s, "head": [n, wl.num_anchors, 5 + wl.num_classes],
+                "crops": [list(b) for b in wl.branches], "items_per_step": [t[1] for t in totals],
+                "candidates_per_step": cand_per_step, "parallelism": f"replicas x{world}",
+                "l2": (f"{n_sets} rotating input/output sets, {n_sets * (in_bytes + out_bytes) / 2**20:.0f} MiB working set"
+                       if n_sets > 1 else f"one set of {(in_bytes + out_bytes) / 2**20:.0f} MiB per step, larger than L2"),
+            },
+            "e2e": e2e,
+            "gpu_launches": int(gpu_launches),
+            "clocks": clocks,
+            "roofline": roofline,
+            "kernels": kern,
+            "ms_per_step_with_kernel_events": ms_ev_total / args.steps,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    stage.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_octo(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -214,6 +214,24 @@ OCTO_API int octo_stage_item_table(octo_stage_t* st, int32_t branch, const octo_
 OCTO_API int octo_stage_copy_items(octo_stage_t* st, int32_t branch, octo_item_t* items_out, int32_t count,
                                    void* cuda_stream);
 
+/* Kernel order used by octo_kernel_times_t. */
+enum { OCTO_K_LETTERBOX = 0, OCTO_K_DECODE = 1, OCTO_K_NMS = 2, OCTO_K_ASSEMBLE = 3, OCTO_K_CROP = 4,
+       OCTO_K_COUNT = 5 };
+
+typedef struct {
+    double ms[OCTO_K_COUNT];        /* summed device time of each kernel's launches            */
+    int64_t launches[OCTO_K_COUNT]; /* launches measured                                       */
+    int64_t dropped;                /* launches not measured because the event pool was full   */
+} octo_kernel_times_t;
+
+/* Per-kernel timing for profiling: while enabled, every kernel launch is bracketed by CUDA
+ * events recorded on the launching stream (a small cost per launch).  Off by default. */
+OCTO_API int octo_stage_set_timing(octo_stage_t* st, int32_t enable);
+
+/* Synchronise `cuda_stream`, sum the event pairs recorded since the previous call into
+ * *times and release them. */
+OCTO_API int octo_stage_kernel_times(octo_stage_t* st, octo_kernel_times_t* times, void* cuda_stream);
+
 /* Bytes of device memory the stage holds. */
 OCTO_API int64_t octo_stage_workspace_bytes(const octo_stage_t* st);
 

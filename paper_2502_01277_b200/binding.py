@@ -38,7 +38,8 @@ OCTO_STATUS_BIG_NMS = 0x8
 EXPORTS = (
     "octo_stage_create", "octo_stage_destroy", "octo_preprocess_batch", "octo_postprocess_batch",
     "octo_crop_batch", "octo_stage_status", "octo_stage_clear_status", "octo_stage_get_stats",
-    "octo_stage_item_table", "octo_stage_copy_items", "octo_stage_workspace_bytes", "octo_stage_launch_count",
+    "octo_stage_item_table", "octo_stage_copy_items", "octo_stage_set_timing", "octo_stage_kernel_times",
+    "octo_stage_workspace_bytes", "octo_stage_launch_count",
     "octo_strerror", "octo_last_cuda_error", "octo_version",
 )
 
@@ -67,6 +68,13 @@ class StageStats(ctypes.Structure):
     _fields_ = [("candidates", ctypes.c_int64), ("kept", ctypes.c_int64), ("packed", ctypes.c_int64),
                 ("total_items", ctypes.c_int64), ("status_word", ctypes.c_uint32),
                 ("max_candidates_per_image", ctypes.c_int32)]
+
+
+KERNEL_NAMES = ("letterbox", "decode", "nms", "assemble", "crop")
+
+
+class KernelTimes(ctypes.Structure):
+    _fields_ = [("ms", ctypes.c_double * 5), ("launches", ctypes.c_int64 * 5), ("dropped", ctypes.c_int64)]
 
 
 DET_DTYPE = np.dtype([("x1", "<f4"), ("y1", "<f4"), ("x2", "<f4"), ("y2", "<f4"), ("score", "<f4"),
@@ -111,6 +119,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_stage_item_table.argtypes = [vp, i32, ctypes.POINTER(vp)]
     lib.octo_stage_copy_items.argtypes = [vp, i32, vp, i32, vp]
     lib.octo_stage_copy_items.restype = ctypes.c_int
+    lib.octo_stage_set_timing.argtypes = [vp, i32]
+    lib.octo_stage_set_timing.restype = ctypes.c_int
+    lib.octo_stage_kernel_times.argtypes = [vp, ctypes.POINTER(KernelTimes), vp]
+    lib.octo_stage_kernel_times.restype = ctypes.c_int
     lib.octo_stage_workspace_bytes.argtypes = [vp]
     lib.octo_stage_workspace_bytes.restype = ctypes.c_int64
     lib.octo_stage_launch_count.argtypes = [vp]
@@ -245,6 +257,23 @@ class Stage:
         self.n = n
         return out
 
+    def frame_array(self, frames, sizes):
+        """Descriptor array for tensors whose addresses stay fixed; reuse it with
+        preprocess_array to skip the per-call marshalling."""
+        arr = (Frame * max(len(frames), 1))()
+        for i, (f, (w, h)) in enumerate(zip(frames, sizes)):
+            arr[i].d_data, arr[i].width, arr[i].height, arr[i].pitch_bytes = f.data_ptr(), w, h, f.stride(0)
+        return arr
+
+    def preprocess_array(self, arr, n, out, stream=None, keepalive=None):
+        rc = load_library().octo_preprocess_batch(self.handle, arr, n, out.data_ptr(), self._stream(stream))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_preprocess_batch")
+        if keepalive is not None:
+            self._frames_keepalive = keepalive
+        self.n = n
+        return out
+
     def postprocess(self, head, dets=None, counts=None, stream=None):
         """head: float32 CUDA tensor [n, A, 5+C].  Returns (dets uint8 [n, max_det, 32], counts int32 [n])."""
         t = self._torch
@@ -288,6 +317,21 @@ class Stage:
 
     def stats(self, stream=None) -> dict:
         return octo_stage_get_stats(self.handle, self._stream(stream))
+
+    def set_timing(self, enable: bool) -> None:
+        rc = load_library().octo_stage_set_timing(self.handle, 1 if enable else 0)
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_stage_set_timing")
+
+    def kernel_times(self, stream=None) -> dict:
+        """{kernel: (summed ms, launches)} since the previous call; synchronises the stream."""
+        kt = KernelTimes()
+        rc = load_library().octo_stage_kernel_times(self.handle, ctypes.byref(kt), self._stream(stream))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_stage_kernel_times")
+        out = {name: (float(kt.ms[i]), int(kt.launches[i])) for i, name in enumerate(KERNEL_NAMES)}
+        out["dropped"] = int(kt.dropped)
+        return out
 
     @property
     def launch_count(self) -> int:

@@ -162,15 +162,19 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
 }
 
 template <int CAP>
-static cudaError_t launch_cap(const CropArgs& a, cudaStream_t stream) {
+static cudaError_t launch_assemble_cap(const CropArgs& a, cudaStream_t stream) {
     static FrameTable<CAP> tab;
     for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
     assemble_kernel<CAP><<<1, kAsmThreads, 0, stream>>>(tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount,
                                                        a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items, a.d_items,
                                                        a.d_ctr);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    if (a.max_items <= 0) return cudaSuccess;
+    return cudaGetLastError();
+}
+
+template <int CAP>
+static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
+    static FrameTable<CAP> tab;
+    for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
     int band_rows = 2048 / a.out_w;
     band_rows = band_rows < 1 ? 1 : (band_rows > a.out_h ? a.out_h : band_rows);
     const int bands = (a.out_h + band_rows - 1) / band_rows;
@@ -183,10 +187,17 @@ static cudaError_t launch_cap(const CropArgs& a, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
+cudaError_t launch_assemble(const CropArgs& a, cudaStream_t stream) {
+    if (a.n <= 8) return launch_assemble_cap<8>(a, stream);
+    if (a.n <= 64) return launch_assemble_cap<64>(a, stream);
+    return launch_assemble_cap<512>(a, stream);
+}
+
+// Requires a.max_items > 0.
 cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream) {
-    if (a.n <= 8) return launch_cap<8>(a, stream);
-    if (a.n <= 64) return launch_cap<64>(a, stream);
-    return launch_cap<512>(a, stream);
+    if (a.n <= 8) return launch_crop_cap<8>(a, stream);
+    if (a.n <= 64) return launch_crop_cap<64>(a, stream);
+    return launch_crop_cap<512>(a, stream);
 }
 
 }  // namespace octo

@@ -9,6 +9,8 @@
 
 using namespace octo;
 
+constexpr int kEventPairs = 2048;
+
 struct octo_stage {
     octo_stage_config_t cfg;
     int sm_count;
@@ -29,6 +31,29 @@ struct octo_stage {
     bool have_dets;
     const octo_det_t* d_dets;
     int64_t launches;
+    // optional per-kernel timing
+    bool timing;
+    cudaEvent_t ev[2 * kEventPairs];
+    int ev_kernel[kEventPairs];
+    int ev_used;
+    int64_t ev_dropped;
+};
+
+// Records an event pair around one kernel launch while timing is enabled.
+struct ScopedKernelTimer {
+    octo_stage* st;
+    cudaStream_t stream;
+    int slot;
+    ScopedKernelTimer(octo_stage* s, int kernel, cudaStream_t str) : st(s), stream(str), slot(-1) {
+        if (!st->timing) return;
+        if (st->ev_used >= kEventPairs) { st->ev_dropped += 1; return; }
+        slot = st->ev_used++;
+        st->ev_kernel[slot] = kernel;
+        cudaEventRecord(st->ev[2 * slot], stream);
+    }
+    ~ScopedKernelTimer() {
+        if (slot >= 0) cudaEventRecord(st->ev[2 * slot + 1], stream);
+    }
 };
 
 static thread_local char g_cuda_err[256] = "";
@@ -84,6 +109,8 @@ static void free_all(octo_stage* st) {
     cudaFree(st->d_bidx);
     for (int b = 0; b < OCTO_MAX_BRANCHES; ++b) cudaFree(st->d_items[b]);
     cudaFree(st->d_ctr);
+    for (int i = 0; i < 2 * kEventPairs; ++i)
+        if (st->ev[i]) cudaEventDestroy(st->ev[i]);
 }
 
 extern "C" int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** out) {
@@ -185,8 +212,11 @@ extern "C" int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frame
     }
     st->max_w = max_w;
     OCTO_CUDA(cudaSetDevice(st->cfg.device));
-    OCTO_CUDA(launch_letterbox(st->frames, n, d_out_f16_nchw, st->cfg.net_size, max_w, st->cfg.pad_value,
-                               st->cfg.swap_rb, &st->d_ctr->status, static_cast<cudaStream_t>(cuda_stream)));
+    {
+        ScopedKernelTimer t(st, OCTO_K_LETTERBOX, static_cast<cudaStream_t>(cuda_stream));
+        OCTO_CUDA(launch_letterbox(st->frames, n, d_out_f16_nchw, st->cfg.net_size, max_w, st->cfg.pad_value,
+                                   st->cfg.swap_rb, &st->d_ctr->status, static_cast<cudaStream_t>(cuda_stream)));
+    }
     st->launches += 1;
     st->n_frames = n;
     return OCTO_OK;
@@ -204,8 +234,11 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     const octo_stage_config_t& c = st->cfg;
     st->have_dets = false;
     OCTO_CUDA(cudaSetDevice(c.device));
-    OCTO_CUDA(launch_decode(d_head, n, c.num_anchors, c.num_classes, c.head_is_logits, c.conf_thresh,
-                            st->key_stride, st->d_keys, st->d_cand_count, &st->d_ctr->status, stream));
+    {
+        ScopedKernelTimer t(st, OCTO_K_DECODE, stream);
+        OCTO_CUDA(launch_decode(d_head, n, c.num_anchors, c.num_classes, c.head_is_logits, c.conf_thresh,
+                                st->key_stride, st->d_keys, st->d_cand_count, &st->d_ctr->status, stream));
+    }
     st->launches += 1;
     NmsArgs a;
     a.frames = st->frames;
@@ -228,7 +261,11 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     a.d_bidx = st->d_bidx;
     a.max_batch = c.max_batch;
     a.d_ctr = st->d_ctr;
-    cudaError_t e = launch_nms(a, stream);
+    cudaError_t e;
+    {
+        ScopedKernelTimer t(st, OCTO_K_NMS, stream);
+        e = launch_nms(a, stream);
+    }
     if (e != cudaSuccess) {
         // keep the "candidate counters are zero on entry" invariant after a failed launch
         cudaMemsetAsync(st->d_cand_count, 0, sizeof(int) * (size_t)c.max_batch, stream);
@@ -273,8 +310,17 @@ extern "C" int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_i
     a.sm_count = st->sm_count;
     a.d_ctr = st->d_ctr;
     OCTO_CUDA(cudaSetDevice(c.device));
-    OCTO_CUDA(launch_crop(a, static_cast<cudaStream_t>(cuda_stream)));
-    st->launches += max_items > 0 ? 2 : 1;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    {
+        ScopedKernelTimer t(st, OCTO_K_ASSEMBLE, stream);
+        OCTO_CUDA(launch_assemble(a, stream));
+    }
+    st->launches += 1;
+    if (max_items > 0) {
+        ScopedKernelTimer t(st, OCTO_K_CROP, stream);
+        OCTO_CUDA(launch_crop(a, stream));
+        st->launches += 1;
+    }
     return OCTO_OK;
 }
 
@@ -329,6 +375,33 @@ extern "C" int octo_stage_copy_items(octo_stage_t* st, int32_t branch, octo_item
     if (count > 0)
         OCTO_CUDA(cudaMemcpy(items_out, st->d_items[branch], sizeof(octo_item_t) * (size_t)count,
                              cudaMemcpyDeviceToHost));
+    return OCTO_OK;
+}
+
+extern "C" int octo_stage_set_timing(octo_stage_t* st, int32_t enable) {
+    if (!st) return OCTO_E_INVALID_ARG;
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    if (enable && !st->ev[0]) {
+        for (int i = 0; i < 2 * kEventPairs; ++i) OCTO_CUDA(cudaEventCreate(&st->ev[i]));
+    }
+    st->timing = enable != 0;
+    return OCTO_OK;
+}
+
+extern "C" int octo_stage_kernel_times(octo_stage_t* st, octo_kernel_times_t* times, void* cuda_stream) {
+    if (!st || !times) return OCTO_E_INVALID_ARG;
+    memset(times, 0, sizeof(*times));
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    OCTO_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+    for (int i = 0; i < st->ev_used; ++i) {
+        float ms = 0.0f;
+        OCTO_CUDA(cudaEventElapsedTime(&ms, st->ev[2 * i], st->ev[2 * i + 1]));
+        times->ms[st->ev_kernel[i]] += (double)ms;
+        times->launches[st->ev_kernel[i]] += 1;
+    }
+    times->dropped = st->ev_dropped;
+    st->ev_used = 0;
+    st->ev_dropped = 0;
     return OCTO_OK;
 }
 
