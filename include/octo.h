@@ -238,6 +238,42 @@ OCTO_API int64_t octo_stage_workspace_bytes(const octo_stage_t* st);
 /* Number of kernels the stage has launched since creation (for launch accounting). */
 OCTO_API int64_t octo_stage_launch_count(const octo_stage_t* st);
 
+/*
+ * Decode + class-aware NMS of ONE frame's head without any device allocation.
+ * (An addition for embedders; the paper has no counterpart to it.)
+ *
+ * Who needs it: callers that are not allowed to allocate GPU memory when they run, e.g. a
+ * real-time loop that fixed its memory budget at start-up and may not enter the allocator
+ * again, or a component hosted inside another application's memory pool with buffers handed
+ * to it.  octo_stage_create allocates a workspace, so those callers cannot own a stage.
+ * This call does the work of octo_postprocess_batch for n = 1 with the same kernels and the
+ * same rules, on a fixed workspace that is part of the library itself: about 0.8 MB of
+ * device memory that every GPU loading the library holds until the process exits.  It
+ * calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * Limits: num_anchors <= OCTO_STATIC_MAX_ANCHORS and max_det <= OCTO_STATIC_MAX_DET, else
+ * OCTO_E_CAPACITY.  The caller passes the input and both outputs:
+ *   d_head   device, [num_anchors, 5 + num_classes] float32 (same layout as a stage's head)
+ *   d_dets   device, [max_det] records; entries [0, *d_count) are written
+ *   d_count  device, one int32
+ * frame_w / frame_h / net_size give the letterbox geometry used to map boxes back to frame
+ * pixels, exactly as a stage would after preprocessing a frame of that size.
+ *
+ * The first call on a device looks up the workspace's device address and configures the
+ * kernels; make that first call before starting any stream capture.  All calls on a device
+ * share the one workspace, which keeps the previous call's contents (the call clears what
+ * has to start at zero): two calls whose GPU work overlaps, e.g. on different streams, race.
+ * Issue them on one stream or order them with events.
+ * Errors: OCTO_E_INVALID_ARG, OCTO_E_CAPACITY, OCTO_E_ALIGNMENT, OCTO_E_CUDA.
+ */
+#define OCTO_STATIC_MAX_ANCHORS 32768
+#define OCTO_STATIC_MAX_DET 1024
+OCTO_API int octo_postprocess_frame_static(int32_t device, const float* d_head, int32_t num_anchors,
+                                           int32_t num_classes, int32_t head_is_logits, float conf_thresh,
+                                           float iou_thresh, int32_t max_det, int32_t net_size,
+                                           int32_t frame_w, int32_t frame_h, octo_det_t* d_dets,
+                                           int32_t* d_count, void* cuda_stream);
+
 /* Text of a status code; never NULL. */
 OCTO_API const char* octo_strerror(int code);
 

@@ -40,7 +40,7 @@ EXPORTS = (
     "octo_crop_batch", "octo_stage_status", "octo_stage_clear_status", "octo_stage_get_stats",
     "octo_stage_item_table", "octo_stage_copy_items", "octo_stage_set_timing", "octo_stage_kernel_times",
     "octo_stage_workspace_bytes", "octo_stage_launch_count",
-    "octo_strerror", "octo_last_cuda_error", "octo_version",
+    "octo_strerror", "octo_last_cuda_error", "octo_version", "octo_postprocess_frame_static",
 )
 
 
@@ -123,6 +123,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_stage_set_timing.restype = ctypes.c_int
     lib.octo_stage_kernel_times.argtypes = [vp, ctypes.POINTER(KernelTimes), vp]
     lib.octo_stage_kernel_times.restype = ctypes.c_int
+    lib.octo_postprocess_frame_static.argtypes = [i32, vp, i32, i32, i32, ctypes.c_float, ctypes.c_float,
+                                                  i32, i32, i32, i32, vp, vp, vp]
+    lib.octo_postprocess_frame_static.restype = ctypes.c_int
     lib.octo_stage_workspace_bytes.argtypes = [vp]
     lib.octo_stage_workspace_bytes.restype = ctypes.c_int64
     lib.octo_stage_launch_count.argtypes = [vp]
@@ -196,6 +199,19 @@ def octo_crop_batch(handle, branch: int, first_item: int, max_items: int, d_out:
     rc = load_library().octo_crop_batch(handle, branch, first_item, max_items, d_out, d_offsets, d_n_items, stream)
     if rc != OCTO_OK:
         raise OctoError(rc, "octo_crop_batch")
+
+
+def octo_postprocess_frame_static(device: int, d_head: int, num_anchors: int, num_classes: int,
+                                  head_is_logits: bool, conf_thresh: float, iou_thresh: float, max_det: int,
+                                  net_size: int, frame_w: int, frame_h: int, d_dets: int, d_count: int,
+                                  stream: int = 0) -> None:
+    """Single-frame decode + NMS on the library's built-in workspace, for callers that may
+    not allocate device memory (see include/octo.h).  Pointers are raw device addresses."""
+    rc = load_library().octo_postprocess_frame_static(
+        device, d_head, num_anchors, num_classes, 1 if head_is_logits else 0, conf_thresh, iou_thresh,
+        max_det, net_size, frame_w, frame_h, d_dets, d_count, stream)
+    if rc != OCTO_OK:
+        raise OctoError(rc, "octo_postprocess_frame_static")
 
 
 def octo_stage_status(handle, stream: int = 0) -> int:
