@@ -92,6 +92,43 @@ __device__ __forceinline__ void row_taps(uint32_t lo, uint32_t hi, float fx, boo
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Table-driven horizontal sampling.  For every destination column a kernel precomputes, once
+// per tile, the byte offset of the left tap inside the staged source row and the two integer
+// weights (den - rem, rem) with den = 2 * dst <= 65535, packed as two 16-bit halves.  The
+// horizontal lerp of one colour channel is then a single two-way dot product of those
+// weights with the two tap bytes (exact in integers); the result carries a factor `den`.
+// ---------------------------------------------------------------------------------------
+struct XEntry {
+    uint32_t off;  // byte offset of pixel x0 in the staged row
+    uint32_t wts;  // (den - rem) | rem << 16
+};
+
+__device__ __forceinline__ XEntry make_xentry(int d, int src, int dst, float inv_den, int byte_base) {
+    int x0, rem;
+    src_coord(d, src, dst, inv_den, x0, rem);
+    XEntry e;
+    e.off = (uint32_t)(byte_base + 3 * x0);
+    e.wts = (uint32_t)(2 * dst - rem) | ((uint32_t)rem << 16);
+    return e;
+}
+
+// Integer horizontal lerp of the three channels of one destination pixel from a staged row
+// (4-byte aligned words in shared memory, with at least 12 readable bytes past any offset).
+__device__ __forceinline__ void hsample(const uint32_t* __restrict__ row, const XEntry e, uint32_t& c0, uint32_t& c1,
+                                        uint32_t& c2) {
+    const uint32_t wi = e.off >> 2;
+    const uint32_t sh = (e.off & 3u) * 8u;
+    const uint32_t a = row[wi], b = row[wi + 1], c = row[wi + 2];
+    const uint32_t lo = __funnelshift_r(a, b, sh);  // B0 G0 R0 B1
+    const uint32_t hi = __funnelshift_r(b, c, sh);  // G1 R1 .. ..
+    const uint32_t p01 = __byte_perm(lo, hi, 0x4130);  // B0 B1 G0 G1
+    const uint32_t p2 = __byte_perm(lo, hi, 0x5252);   // R0 R1 R0 R1
+    c0 = __dp2a_lo(e.wts, p01, 0u);
+    c1 = __dp2a_hi(e.wts, p01, 0u);
+    c2 = __dp2a_lo(e.wts, p2, 0u);
+}
+
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
     __half2 h = __floats2half2_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);

@@ -4,12 +4,15 @@
 // counts -> offsets[n+1]; then the item table of the requested window (frame, detection,
 // integer crop rectangle).  Integer work only.
 //
-// crop_kernel: HBM-write-bound.  A persistent grid strides over (slot, row band) work items;
-// the number of packed items is read from device memory, so no host synchronisation sits
-// between NMS and cropping.  Each thread produces 8 consecutive pixels of a row for all three
-// planes and writes them with 16-byte stores straight into the slot of the downstream batch.
-// Source taps are 32-bit words fetched through the read-only path (rectangles are small and
-// overlap, so they are served by L1/L2 after first touch).
+// crop_kernel: HBM-bound (the fp16 output is as large as the source rectangles).  A
+// persistent grid strides over (slot, row band) tiles; the number of packed items is read
+// from device memory, so no host synchronisation sits between NMS and cropping.  Per tile the
+// CTA builds a table of horizontal taps (byte offset + exact integer weights per column),
+// one thread has the bulk-copy engine stage the 16-byte aligned segments of the source rows
+// the band taps into shared memory (mbarrier, bounded wait), and every thread then produces
+// 8 consecutive pixels of a row for all three planes: the horizontal lerp is an exact
+// integer two-way dot product per channel, the vertical lerp and all scaling are two fp32
+// operations, and the result leaves as 16-byte stores straight into the downstream slot.
 #include "octo_common.cuh"
 #include "octo_kernels.h"
 
@@ -91,17 +94,37 @@ assemble_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det,
     }
 }
 
+// Bytes of shared memory for staged source rows: two rows of the widest supported frame.
+constexpr int kCropRowBudget = 2 * (3 * kLetterboxMaxWidth + 64);
+constexpr int kCropMaxPassRows = 32;
+
 template <int CAP>
-__global__ void __launch_bounds__(kCropThreads)
+__global__ void __launch_bounds__(kCropThreads, 4)
 crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __restrict__ items,
             const int* __restrict__ n_items, __half* __restrict__ out, int ow, int oh, int band_rows,
-            int swap_rb) {
+            int swap_rb, unsigned int* __restrict__ status) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ float2 s_roww[kCropMaxPassRows];  // vertical weights of the rows of a pass
+
+    unsigned char* const s_rows = smem;
+    XEntry* const s_xtab = reinterpret_cast<XEntry*>(smem + kCropRowBudget);
+
     const int packed = n_items[0];
     const int bands = (oh + band_rows - 1) / band_rows;
     const int chunks = ow >> 3;
     const size_t plane = (size_t)ow * (size_t)oh;
     const float inv_dx = 1.0f / (float)(2 * ow), inv_dy = 1.0f / (float)(2 * oh);
+    // every scale factor folded into the vertical weights: 1 / (255 * den_x * den_y)
+    const float inv_all = 1.0f / (255.0f * (float)(2 * ow) * (float)(2 * oh));
     const long long work = (long long)packed * bands;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    uint32_t phase = 0;
+    bool failed = false;
 
     for (long long wi = blockIdx.x; wi < work; wi += gridDim.x) {
         const int slot = (int)(wi / bands);
@@ -109,56 +132,85 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
         const octo_item_t it = items[slot];
         const FrameDesc& fd = tab.f[it.frame];
         const int cw = it.rx1 - it.rx0, ch = it.ry1 - it.ry0;
-        const int last_word = (fd.pitch >> 2) - 1;
+        // 16-byte aligned byte range of the rectangle's columns inside a frame row
+        const int seg_lo = (3 * it.rx0) & ~15;
+        const int seg = ((3 * it.rx1 + 15) & ~15) - seg_lo;
+        const int stride = seg + 16;
+        int pass_rows = kCropRowBudget / (2 * stride);
+        pass_rows = min(min(pass_rows, kCropMaxPassRows), band_rows);
         __half* const out_slot = out + (size_t)slot * 3 * plane;
-        const int rows = min(band_rows, oh - band * band_rows);
+        const int row_lo = band * band_rows;
+        const int row_hi = min(row_lo + band_rows, oh);
 
-        for (int t = threadIdx.x; t < rows * chunks; t += kCropThreads) {
-            const int r = t / chunks;
-            const int dx0 = (t - r * chunks) << 3;
-            const int dy = band * band_rows + r;
-            int y0, ry;
-            src_coord(dy, ch, oh, inv_dy, y0, ry);
-            const bool lerp_y = ry != 0;
-            const float fy = (float)ry * inv_dy;
-            const uint32_t* row0 =
-                reinterpret_cast<const uint32_t*>(fd.data + (size_t)(it.ry0 + y0) * (size_t)fd.pitch);
-            const uint32_t* row1 = reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(row0) + fd.pitch);
-            float v[3][8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                int x0, rx;
-                src_coord(dx0 + i, cw, ow, inv_dx, x0, rx);
-                const bool lerp_x = rx != 0;
-                const float fx = (float)rx * inv_dx;
-                const int o = 3 * (it.rx0 + x0);
-                uint32_t lo, hi;
-                float a0, a1, a2;
-                load6(row0, o, last_word, lo, hi);
-                row_taps(lo, hi, fx, lerp_x, a0, a1, a2);
-                if (lerp_y) {
-                    float b0, b1, b2;
-                    load6(row1, o, last_word, lo, hi);
-                    row_taps(lo, hi, fx, lerp_x, b0, b1, b2);
-                    a0 = fmaf(fy, b0 - a0, a0);
-                    a1 = fmaf(fy, b1 - a1, a1);
-                    a2 = fmaf(fy, b2 - a2, a2);
+        __syncthreads();  // everyone is done with the previous tile's table and rows
+        for (int dx = threadIdx.x; dx < ow; dx += kCropThreads)
+            s_xtab[dx] = make_xentry(dx, cw, ow, inv_dx, 3 * it.rx0 - seg_lo);
+
+        for (int r0 = row_lo; r0 < row_hi; r0 += pass_rows) {
+            const int nr = min(pass_rows, row_hi - r0);
+            if (r0 != row_lo) __syncthreads();  // previous pass fully consumed
+            if (threadIdx.x == 0) {
+                fence_proxy_async();
+                uint32_t total = 0;
+                for (int r = 0; r < nr; ++r) {
+                    int y0, ry;
+                    src_coord(r0 + r, ch, oh, inv_dy, y0, ry);
+                    total += (uint32_t)seg * (ry != 0 ? 2u : 1u);
+                    s_roww[r] = make_float2((float)(2 * oh - ry) * inv_all, (float)ry * inv_all);
                 }
-                v[0][i] = a0 * (1.0f / 255.0f);
-                v[1][i] = a1 * (1.0f / 255.0f);
-                v[2][i] = a2 * (1.0f / 255.0f);
+                mbar_expect_tx(&bar, total);
+                for (int r = 0; r < nr; ++r) {
+                    int y0, ry;
+                    src_coord(r0 + r, ch, oh, inv_dy, y0, ry);
+                    const uint8_t* src = fd.data + (size_t)(it.ry0 + y0) * (size_t)fd.pitch + seg_lo;
+                    bulk_g2s(s_rows + (size_t)(2 * r) * stride, src, (uint32_t)seg, &bar);
+                    if (ry != 0) bulk_g2s(s_rows + (size_t)(2 * r + 1) * stride, src + fd.pitch, (uint32_t)seg, &bar);
+                }
             }
-            __half* const o0 = out_slot + (size_t)dy * ow + dx0;
+            __syncthreads();  // table, row weights and the armed barrier are visible
+            if (!failed && !mbar_wait_bounded(&bar, phase)) {
+                if (!mbar_wait_bounded(&bar, phase)) failed = true;
+            }
+            phase ^= 1u;
+            if (failed) continue;
+
+            for (int t = threadIdx.x; t < nr * chunks; t += kCropThreads) {
+                const int r = t / chunks;
+                const int dx0 = (t - r * chunks) << 3;
+                const float2 wy = s_roww[r];
+                const bool lerp_y = wy.y != 0.0f;
+                const uint32_t* row0 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(2 * r) * stride);
+                const uint32_t* row1 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(2 * r + 1) * stride);
+                float v[3][8];
 #pragma unroll
-            for (int c = 0; c < 3; ++c) {
-                uint32_t p[4];
+                for (int i = 0; i < 8; ++i) {
+                    const XEntry e = s_xtab[dx0 + i];
+                    uint32_t a0, a1, a2;
+                    hsample(row0, e, a0, a1, a2);
+                    float f0 = __uint2float_rn(a0) * wy.x, f1 = __uint2float_rn(a1) * wy.x,
+                          f2 = __uint2float_rn(a2) * wy.x;
+                    if (lerp_y) {
+                        uint32_t b0, b1, b2;
+                        hsample(row1, e, b0, b1, b2);
+                        f0 = fmaf(__uint2float_rn(b0), wy.y, f0);
+                        f1 = fmaf(__uint2float_rn(b1), wy.y, f1);
+                        f2 = fmaf(__uint2float_rn(b2), wy.y, f2);
+                    }
+                    v[0][i] = f0; v[1][i] = f1; v[2][i] = f2;
+                }
+                __half* const o0 = out_slot + (size_t)(r0 + r) * ow + dx0;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) p[i] = pack_half2(v[c][2 * i], v[c][2 * i + 1]);
-                const int pl = swap_rb ? 2 - c : c;
-                *reinterpret_cast<uint4*>(o0 + (size_t)pl * plane) = make_uint4(p[0], p[1], p[2], p[3]);
+                for (int c = 0; c < 3; ++c) {
+                    uint32_t p[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) p[i] = pack_half2(v[c][2 * i], v[c][2 * i + 1]);
+                    const int pl = swap_rb ? 2 - c : c;
+                    *reinterpret_cast<uint4*>(o0 + (size_t)pl * plane) = make_uint4(p[0], p[1], p[2], p[3]);
+                }
             }
         }
     }
+    if (failed && threadIdx.x == 0) atomicOr(status, 0x4u);
 }
 
 template <int CAP>
@@ -179,12 +231,23 @@ static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     band_rows = band_rows < 1 ? 1 : (band_rows > a.out_h ? a.out_h : band_rows);
     const int bands = (a.out_h + band_rows - 1) / band_rows;
     long long work = (long long)a.max_items * bands;
-    long long cap = (long long)a.sm_count * 8;
+    long long cap = (long long)a.sm_count * 4;
     const int grid = (int)(work < cap ? work : cap);
-    crop_kernel<CAP><<<grid, kCropThreads, 0, stream>>>(tab, a.d_items, a.d_n_items,
-                                                       reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h,
-                                                       band_rows, a.swap_rb);
+    const size_t smem = (size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w;
+    crop_kernel<CAP><<<grid, kCropThreads, smem, stream>>>(tab, a.d_items, a.d_n_items,
+                                                          reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h,
+                                                          band_rows, a.swap_rb, &a.d_ctr->status);
     return cudaGetLastError();
+}
+
+cudaError_t prepare_crop() {
+    const int smem = kCropRowBudget + (int)sizeof(XEntry) * 2048;
+    cudaError_t e;
+    e = cudaFuncSetAttribute(crop_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(crop_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(crop_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 
 cudaError_t launch_assemble(const CropArgs& a, cudaStream_t stream) {

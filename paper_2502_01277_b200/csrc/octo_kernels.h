@@ -53,6 +53,7 @@ struct CropArgs {
 // Opt the kernels of every table capacity into the shared memory they need (current device).
 cudaError_t prepare_letterbox();
 cudaError_t prepare_nms();
+cudaError_t prepare_crop();
 
 cudaError_t launch_letterbox(const FrameDesc* frames, int n, void* d_out, int S, int max_w, int pad_value,
                              int swap_rb, unsigned int* d_status, cudaStream_t stream);

@@ -146,6 +146,7 @@ extern "C" int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** 
     if (e == cudaSuccess) e = dev_alloc(&st->d_ctr, 1, &st->workspace_bytes);
     if (e == cudaSuccess) e = prepare_letterbox();
     if (e == cudaSuccess) e = prepare_nms();
+    if (e == cudaSuccess) e = prepare_crop();
     if (e != cudaSuccess) {
         free_all(st);
         delete st;
