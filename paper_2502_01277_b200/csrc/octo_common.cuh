@@ -129,6 +129,25 @@ __device__ __forceinline__ void hsample(const uint32_t* __restrict__ row, const 
     c2 = __dp2a_lo(e.wts, p2, 0u);
 }
 
+// One destination pixel: horizontal integer lerp on one or two staged rows, then the
+// vertical lerp and all scaling in fp32 (wy.x / wy.y carry 1 / (255 * den_x * den_y)).
+template <bool LERP_Y>
+__device__ __forceinline__ void sample_px(const uint32_t* __restrict__ row0, const uint32_t* __restrict__ row1,
+                                          const XEntry e, const float2 wy, float& f0, float& f1, float& f2) {
+    uint32_t a0, a1, a2;
+    hsample(row0, e, a0, a1, a2);
+    f0 = __uint2float_rn(a0) * wy.x;
+    f1 = __uint2float_rn(a1) * wy.x;
+    f2 = __uint2float_rn(a2) * wy.x;
+    if (LERP_Y) {
+        uint32_t b0, b1, b2;
+        hsample(row1, e, b0, b1, b2);
+        f0 = fmaf(__uint2float_rn(b0), wy.y, f0);
+        f1 = fmaf(__uint2float_rn(b1), wy.y, f1);
+        f2 = fmaf(__uint2float_rn(b2), wy.y, f2);
+    }
+}
+
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
     __half2 h = __floats2half2_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);

@@ -10,9 +10,11 @@
 // CTA builds a table of horizontal taps (byte offset + exact integer weights per column),
 // one thread has the bulk-copy engine stage the 16-byte aligned segments of the source rows
 // the band taps into shared memory (mbarrier, bounded wait), and every thread then produces
-// 8 consecutive pixels of a row for all three planes: the horizontal lerp is an exact
+// pixel pairs (lane l of a warp takes pixels 2l, 2l+1 of a 64-pixel run, so table and row
+// reads of neighbouring lanes fall into neighbouring banks): the horizontal lerp is an exact
 // integer two-way dot product per channel, the vertical lerp and all scaling are two fp32
-// operations, and the result leaves as 16-byte stores straight into the downstream slot.
+// operations, and each warp writes 128 contiguous bytes per plane straight into the
+// downstream slot.
 #include "octo_common.cuh"
 #include "octo_kernels.h"
 
@@ -112,8 +114,9 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
 
     const int packed = n_items[0];
     const int bands = (oh + band_rows - 1) / band_rows;
-    const int chunks = ow >> 3;
+    const int pairs = ow >> 1;
     const size_t plane = (size_t)ow * (size_t)oh;
+    const size_t pl0 = swap_rb ? 2 : 0, pl2 = swap_rb ? 0 : 2;  // planes of input channels 0 and 2
     const float inv_dx = 1.0f / (float)(2 * ow), inv_dy = 1.0f / (float)(2 * oh);
     // every scale factor folded into the vertical weights: 1 / (255 * den_x * den_y)
     const float inv_all = 1.0f / (255.0f * (float)(2 * ow) * (float)(2 * oh));
@@ -149,19 +152,21 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
         for (int r0 = row_lo; r0 < row_hi; r0 += pass_rows) {
             const int nr = min(pass_rows, row_hi - r0);
             if (r0 != row_lo) __syncthreads();  // previous pass fully consumed
-            if (threadIdx.x == 0) {
-                fence_proxy_async();
-                uint32_t total = 0;
-                for (int r = 0; r < nr; ++r) {
-                    int y0, ry;
+            if (threadIdx.x < 32) {
+                // warp 0 stages the pass: lane r owns output row r0 + r
+                const int r = threadIdx.x;
+                int y0 = 0, ry = 0;
+                uint32_t bytes = 0;
+                if (r < nr) {
                     src_coord(r0 + r, ch, oh, inv_dy, y0, ry);
-                    total += (uint32_t)seg * (ry != 0 ? 2u : 1u);
+                    bytes = (uint32_t)seg * (ry != 0 ? 2u : 1u);
                     s_roww[r] = make_float2((float)(2 * oh - ry) * inv_all, (float)ry * inv_all);
                 }
-                mbar_expect_tx(&bar, total);
-                for (int r = 0; r < nr; ++r) {
-                    int y0, ry;
-                    src_coord(r0 + r, ch, oh, inv_dy, y0, ry);
+                const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+                fence_proxy_async();
+                if (r == 0) mbar_expect_tx(&bar, total);
+                __syncwarp();
+                if (r < nr) {
                     const uint8_t* src = fd.data + (size_t)(it.ry0 + y0) * (size_t)fd.pitch + seg_lo;
                     bulk_g2s(s_rows + (size_t)(2 * r) * stride, src, (uint32_t)seg, &bar);
                     if (ry != 0) bulk_g2s(s_rows + (size_t)(2 * r + 1) * stride, src + fd.pitch, (uint32_t)seg, &bar);
@@ -174,39 +179,31 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
             phase ^= 1u;
             if (failed) continue;
 
-            for (int t = threadIdx.x; t < nr * chunks; t += kCropThreads) {
-                const int r = t / chunks;
-                const int dx0 = (t - r * chunks) << 3;
+            // Lane l of a warp takes the pixel pair 2l, 2l+1 of a 64-pixel run: neighbouring
+            // lanes read neighbouring table entries and row words (no bank conflicts) and the
+            // warp writes 128 contiguous bytes per plane.
+            int r = 0, pair = threadIdx.x;
+            while (pair >= pairs) { pair -= pairs; ++r; }
+            for (; r < nr;) {
                 const float2 wy = s_roww[r];
-                const bool lerp_y = wy.y != 0.0f;
                 const uint32_t* row0 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(2 * r) * stride);
                 const uint32_t* row1 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(2 * r + 1) * stride);
-                float v[3][8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const XEntry e = s_xtab[dx0 + i];
-                    uint32_t a0, a1, a2;
-                    hsample(row0, e, a0, a1, a2);
-                    float f0 = __uint2float_rn(a0) * wy.x, f1 = __uint2float_rn(a1) * wy.x,
-                          f2 = __uint2float_rn(a2) * wy.x;
-                    if (lerp_y) {
-                        uint32_t b0, b1, b2;
-                        hsample(row1, e, b0, b1, b2);
-                        f0 = fmaf(__uint2float_rn(b0), wy.y, f0);
-                        f1 = fmaf(__uint2float_rn(b1), wy.y, f1);
-                        f2 = fmaf(__uint2float_rn(b2), wy.y, f2);
-                    }
-                    v[0][i] = f0; v[1][i] = f1; v[2][i] = f2;
+                const uint4 ee = *reinterpret_cast<const uint4*>(s_xtab + 2 * pair);
+                const XEntry e0 = {ee.x, ee.y}, e1 = {ee.z, ee.w};
+                float f[6];
+                if (wy.y != 0.0f) {
+                    sample_px<true>(row0, row1, e0, wy, f[0], f[1], f[2]);
+                    sample_px<true>(row0, row1, e1, wy, f[3], f[4], f[5]);
+                } else {
+                    sample_px<false>(row0, row1, e0, wy, f[0], f[1], f[2]);
+                    sample_px<false>(row0, row1, e1, wy, f[3], f[4], f[5]);
                 }
-                __half* const o0 = out_slot + (size_t)(r0 + r) * ow + dx0;
-#pragma unroll
-                for (int c = 0; c < 3; ++c) {
-                    uint32_t p[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) p[i] = pack_half2(v[c][2 * i], v[c][2 * i + 1]);
-                    const int pl = swap_rb ? 2 - c : c;
-                    *reinterpret_cast<uint4*>(o0 + (size_t)pl * plane) = make_uint4(p[0], p[1], p[2], p[3]);
-                }
+                __half* const o0 = out_slot + (size_t)(r0 + r) * ow + 2 * pair;
+                *reinterpret_cast<uint32_t*>(o0 + pl0 * plane) = pack_half2(f[0], f[3]);
+                *reinterpret_cast<uint32_t*>(o0 + plane) = pack_half2(f[1], f[4]);
+                *reinterpret_cast<uint32_t*>(o0 + pl2 * plane) = pack_half2(f[2], f[5]);
+                pair += kCropThreads;
+                while (pair >= pairs) { pair -= pairs; ++r; }
             }
         }
     }
@@ -227,7 +224,7 @@ template <int CAP>
 static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     static FrameTable<CAP> tab;
     for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
-    int band_rows = 2048 / a.out_w;
+    int band_rows = 4096 / a.out_w;
     band_rows = band_rows < 1 ? 1 : (band_rows > a.out_h ? a.out_h : band_rows);
     const int bands = (a.out_h + band_rows - 1) / band_rows;
     long long work = (long long)a.max_items * bands;

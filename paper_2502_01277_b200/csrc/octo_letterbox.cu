@@ -4,9 +4,11 @@
 // those output rows tap (one row where the vertical weight is zero, e.g. the 3:1 reduction
 // of 1080p, else two) are fetched whole into shared memory by the bulk-copy (TMA) engine
 // with 16-byte coalesced transactions and an mbarrier; rows that carry no weight are never
-// read.  Threads then take 8 consecutive destination pixels each, read the 2x2 taps from
-// shared memory as 32-bit words, interpolate in fp32 with exact rational sampling
-// coordinates and write one 16-byte store per colour plane.
+// read.  While the copies are in flight the CTA builds a table of horizontal taps (byte
+// offset + exact integer weights per canvas column).  Threads then take pixel pairs (lane l
+// of a warp owns pixels 2l, 2l+1 of a 64-pixel run): the horizontal lerp is an exact integer
+// two-way dot product per channel, the vertical lerp and all scaling are two fp32
+// operations, and each warp writes 128 contiguous bytes per colour plane.
 #include "octo_common.cuh"
 #include "octo_kernels.h"
 
@@ -14,7 +16,6 @@ namespace octo {
 
 constexpr int kLbThreads = 256;
 constexpr int kLbRows = 8;  // most output rows a CTA produces; fewer for very wide frames
-constexpr uint32_t kLbFillOff = 0xffffffffu;  // table entry of a canvas column outside the image
 
 template <int CAP>
 __global__ void __launch_bounds__(kLbThreads)
@@ -87,7 +88,7 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
     for (int dx = threadIdx.x; dx < S; dx += kLbThreads) {
         const int ix = dx - pad_l;
         XEntry e;
-        if (ix < 0 || ix >= nw) { e.off = kLbFillOff; e.wts = 0; }
+        if (ix < 0 || ix >= nw) { e.off = 0; e.wts = 0; }  // zero weights mark a canvas column
         else e = make_xentry(ix, w, nw, inv_dx, 0);
         s_xtab[dx] = e;
     }
@@ -99,50 +100,43 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
         if (!copy_ok && threadIdx.x == 0) atomicOr(status, 0x4u);
     }
 
-    for (int t = threadIdx.x; t < nrows * chunks; t += kLbThreads) {
-        const int r = t / chunks;
-        const int dx0 = (t - r * chunks) << 3;
-        __half* const o0 = out_img + (size_t)(dy0 + r) * S + dx0;
+    // Lane l of a warp takes the pixel pair 2l, 2l+1 of a 64-pixel run: neighbouring lanes read
+    // neighbouring table entries and row words, and the warp writes 128 contiguous bytes per plane.
+    const int pairs = S >> 1;
+    const size_t pl0 = swap_rb ? 2 : 0, pl2 = swap_rb ? 0 : 2;  // planes of input channels 0 and 2
+    int r = 0, pair = threadIdx.x;
+    while (pair >= pairs) { pair -= pairs; ++r; }
+    for (; r < nrows;) {
+        __half* const o0 = out_img + (size_t)(dy0 + r) * S + 2 * pair;
         const float2 wy = s_roww[r];
         if (wy.x < 0.0f || !copy_ok) {
-            *reinterpret_cast<uint4*>(o0) = fill4;
-            *reinterpret_cast<uint4*>(o0 + plane) = fill4;
-            *reinterpret_cast<uint4*>(o0 + 2 * plane) = fill4;
-            continue;
-        }
-        const bool lerp_y = wy.y != 0.0f;
-        const int slot = s_rowslot[r];
-        const uint32_t* row0 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)slot * slot_bytes);
-        const uint32_t* row1 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(slot + 1) * slot_bytes);
-
-        float v[3][8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const XEntry e = s_xtab[dx0 + i];
-            if (e.off == kLbFillOff) {
-                v[0][i] = v[1][i] = v[2][i] = fill_f;  // exact fp16 value, converts back unchanged
-                continue;
+            *reinterpret_cast<uint32_t*>(o0) = fill_h2;
+            *reinterpret_cast<uint32_t*>(o0 + plane) = fill_h2;
+            *reinterpret_cast<uint32_t*>(o0 + 2 * plane) = fill_h2;
+        } else {
+            const int slot = s_rowslot[r];
+            const uint32_t* row0 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)slot * slot_bytes);
+            const uint32_t* row1 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(slot + 1) * slot_bytes);
+            const uint4 ee = *reinterpret_cast<const uint4*>(s_xtab + 2 * pair);
+            const XEntry e0 = {ee.x, ee.y}, e1 = {ee.z, ee.w};
+            float f[6];
+            if (wy.y != 0.0f) {
+                sample_px<true>(row0, row1, e0, wy, f[0], f[1], f[2]);
+                sample_px<true>(row0, row1, e1, wy, f[3], f[4], f[5]);
+            } else {
+                sample_px<false>(row0, row1, e0, wy, f[0], f[1], f[2]);
+                sample_px<false>(row0, row1, e1, wy, f[3], f[4], f[5]);
             }
-            uint32_t a0, a1, a2;
-            hsample(row0, e, a0, a1, a2);
-            float f0 = __uint2float_rn(a0) * wy.x, f1 = __uint2float_rn(a1) * wy.x, f2 = __uint2float_rn(a2) * wy.x;
-            if (lerp_y) {
-                uint32_t b0, b1, b2;
-                hsample(row1, e, b0, b1, b2);
-                f0 = fmaf(__uint2float_rn(b0), wy.y, f0);
-                f1 = fmaf(__uint2float_rn(b1), wy.y, f1);
-                f2 = fmaf(__uint2float_rn(b2), wy.y, f2);
-            }
-            v[0][i] = f0; v[1][i] = f1; v[2][i] = f2;
+            // canvas columns outside the image carry zero weights: replace them by the fill
+            // (an exact fp16 value, so it converts back unchanged)
+            if (e0.wts == 0u) { f[0] = fill_f; f[1] = fill_f; f[2] = fill_f; }
+            if (e1.wts == 0u) { f[3] = fill_f; f[4] = fill_f; f[5] = fill_f; }
+            *reinterpret_cast<uint32_t*>(o0 + pl0 * plane) = pack_half2(f[0], f[3]);
+            *reinterpret_cast<uint32_t*>(o0 + plane) = pack_half2(f[1], f[4]);
+            *reinterpret_cast<uint32_t*>(o0 + pl2 * plane) = pack_half2(f[2], f[5]);
         }
-#pragma unroll
-        for (int c = 0; c < 3; ++c) {
-            uint32_t p[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) p[i] = pack_half2(v[c][2 * i], v[c][2 * i + 1]);
-            const int pl = swap_rb ? 2 - c : c;  // input channel c lands in plane pl
-            *reinterpret_cast<uint4*>(o0 + (size_t)pl * plane) = make_uint4(p[0], p[1], p[2], p[3]);
-        }
+        pair += kLbThreads;
+        while (pair >= pairs) { pair -= pairs; ++r; }
     }
 }
 
