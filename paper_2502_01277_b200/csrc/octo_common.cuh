@@ -113,38 +113,40 @@ __device__ __forceinline__ XEntry make_xentry(int d, int src, int dst, float inv
     return e;
 }
 
-// Integer horizontal lerp of the three channels of one destination pixel from a staged row
-// (4-byte aligned words in shared memory, with at least 12 readable bytes past any offset).
-__device__ __forceinline__ void hsample(const uint32_t* __restrict__ row, const XEntry e, uint32_t& c0, uint32_t& c1,
-                                        uint32_t& c2) {
-    const uint32_t wi = e.off >> 2;
-    const uint32_t sh = (e.off & 3u) * 8u;
-    const uint32_t a = row[wi], b = row[wi + 1], c = row[wi + 2];
+// Integer horizontal lerp of the three channels of one destination pixel.  `row` is the byte
+// address of a staged row (4-byte aligned, shared memory, at least 12 readable bytes past
+// any offset); `woff` = e.off & ~3 and `sh` = 8 * (e.off & 3) are shared by both rows.
+__device__ __forceinline__ void hsample(const unsigned char* __restrict__ row, uint32_t woff, uint32_t sh,
+                                        uint32_t wts, uint32_t& c0, uint32_t& c1, uint32_t& c2) {
+    const uint32_t* p = reinterpret_cast<const uint32_t*>(row + woff);
+    const uint32_t a = p[0], b = p[1], c = p[2];
     const uint32_t lo = __funnelshift_r(a, b, sh);  // B0 G0 R0 B1
     const uint32_t hi = __funnelshift_r(b, c, sh);  // G1 R1 .. ..
     const uint32_t p01 = __byte_perm(lo, hi, 0x4130);  // B0 B1 G0 G1
     const uint32_t p2 = __byte_perm(lo, hi, 0x5252);   // R0 R1 R0 R1
-    c0 = __dp2a_lo(e.wts, p01, 0u);
-    c1 = __dp2a_hi(e.wts, p01, 0u);
-    c2 = __dp2a_lo(e.wts, p2, 0u);
+    c0 = __dp2a_lo(wts, p01, 0u);
+    c1 = __dp2a_hi(wts, p01, 0u);
+    c2 = __dp2a_lo(wts, p2, 0u);
 }
 
 // One destination pixel: horizontal integer lerp on one or two staged rows, then the
-// vertical lerp and all scaling in fp32 (wy.x / wy.y carry 1 / (255 * den_x * den_y)).
+// vertical lerp and all scaling in fp32 (wx / wy carry 1 / (255 * den_x * den_y)).
 template <bool LERP_Y>
-__device__ __forceinline__ void sample_px(const uint32_t* __restrict__ row0, const uint32_t* __restrict__ row1,
-                                          const XEntry e, const float2 wy, float& f0, float& f1, float& f2) {
+__device__ __forceinline__ void sample_px(const unsigned char* __restrict__ row0,
+                                          const unsigned char* __restrict__ row1, const XEntry e, float wx,
+                                          float wy, float& f0, float& f1, float& f2) {
+    const uint32_t woff = e.off & ~3u, sh = (e.off & 3u) << 3;
     uint32_t a0, a1, a2;
-    hsample(row0, e, a0, a1, a2);
-    f0 = __uint2float_rn(a0) * wy.x;
-    f1 = __uint2float_rn(a1) * wy.x;
-    f2 = __uint2float_rn(a2) * wy.x;
+    hsample(row0, woff, sh, e.wts, a0, a1, a2);
+    f0 = __uint2float_rn(a0) * wx;
+    f1 = __uint2float_rn(a1) * wx;
+    f2 = __uint2float_rn(a2) * wx;
     if (LERP_Y) {
         uint32_t b0, b1, b2;
-        hsample(row1, e, b0, b1, b2);
-        f0 = fmaf(__uint2float_rn(b0), wy.y, f0);
-        f1 = fmaf(__uint2float_rn(b1), wy.y, f1);
-        f2 = fmaf(__uint2float_rn(b2), wy.y, f2);
+        hsample(row1, woff, sh, e.wts, b0, b1, b2);
+        f0 = fmaf(__uint2float_rn(b0), wy, f0);
+        f1 = fmaf(__uint2float_rn(b1), wy, f1);
+        f2 = fmaf(__uint2float_rn(b2), wy, f2);
     }
 }
 
@@ -152,6 +154,41 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
     __half2 h = __floats2half2_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);
 }
+
+// One output row (or column tile of it) by one warp: lane l owns the pixel pairs l, l + 32, ...
+// so neighbouring lanes read neighbouring table entries and row words (no bank conflicts)
+// and the warp writes 128 contiguous bytes per plane and step.  o0 / o1 / o2 point at the
+// row's first pixel in the planes of input channels 0 / 1 / 2.  With FILL, columns whose
+// table entry has zero weights (canvas outside the image) receive fill_f.
+template <bool LERP_Y, bool FILL>
+__device__ __forceinline__ void sample_row(const unsigned char* __restrict__ row0,
+                                           const unsigned char* __restrict__ row1, float wx, float wy,
+                                           const XEntry* __restrict__ xt, int pairs, int lane,
+                                           __half* __restrict__ o0, __half* __restrict__ o1,
+                                           __half* __restrict__ o2, float fill_f) {
+    for (int pair = lane; pair < pairs; pair += 32) {
+        const uint4 ee = *reinterpret_cast<const uint4*>(xt + 2 * pair);
+        const XEntry e0 = {ee.x, ee.y}, e1 = {ee.z, ee.w};
+        float a0, a1, a2, b0, b1, b2;
+        sample_px<LERP_Y>(row0, row1, e0, wx, wy, a0, a1, a2);
+        sample_px<LERP_Y>(row0, row1, e1, wx, wy, b0, b1, b2);
+        if (FILL) {
+            if (e0.wts == 0u) { a0 = fill_f; a1 = fill_f; a2 = fill_f; }
+            if (e1.wts == 0u) { b0 = fill_f; b1 = fill_f; b2 = fill_f; }
+        }
+        *reinterpret_cast<uint32_t*>(o0 + 2 * pair) = pack_half2(a0, b0);
+        *reinterpret_cast<uint32_t*>(o1 + 2 * pair) = pack_half2(a1, b1);
+        *reinterpret_cast<uint32_t*>(o2 + 2 * pair) = pack_half2(a2, b2);
+    }
+}
+
+// What a warp needs to know about one output row of a staged pass.
+struct RowInfo {
+    int32_t row0;  // byte offset of the first staged row inside the row buffer; < 0: canvas row
+    int32_t row1;  // byte offset of the second staged row (unused when wy == 0)
+    float wx, wy;  // vertical weights with all scaling folded in
+};
+
 
 // ---------------------------------------------------------------------------------------
 // mbarrier + bulk-copy (TMA engine, untiled) helpers.  Every wait is bounded.

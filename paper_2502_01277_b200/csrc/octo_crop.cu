@@ -96,116 +96,208 @@ assemble_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det,
     }
 }
 
-// Bytes of shared memory for staged source rows: two rows of the widest supported frame.
-constexpr int kCropRowBudget = 2 * (3 * kLetterboxMaxWidth + 64);
+// Shared memory for staged source rows.  A pass stages two row segments per output row; a
+// segment longer than kCropMaxStride - 16 bytes (a rectangle wider than about 4000 pixels)
+// is split into column tiles, so one row pair always fits.  Two buffers: while the CTA
+// computes one pass, the bulk copies of the next are in flight.
+constexpr int kCropRowBudget = 24576;
+constexpr int kCropMaxStride = kCropRowBudget / 2;
+constexpr int kCropTilePx = 4000;
 constexpr int kCropMaxPassRows = 32;
+constexpr int kCropCtasPerSm = 4;
+
+// One pass of a CTA: output rows [r0, r0 + nr) x columns [c0, c0 + ncols) of one item.  Warp 0
+// walks the CTA's sequence of passes and publishes each one here for the other warps.
+struct __align__(16) CropPass {
+    int32_t valid;     // 0: no more passes
+    int32_t new_item;  // first pass of its (slot, band) tile: the tap table has to be built
+    int32_t slot, r0, nr, c0, ncols;
+    int32_t rx0, cw;   // rectangle columns, for the tap table
+    int32_t _pad[3];
+};
 
 template <int CAP>
-__global__ void __launch_bounds__(kCropThreads, 4)
+__global__ void __launch_bounds__(kCropThreads, kCropCtasPerSm)
 crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __restrict__ items,
             const int* __restrict__ n_items, __half* __restrict__ out, int ow, int oh, int band_rows,
             int swap_rb, unsigned int* __restrict__ status) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t bar;
-    __shared__ float2 s_roww[kCropMaxPassRows];  // vertical weights of the rows of a pass
+    __shared__ __align__(8) uint64_t bar[2];
+    __shared__ CropPass s_pass[2];
+    __shared__ __align__(16) RowInfo s_row[2][kCropMaxPassRows];  // per-row data of the staged passes
 
-    unsigned char* const s_rows = smem;
-    XEntry* const s_xtab = reinterpret_cast<XEntry*>(smem + kCropRowBudget);
+    unsigned char* const s_rows0 = smem;
+    XEntry* const s_xtab = reinterpret_cast<XEntry*>(smem + 2 * kCropRowBudget);
 
     const int packed = n_items[0];
     const int bands = (oh + band_rows - 1) / band_rows;
-    const int pairs = ow >> 1;
     const size_t plane = (size_t)ow * (size_t)oh;
-    const size_t pl0 = swap_rb ? 2 : 0, pl2 = swap_rb ? 0 : 2;  // planes of input channels 0 and 2
     const float inv_dx = 1.0f / (float)(2 * ow), inv_dy = 1.0f / (float)(2 * oh);
     // every scale factor folded into the vertical weights: 1 / (255 * den_x * den_y)
     const float inv_all = 1.0f / (255.0f * (float)(2 * ow) * (float)(2 * oh));
-    const long long work = (long long)packed * bands;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    // ---- state of the pass sequence, meaningful in warp 0 only --------------------------------
+    // tile index = slot * bands + band, advanced by gridDim.x per tile without divisions
+    const int step_slot = (int)(gridDim.x / (unsigned)bands), step_band = (int)(gridDim.x % (unsigned)bands);
+    int w_slot = (int)(blockIdx.x / (unsigned)bands), w_band = (int)(blockIdx.x % (unsigned)bands);
+    int w_frame = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
+    int w_row_lo = 0, w_row_hi = 0, w_tile_cols = ow;
+    int w_c0 = 0, w_ncols = 0, w_r0 = 0, w_nr = 0;
+    int w_seg_lo = 0, w_seg = 0, w_stride = 16, w_pass_rows = 1;
+    bool w_valid = false, w_new = false;
+
+    // geometry of the column tile starting at w_c0
+    auto set_tile = [&]() {
+        w_ncols = min(w_tile_cols, ow - w_c0);
+        const int full_lo = (3 * w_rx0) & ~15;
+        const int full_hi = (3 * (w_rx0 + w_cw) + 15) & ~15;
+        int lo = full_lo, hi = full_hi;
+        if (w_tile_cols != ow) {
+            int xa, xb, rem;
+            src_coord(w_c0, w_cw, ow, inv_dx, xa, rem);
+            src_coord(w_c0 + w_ncols - 1, w_cw, ow, inv_dx, xb, rem);
+            lo = (3 * (w_rx0 + xa)) & ~15;
+            hi = min((3 * (w_rx0 + xb) + 6 + 15) & ~15, full_hi);
+        }
+        w_seg_lo = lo;
+        w_seg = hi - lo;
+        w_stride = w_seg + 16;
+        // whole multiples of the warp count keep every warp busy (one warp per row)
+        int pr = min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows);
+        if (pr >= kCropThreads / 32) pr &= ~(kCropThreads / 32 - 1);
+        w_pass_rows = max(1, min(pr, band_rows));
+    };
+    // first pass of the tile (w_slot, w_band), if there is one
+    auto open_tile = [&]() {
+        w_valid = w_slot < packed;
+        if (!w_valid) return;
+        const octo_item_t it = items[w_slot];
+        w_frame = it.frame;
+        w_rx0 = it.rx0; w_ry0 = it.ry0; w_cw = it.rx1 - it.rx0; w_ch = it.ry1 - it.ry0;
+        const int full = ((3 * it.rx1 + 15) & ~15) - ((3 * it.rx0) & ~15);
+        w_tile_cols = (full + 16 > kCropMaxStride) ? max(2, (int)((long long)kCropTilePx * ow / w_cw) & ~1) : ow;
+        w_c0 = 0;
+        set_tile();
+        w_row_lo = w_band * band_rows;
+        w_row_hi = min(w_row_lo + band_rows, oh);
+        w_r0 = w_row_lo;
+        w_nr = min(w_pass_rows, w_row_hi - w_r0);
+        w_new = true;
+    };
+    auto advance = [&]() {
+        w_new = false;
+        if (w_r0 + w_nr < w_row_hi) {
+            w_r0 += w_nr;
+        } else if (w_c0 + w_ncols < ow) {
+            w_c0 += w_ncols;
+            set_tile();
+            w_r0 = w_row_lo;
+        } else {
+            w_slot += step_slot;
+            w_band += step_band;
+            if (w_band >= bands) { w_band -= bands; w_slot += 1; }
+            open_tile();
+            return;
+        }
+        w_nr = min(w_pass_rows, w_row_hi - w_r0);
+    };
+    // warp 0: publish the current pass in s_pass[b] and start its bulk copies into row buffer b
+    // (lane r owns output row w_r0 + r)
+    auto publish_and_stage = [&](int b) {
+        if (lane == 0) {
+            CropPass p;
+            p.valid = w_valid ? 1 : 0;
+            p.new_item = w_new ? 1 : 0;
+            p.slot = w_slot; p.r0 = w_r0; p.nr = w_nr; p.c0 = w_c0; p.ncols = w_ncols;
+            p.rx0 = w_rx0; p.cw = w_cw;
+            p._pad[0] = p._pad[1] = p._pad[2] = 0;
+            s_pass[b] = p;
+        }
+        if (!w_valid) return;
+        const FrameDesc& fd = tab.f[w_frame];
+        int y0 = 0, ry = 0;
+        uint32_t bytes = 0;
+        if (lane < w_nr) {
+            src_coord(w_r0 + lane, w_ch, oh, inv_dy, y0, ry);
+            bytes = (uint32_t)w_seg * (ry != 0 ? 2u : 1u);
+            RowInfo ri;
+            ri.row0 = 2 * lane * w_stride - w_seg_lo;  // table offsets are relative to the frame row
+            ri.row1 = ri.row0 + w_stride;
+            ri.wx = (float)(2 * oh - ry) * inv_all;
+            ri.wy = (float)ry * inv_all;
+            s_row[b][lane] = ri;
+        }
+        const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+        fence_proxy_async();
+        if (lane == 0) mbar_expect_tx(&bar[b], total);
+        __syncwarp();
+        if (lane < w_nr) {
+            unsigned char* dst = s_rows0 + (size_t)b * kCropRowBudget + (size_t)(2 * lane) * w_stride;
+            const uint8_t* src = fd.data + (size_t)(w_ry0 + y0) * (size_t)fd.pitch + w_seg_lo;
+            bulk_g2s(dst, src, (uint32_t)w_seg, &bar[b]);
+            if (ry != 0) bulk_g2s(dst + w_stride, src + fd.pitch, (uint32_t)w_seg, &bar[b]);
+        }
+    };
 
     if (threadIdx.x == 0) {
-        mbar_init(&bar, 1);
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
         mbar_fence_init();
     }
-    uint32_t phase = 0;
+    __syncthreads();
+    if (warp == 0) {
+        open_tile();
+        publish_and_stage(0);
+    }
+    __syncthreads();
+
+    uint32_t phase[2] = {0u, 0u};
     bool failed = false;
+    int buf = 0;
+    __half* const out0 = out + (swap_rb ? 2 : 0) * plane;  // plane of input channel 0
+    __half* const out1 = out + plane;
+    __half* const out2 = out + (swap_rb ? 0 : 2) * plane;  // plane of input channel 2
 
-    for (long long wi = blockIdx.x; wi < work; wi += gridDim.x) {
-        const int slot = (int)(wi / bands);
-        const int band = (int)(wi - (long long)slot * bands);
-        const octo_item_t it = items[slot];
-        const FrameDesc& fd = tab.f[it.frame];
-        const int cw = it.rx1 - it.rx0, ch = it.ry1 - it.ry0;
-        // 16-byte aligned byte range of the rectangle's columns inside a frame row
-        const int seg_lo = (3 * it.rx0) & ~15;
-        const int seg = ((3 * it.rx1 + 15) & ~15) - seg_lo;
-        const int stride = seg + 16;
-        int pass_rows = kCropRowBudget / (2 * stride);
-        pass_rows = min(min(pass_rows, kCropMaxPassRows), band_rows);
-        __half* const out_slot = out + (size_t)slot * 3 * plane;
-        const int row_lo = band * band_rows;
-        const int row_hi = min(row_lo + band_rows, oh);
+    for (;;) {
+        const CropPass cur = s_pass[buf];
+        if (!cur.valid) break;
+        if (cur.new_item) {
+            // taps of every output column: byte offset inside a frame row + integer weights.  The
+            // previous tile's table was last read before the barrier that ended the previous pass.
+            for (int dx = threadIdx.x; dx < ow; dx += kCropThreads)
+                s_xtab[dx] = make_xentry(dx, cur.cw, ow, inv_dx, 3 * cur.rx0);
+        }
+        if (warp == 0) {
+            advance();
+            publish_and_stage(buf ^ 1);  // in flight while cur is computed
+        }
+        __syncthreads();  // table, next pass record, row data and armed barriers are visible
 
-        __syncthreads();  // everyone is done with the previous tile's table and rows
-        for (int dx = threadIdx.x; dx < ow; dx += kCropThreads)
-            s_xtab[dx] = make_xentry(dx, cw, ow, inv_dx, 3 * it.rx0 - seg_lo);
+        if (!failed && !mbar_wait_bounded(&bar[buf], phase[buf])) {
+            if (!mbar_wait_bounded(&bar[buf], phase[buf])) failed = true;
+        }
+        phase[buf] ^= 1u;
 
-        for (int r0 = row_lo; r0 < row_hi; r0 += pass_rows) {
-            const int nr = min(pass_rows, row_hi - r0);
-            if (r0 != row_lo) __syncthreads();  // previous pass fully consumed
-            if (threadIdx.x < 32) {
-                // warp 0 stages the pass: lane r owns output row r0 + r
-                const int r = threadIdx.x;
-                int y0 = 0, ry = 0;
-                uint32_t bytes = 0;
-                if (r < nr) {
-                    src_coord(r0 + r, ch, oh, inv_dy, y0, ry);
-                    bytes = (uint32_t)seg * (ry != 0 ? 2u : 1u);
-                    s_roww[r] = make_float2((float)(2 * oh - ry) * inv_all, (float)ry * inv_all);
-                }
-                const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
-                fence_proxy_async();
-                if (r == 0) mbar_expect_tx(&bar, total);
-                __syncwarp();
-                if (r < nr) {
-                    const uint8_t* src = fd.data + (size_t)(it.ry0 + y0) * (size_t)fd.pitch + seg_lo;
-                    bulk_g2s(s_rows + (size_t)(2 * r) * stride, src, (uint32_t)seg, &bar);
-                    if (ry != 0) bulk_g2s(s_rows + (size_t)(2 * r + 1) * stride, src + fd.pitch, (uint32_t)seg, &bar);
-                }
-            }
-            __syncthreads();  // table, row weights and the armed barrier are visible
-            if (!failed && !mbar_wait_bounded(&bar, phase)) {
-                if (!mbar_wait_bounded(&bar, phase)) failed = true;
-            }
-            phase ^= 1u;
-            if (failed) continue;
-
-            // Lane l of a warp takes the pixel pair 2l, 2l+1 of a 64-pixel run: neighbouring
-            // lanes read neighbouring table entries and row words (no bank conflicts) and the
-            // warp writes 128 contiguous bytes per plane.
-            int r = 0, pair = threadIdx.x;
-            while (pair >= pairs) { pair -= pairs; ++r; }
-            for (; r < nr;) {
-                const float2 wy = s_roww[r];
-                const uint32_t* row0 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(2 * r) * stride);
-                const uint32_t* row1 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(2 * r + 1) * stride);
-                const uint4 ee = *reinterpret_cast<const uint4*>(s_xtab + 2 * pair);
-                const XEntry e0 = {ee.x, ee.y}, e1 = {ee.z, ee.w};
-                float f[6];
-                if (wy.y != 0.0f) {
-                    sample_px<true>(row0, row1, e0, wy, f[0], f[1], f[2]);
-                    sample_px<true>(row0, row1, e1, wy, f[3], f[4], f[5]);
-                } else {
-                    sample_px<false>(row0, row1, e0, wy, f[0], f[1], f[2]);
-                    sample_px<false>(row0, row1, e1, wy, f[3], f[4], f[5]);
-                }
-                __half* const o0 = out_slot + (size_t)(r0 + r) * ow + 2 * pair;
-                *reinterpret_cast<uint32_t*>(o0 + pl0 * plane) = pack_half2(f[0], f[3]);
-                *reinterpret_cast<uint32_t*>(o0 + plane) = pack_half2(f[1], f[4]);
-                *reinterpret_cast<uint32_t*>(o0 + pl2 * plane) = pack_half2(f[2], f[5]);
-                pair += kCropThreads;
-                while (pair >= pairs) { pair -= pairs; ++r; }
+        if (!failed) {
+            // one warp per output row of the pass
+            const XEntry* const xt = s_xtab + cur.c0;
+            const unsigned char* const rows = s_rows0 + (size_t)buf * kCropRowBudget;
+            const size_t tile_off = (size_t)cur.slot * 3 * plane + (size_t)cur.r0 * ow + cur.c0;
+            const int pairs = cur.ncols >> 1;
+            for (int r = warp; r < cur.nr; r += kCropThreads / 32) {
+                const RowInfo ri = s_row[buf][r];
+                const size_t o = tile_off + (size_t)(r * ow);
+                if (ri.wy != 0.0f)
+                    sample_row<true, false>(rows + ri.row0, rows + ri.row1, ri.wx, ri.wy, xt, pairs, lane, out0 + o,
+                                            out1 + o, out2 + o, 0.0f);
+                else
+                    sample_row<false, false>(rows + ri.row0, rows + ri.row1, ri.wx, ri.wy, xt, pairs, lane, out0 + o,
+                                             out1 + o, out2 + o, 0.0f);
             }
         }
+        __syncthreads();  // cur's rows, row data and pass record may now be overwritten
+        buf ^= 1;
     }
     if (failed && threadIdx.x == 0) atomicOr(status, 0x4u);
 }
@@ -224,13 +316,15 @@ template <int CAP>
 static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     static FrameTable<CAP> tab;
     for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
-    int band_rows = 4096 / a.out_w;
-    band_rows = band_rows < 1 ? 1 : (band_rows > a.out_h ? a.out_h : band_rows);
+    // rows per (slot, band) tile: about 4096 pixels, a multiple of the warp count
+    int band_rows = (4096 / a.out_w) & ~7;
+    band_rows = band_rows < 8 ? 8 : band_rows;
+    band_rows = band_rows > a.out_h ? a.out_h : band_rows;
     const int bands = (a.out_h + band_rows - 1) / band_rows;
     long long work = (long long)a.max_items * bands;
-    long long cap = (long long)a.sm_count * 4;
+    long long cap = (long long)a.sm_count * kCropCtasPerSm;
     const int grid = (int)(work < cap ? work : cap);
-    const size_t smem = (size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w;
+    const size_t smem = 2 * (size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w;
     crop_kernel<CAP><<<grid, kCropThreads, smem, stream>>>(tab, a.d_items, a.d_n_items,
                                                           reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h,
                                                           band_rows, a.swap_rb, &a.d_ctr->status);
@@ -238,7 +332,7 @@ static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
 }
 
 cudaError_t prepare_crop() {
-    const int smem = kCropRowBudget + (int)sizeof(XEntry) * 2048;
+    const int smem = 2 * kCropRowBudget + (int)sizeof(XEntry) * 2048;
     cudaError_t e;
     e = cudaFuncSetAttribute(crop_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;

@@ -23,8 +23,7 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
                  int slot_bytes, uint32_t fill_h2, float fill_f, int swap_rb, unsigned int* __restrict__ status) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t bar;
-    __shared__ float2 s_roww[kLbRows];  // vertical weights; x < 0 marks a canvas (pad) row
-    __shared__ int s_rowslot[kLbRows];  // first staging slot of the row
+    __shared__ __align__(16) RowInfo s_row[kLbRows];  // per-row data; row0 < 0 marks a canvas (pad) row
 
     const FrameDesc& fd = tab.f[blockIdx.y];
     const int dy0 = blockIdx.x * band_rows;
@@ -63,11 +62,16 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
         int slot = 0;
         for (int r = 0; r < nrows; ++r) {
             const int iy = dy0 + r - pad_t;
-            if (iy < 0 || iy >= nh) { s_roww[r] = make_float2(-1.0f, 0.0f); s_rowslot[r] = 0; continue; }
+            RowInfo ri;
+            ri.row0 = -1; ri.row1 = 0; ri.wx = 0.0f; ri.wy = 0.0f;
+            if (iy < 0 || iy >= nh) { s_row[r] = ri; continue; }
             int y0, ry;
             src_coord(iy, h, nh, inv_dy, y0, ry);
-            s_roww[r] = make_float2((float)(2 * nh - ry) * inv_all, (float)ry * inv_all);
-            s_rowslot[r] = slot;
+            ri.row0 = slot * slot_bytes;
+            ri.row1 = ri.row0 + slot_bytes;
+            ri.wx = (float)(2 * nh - ry) * inv_all;
+            ri.wy = (float)ry * inv_all;
+            s_row[r] = ri;
             slot += ry != 0 ? 2 : 1;
             total += row_bytes * (ry != 0 ? 2u : 1u);
         }
@@ -100,43 +104,28 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
         if (!copy_ok && threadIdx.x == 0) atomicOr(status, 0x4u);
     }
 
-    // Lane l of a warp takes the pixel pair 2l, 2l+1 of a 64-pixel run: neighbouring lanes read
-    // neighbouring table entries and row words, and the warp writes 128 contiguous bytes per plane.
+    // one warp per output row of the band
     const int pairs = S >> 1;
-    const size_t pl0 = swap_rb ? 2 : 0, pl2 = swap_rb ? 0 : 2;  // planes of input channels 0 and 2
-    int r = 0, pair = threadIdx.x;
-    while (pair >= pairs) { pair -= pairs; ++r; }
-    for (; r < nrows;) {
-        __half* const o0 = out_img + (size_t)(dy0 + r) * S + 2 * pair;
-        const float2 wy = s_roww[r];
-        if (wy.x < 0.0f || !copy_ok) {
-            *reinterpret_cast<uint32_t*>(o0) = fill_h2;
-            *reinterpret_cast<uint32_t*>(o0 + plane) = fill_h2;
-            *reinterpret_cast<uint32_t*>(o0 + 2 * plane) = fill_h2;
-        } else {
-            const int slot = s_rowslot[r];
-            const uint32_t* row0 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)slot * slot_bytes);
-            const uint32_t* row1 = reinterpret_cast<const uint32_t*>(s_rows + (size_t)(slot + 1) * slot_bytes);
-            const uint4 ee = *reinterpret_cast<const uint4*>(s_xtab + 2 * pair);
-            const XEntry e0 = {ee.x, ee.y}, e1 = {ee.z, ee.w};
-            float f[6];
-            if (wy.y != 0.0f) {
-                sample_px<true>(row0, row1, e0, wy, f[0], f[1], f[2]);
-                sample_px<true>(row0, row1, e1, wy, f[3], f[4], f[5]);
-            } else {
-                sample_px<false>(row0, row1, e0, wy, f[0], f[1], f[2]);
-                sample_px<false>(row0, row1, e1, wy, f[3], f[4], f[5]);
+    const int lane = threadIdx.x & 31;
+    __half* const out0 = out_img + (swap_rb ? 2 : 0) * plane;  // plane of input channel 0
+    __half* const out1 = out_img + plane;
+    __half* const out2 = out_img + (swap_rb ? 0 : 2) * plane;  // plane of input channel 2
+    for (int r = threadIdx.x >> 5; r < nrows; r += kLbThreads / 32) {
+        const RowInfo ri = s_row[r];
+        const size_t o = (size_t)(dy0 + r) * S;
+        if (ri.row0 < 0 || !copy_ok) {
+            for (int pair = lane; pair < pairs; pair += 32) {
+                *reinterpret_cast<uint32_t*>(out0 + o + 2 * pair) = fill_h2;
+                *reinterpret_cast<uint32_t*>(out1 + o + 2 * pair) = fill_h2;
+                *reinterpret_cast<uint32_t*>(out2 + o + 2 * pair) = fill_h2;
             }
-            // canvas columns outside the image carry zero weights: replace them by the fill
-            // (an exact fp16 value, so it converts back unchanged)
-            if (e0.wts == 0u) { f[0] = fill_f; f[1] = fill_f; f[2] = fill_f; }
-            if (e1.wts == 0u) { f[3] = fill_f; f[4] = fill_f; f[5] = fill_f; }
-            *reinterpret_cast<uint32_t*>(o0 + pl0 * plane) = pack_half2(f[0], f[3]);
-            *reinterpret_cast<uint32_t*>(o0 + plane) = pack_half2(f[1], f[4]);
-            *reinterpret_cast<uint32_t*>(o0 + pl2 * plane) = pack_half2(f[2], f[5]);
+        } else if (ri.wy != 0.0f) {
+            sample_row<true, true>(s_rows + ri.row0, s_rows + ri.row1, ri.wx, ri.wy, s_xtab, pairs, lane, out0 + o,
+                                   out1 + o, out2 + o, fill_f);
+        } else {
+            sample_row<false, true>(s_rows + ri.row0, s_rows + ri.row1, ri.wx, ri.wy, s_xtab, pairs, lane, out0 + o,
+                                    out1 + o, out2 + o, fill_f);
         }
-        pair += kLbThreads;
-        while (pair >= pairs) { pair -= pairs; ++r; }
     }
 }
 

@@ -338,3 +338,35 @@ def test_crop_shapes_and_degenerate_boxes():
             _check_branch(res, ref, 0)
         finally:
             st.close()
+
+
+def test_crop_of_very_wide_rectangles_is_tiled_by_columns():
+    """Rectangles wider than one staging buffer (about 4000 source pixels) are processed in
+    column tiles; results must not show the seams."""
+    import paper_2502_01277_b200 as octo
+    rng = np.random.default_rng(8)
+    w, h, s = 7000, 24, 640
+    pitch = (3 * w + 15) // 16 * 16
+    img = np.zeros((h, pitch), dtype=np.uint8)
+    img[:, :3 * w] = rng.integers(0, 256, size=(h, 3 * w), dtype=np.uint8)
+    C, A = 4, 64
+    head = np.full((1, A, 5 + C), -9.0, dtype=np.float32)
+    nw, nh, pl, pt = oracle.letterbox_geometry(w, h, s)
+    g = w / nw
+    boxes = [(3500, 12, 7000, 24), (2100, 10, 4100, 8), (5000, 5, 3990, 6), (6000, 20, 1500, 4)]
+    for k, (cx, cy, bw, bh) in enumerate(boxes):
+        head[0, k, :4] = [cx / g + pl, cy / g + pt, bw / g, bh / g]
+        head[0, k, 4] = 4.0 - 0.1 * k
+        head[0, k, 5 + k] = 5.0
+    for (ow, oh) in [(224, 16), (1024, 8), (8, 8)]:
+        st = octo.Stage(net_size=s, max_batch=1, num_anchors=A, num_classes=C, branches=((ow, oh),))
+        try:
+            res = run_stage_gpu(st, [img], [(w, h)], head)
+            ref = oracle.run_stage([img], [(w, h)], head, s, ((ow, oh),))
+            assert ref.counts[0] == len(boxes)
+            assert (ref.rects[0][:, 2] - ref.rects[0][:, 0]).max() > 6000
+            _check_dets(res, ref)
+            _check_branch(res, ref, 0)
+            assert res.status == 0
+        finally:
+            st.close()
