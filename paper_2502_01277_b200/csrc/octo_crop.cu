@@ -21,7 +21,6 @@
 namespace octo {
 
 constexpr int kAsmThreads = 1024;
-constexpr int kCropThreads = 256;
 
 template <int CAP>
 __global__ void __launch_bounds__(kAsmThreads)
@@ -98,195 +97,206 @@ assemble_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det,
 
 // Shared memory for staged source rows.  A pass stages two row segments per output row; a
 // segment longer than kCropMaxStride - 16 bytes (a rectangle wider than about 4000 pixels)
-// is split into column tiles, so one row pair always fits.  Two buffers: while the CTA
-// computes one pass, the bulk copies of the next are in flight.
+// is split into column tiles, so one row pair always fits.  Two buffers form a ring between
+// the producer warp and the consumer warps.
 constexpr int kCropRowBudget = 24576;
 constexpr int kCropMaxStride = kCropRowBudget / 2;
 constexpr int kCropTilePx = 4000;
 constexpr int kCropMaxPassRows = 32;
 constexpr int kCropCtasPerSm = 4;
+constexpr int kCropConsumerWarps = 8;
+constexpr int kCropKernelThreads = 32 * (kCropConsumerWarps + 1);  // + one producer warp
 
-// One pass of a CTA: output rows [r0, r0 + nr) x columns [c0, c0 + ncols) of one item.  Warp 0
-// walks the CTA's sequence of passes and publishes each one here for the other warps.
+// One pass of a CTA: output rows [r0, r0 + nr) x columns [c0, c0 + ncols) of one item.  The
+// producer warp walks the CTA's sequence of passes and publishes each one for the consumers.
 struct __align__(16) CropPass {
-    int32_t valid;     // 0: no more passes
-    int32_t new_item;  // first pass of its (slot, band) tile: the tap table has to be built
+    int32_t valid;  // 0: no more passes
+    int32_t table;  // which tap table the pass uses
     int32_t slot, r0, nr, c0, ncols;
-    int32_t rx0, cw;   // rectangle columns, for the tap table
-    int32_t _pad[3];
+    int32_t _pad;
 };
 
 template <int CAP>
-__global__ void __launch_bounds__(kCropThreads, kCropCtasPerSm)
+__global__ void __launch_bounds__(kCropKernelThreads, kCropCtasPerSm)
 crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __restrict__ items,
             const int* __restrict__ n_items, __half* __restrict__ out, int ow, int oh, int band_rows,
             int swap_rb, unsigned int* __restrict__ status) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t bar[2];
+    __shared__ __align__(8) uint64_t full[2], empty[2];
     __shared__ CropPass s_pass[2];
     __shared__ __align__(16) RowInfo s_row[2][kCropMaxPassRows];  // per-row data of the staged passes
 
     unsigned char* const s_rows0 = smem;
-    XEntry* const s_xtab = reinterpret_cast<XEntry*>(smem + 2 * kCropRowBudget);
+    XEntry* const s_xtab0 = reinterpret_cast<XEntry*>(smem + 2 * kCropRowBudget);  // two tables of ow entries
 
     const int packed = n_items[0];
     const int bands = (oh + band_rows - 1) / band_rows;
     const size_t plane = (size_t)ow * (size_t)oh;
-    const float inv_dx = 1.0f / (float)(2 * ow), inv_dy = 1.0f / (float)(2 * oh);
-    // every scale factor folded into the vertical weights: 1 / (255 * den_x * den_y)
-    const float inv_all = 1.0f / (255.0f * (float)(2 * ow) * (float)(2 * oh));
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-    // ---- state of the pass sequence, meaningful in warp 0 only --------------------------------
-    // tile index = slot * bands + band, advanced by gridDim.x per tile without divisions
-    const int step_slot = (int)(gridDim.x / (unsigned)bands), step_band = (int)(gridDim.x % (unsigned)bands);
-    int w_slot = (int)(blockIdx.x / (unsigned)bands), w_band = (int)(blockIdx.x % (unsigned)bands);
-    int w_frame = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
-    int w_row_lo = 0, w_row_hi = 0, w_tile_cols = ow;
-    int w_c0 = 0, w_ncols = 0, w_r0 = 0, w_nr = 0;
-    int w_seg_lo = 0, w_seg = 0, w_stride = 16, w_pass_rows = 1;
-    bool w_valid = false, w_new = false;
-
-    // geometry of the column tile starting at w_c0
-    auto set_tile = [&]() {
-        w_ncols = min(w_tile_cols, ow - w_c0);
-        const int full_lo = (3 * w_rx0) & ~15;
-        const int full_hi = (3 * (w_rx0 + w_cw) + 15) & ~15;
-        int lo = full_lo, hi = full_hi;
-        if (w_tile_cols != ow) {
-            int xa, xb, rem;
-            src_coord(w_c0, w_cw, ow, inv_dx, xa, rem);
-            src_coord(w_c0 + w_ncols - 1, w_cw, ow, inv_dx, xb, rem);
-            lo = (3 * (w_rx0 + xa)) & ~15;
-            hi = min((3 * (w_rx0 + xb) + 6 + 15) & ~15, full_hi);
-        }
-        w_seg_lo = lo;
-        w_seg = hi - lo;
-        w_stride = w_seg + 16;
-        // whole multiples of the warp count keep every warp busy (one warp per row)
-        int pr = min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows);
-        if (pr >= kCropThreads / 32) pr &= ~(kCropThreads / 32 - 1);
-        w_pass_rows = max(1, min(pr, band_rows));
-    };
-    // first pass of the tile (w_slot, w_band), if there is one
-    auto open_tile = [&]() {
-        w_valid = w_slot < packed;
-        if (!w_valid) return;
-        const octo_item_t it = items[w_slot];
-        w_frame = it.frame;
-        w_rx0 = it.rx0; w_ry0 = it.ry0; w_cw = it.rx1 - it.rx0; w_ch = it.ry1 - it.ry0;
-        const int full = ((3 * it.rx1 + 15) & ~15) - ((3 * it.rx0) & ~15);
-        w_tile_cols = (full + 16 > kCropMaxStride) ? max(2, (int)((long long)kCropTilePx * ow / w_cw) & ~1) : ow;
-        w_c0 = 0;
-        set_tile();
-        w_row_lo = w_band * band_rows;
-        w_row_hi = min(w_row_lo + band_rows, oh);
-        w_r0 = w_row_lo;
-        w_nr = min(w_pass_rows, w_row_hi - w_r0);
-        w_new = true;
-    };
-    auto advance = [&]() {
-        w_new = false;
-        if (w_r0 + w_nr < w_row_hi) {
-            w_r0 += w_nr;
-        } else if (w_c0 + w_ncols < ow) {
-            w_c0 += w_ncols;
-            set_tile();
-            w_r0 = w_row_lo;
-        } else {
-            w_slot += step_slot;
-            w_band += step_band;
-            if (w_band >= bands) { w_band -= bands; w_slot += 1; }
-            open_tile();
-            return;
-        }
-        w_nr = min(w_pass_rows, w_row_hi - w_r0);
-    };
-    // warp 0: publish the current pass in s_pass[b] and start its bulk copies into row buffer b
-    // (lane r owns output row w_r0 + r)
-    auto publish_and_stage = [&](int b) {
-        if (lane == 0) {
-            CropPass p;
-            p.valid = w_valid ? 1 : 0;
-            p.new_item = w_new ? 1 : 0;
-            p.slot = w_slot; p.r0 = w_r0; p.nr = w_nr; p.c0 = w_c0; p.ncols = w_ncols;
-            p.rx0 = w_rx0; p.cw = w_cw;
-            p._pad[0] = p._pad[1] = p._pad[2] = 0;
-            s_pass[b] = p;
-        }
-        if (!w_valid) return;
-        const FrameDesc& fd = tab.f[w_frame];
-        int y0 = 0, ry = 0;
-        uint32_t bytes = 0;
-        if (lane < w_nr) {
-            src_coord(w_r0 + lane, w_ch, oh, inv_dy, y0, ry);
-            bytes = (uint32_t)w_seg * (ry != 0 ? 2u : 1u);
-            RowInfo ri;
-            ri.row0 = 2 * lane * w_stride - w_seg_lo;  // table offsets are relative to the frame row
-            ri.row1 = ri.row0 + w_stride;
-            ri.wx = (float)(2 * oh - ry) * inv_all;
-            ri.wy = (float)ry * inv_all;
-            s_row[b][lane] = ri;
-        }
-        const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
-        fence_proxy_async();
-        if (lane == 0) mbar_expect_tx(&bar[b], total);
-        __syncwarp();
-        if (lane < w_nr) {
-            unsigned char* dst = s_rows0 + (size_t)b * kCropRowBudget + (size_t)(2 * lane) * w_stride;
-            const uint8_t* src = fd.data + (size_t)(w_ry0 + y0) * (size_t)fd.pitch + w_seg_lo;
-            bulk_g2s(dst, src, (uint32_t)w_seg, &bar[b]);
-            if (ry != 0) bulk_g2s(dst + w_stride, src + fd.pitch, (uint32_t)w_seg, &bar[b]);
-        }
-    };
-
     if (threadIdx.x == 0) {
-        mbar_init(&bar[0], 1);
-        mbar_init(&bar[1], 1);
+        mbar_init(&full[0], 1);
+        mbar_init(&full[1], 1);
+        mbar_init(&empty[0], kCropConsumerWarps);
+        mbar_init(&empty[1], kCropConsumerWarps);
         mbar_fence_init();
     }
     __syncthreads();
-    if (warp == 0) {
+
+    if (warp == kCropConsumerWarps) {
+        // =============================== producer warp ===================================
+        const float inv_dx = 1.0f / (float)(2 * ow), inv_dy = 1.0f / (float)(2 * oh);
+        // every scale factor folded into the vertical weights: 1 / (255 * den_x * den_y)
+        const float inv_all = 1.0f / (255.0f * (float)(2 * ow) * (float)(2 * oh));
+        // tile index = slot * bands + band, advanced by gridDim.x per tile without divisions
+        const int step_slot = (int)(gridDim.x / (unsigned)bands), step_band = (int)(gridDim.x % (unsigned)bands);
+        int w_slot = (int)(blockIdx.x / (unsigned)bands), w_band = (int)(blockIdx.x % (unsigned)bands);
+        int w_frame = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
+        int w_row_lo = 0, w_row_hi = 0, w_tile_cols = ow;
+        int w_c0 = 0, w_ncols = 0, w_r0 = 0, w_nr = 0;
+        int w_seg_lo = 0, w_seg = 0, w_stride = 16, w_pass_rows = 1;
+        bool w_valid = false, w_new = false;
+
+        // geometry of the column tile starting at w_c0
+        auto set_tile = [&]() {
+            w_ncols = min(w_tile_cols, ow - w_c0);
+            const int full_lo = (3 * w_rx0) & ~15;
+            const int full_hi = (3 * (w_rx0 + w_cw) + 15) & ~15;
+            int lo = full_lo, hi = full_hi;
+            if (w_tile_cols != ow) {
+                int xa, xb, rem;
+                src_coord(w_c0, w_cw, ow, inv_dx, xa, rem);
+                src_coord(w_c0 + w_ncols - 1, w_cw, ow, inv_dx, xb, rem);
+                lo = (3 * (w_rx0 + xa)) & ~15;
+                hi = min((3 * (w_rx0 + xb) + 6 + 15) & ~15, full_hi);
+            }
+            w_seg_lo = lo;
+            w_seg = hi - lo;
+            w_stride = w_seg + 16;
+            // whole multiples of the consumer warp count keep every warp busy (one warp per row)
+            int pr = min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows);
+            if (pr >= kCropConsumerWarps) pr &= ~(kCropConsumerWarps - 1);
+            w_pass_rows = max(1, min(pr, band_rows));
+        };
+        // first pass of the tile (w_slot, w_band), if there is one
+        auto open_tile = [&]() {
+            w_valid = w_slot < packed;
+            if (!w_valid) return;
+            const octo_item_t it = items[w_slot];
+            w_frame = it.frame;
+            w_rx0 = it.rx0; w_ry0 = it.ry0; w_cw = it.rx1 - it.rx0; w_ch = it.ry1 - it.ry0;
+            const int full_seg = ((3 * it.rx1 + 15) & ~15) - ((3 * it.rx0) & ~15);
+            w_tile_cols =
+                (full_seg + 16 > kCropMaxStride) ? max(2, (int)((long long)kCropTilePx * ow / w_cw) & ~1) : ow;
+            w_c0 = 0;
+            set_tile();
+            w_row_lo = w_band * band_rows;
+            w_row_hi = min(w_row_lo + band_rows, oh);
+            w_r0 = w_row_lo;
+            w_nr = min(w_pass_rows, w_row_hi - w_r0);
+            w_new = true;
+        };
+        auto advance = [&]() {
+            w_new = false;
+            if (w_r0 + w_nr < w_row_hi) {
+                w_r0 += w_nr;
+            } else if (w_c0 + w_ncols < ow) {
+                w_c0 += w_ncols;
+                set_tile();
+                w_r0 = w_row_lo;
+            } else {
+                w_slot += step_slot;
+                w_band += step_band;
+                if (w_band >= bands) { w_band -= bands; w_slot += 1; }
+                open_tile();
+                return;
+            }
+            w_nr = min(w_pass_rows, w_row_hi - w_r0);
+        };
+
         open_tile();
-        publish_and_stage(0);
-    }
-    __syncthreads();
-
-    uint32_t phase[2] = {0u, 0u};
-    bool failed = false;
-    int buf = 0;
-    __half* const out0 = out + (swap_rb ? 2 : 0) * plane;  // plane of input channel 0
-    __half* const out1 = out + plane;
-    __half* const out2 = out + (swap_rb ? 0 : 2) * plane;  // plane of input channel 2
-
-    for (;;) {
-        const CropPass cur = s_pass[buf];
-        if (!cur.valid) break;
-        if (cur.new_item) {
-            // taps of every output column: byte offset inside a frame row + integer weights.  The
-            // previous tile's table was last read before the barrier that ended the previous pass.
-            for (int dx = threadIdx.x; dx < ow; dx += kCropThreads)
-                s_xtab[dx] = make_xentry(dx, cur.cw, ow, inv_dx, 3 * cur.rx0);
-        }
-        if (warp == 0) {
+        uint32_t ephase[2] = {0u, 0u};
+        int tb = 1;
+        for (int k = 0;; ++k) {
+            const int b = k & 1;
+            if (k >= 2) {
+                // the consumers have finished the pass that used ring slot b
+                if (!mbar_wait_bounded(&empty[b], ephase[b]) && !mbar_wait_bounded(&empty[b], ephase[b])) {
+                    if (lane == 0) atomicOr(status, 0x4u);
+                    break;
+                }
+                ephase[b] ^= 1u;
+            }
+            if (w_valid && w_new) {
+                // taps of every output column: byte offset inside a frame row + integer weights.
+                // The other table is still in use by at most the previous pass; this one was last
+                // used two tiles ago, i.e. by passes the wait above has seen finished.
+                tb ^= 1;
+                XEntry* const xt = s_xtab0 + (size_t)tb * ow;
+                for (int dx = lane; dx < ow; dx += 32) xt[dx] = make_xentry(dx, w_cw, ow, inv_dx, 3 * w_rx0);
+            }
+            if (lane == 0) {
+                CropPass p;
+                p.valid = w_valid ? 1 : 0;
+                p.table = tb;
+                p.slot = w_slot; p.r0 = w_r0; p.nr = w_nr; p.c0 = w_c0; p.ncols = w_ncols;
+                p._pad = 0;
+                s_pass[b] = p;
+            }
+            if (!w_valid) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full[b]);  // the end-of-work record
+                break;
+            }
+            // lane r owns output row w_r0 + r of the pass
+            const FrameDesc& fd = tab.f[w_frame];
+            int y0 = 0, ry = 0;
+            uint32_t bytes = 0;
+            if (lane < w_nr) {
+                src_coord(w_r0 + lane, w_ch, oh, inv_dy, y0, ry);
+                bytes = (uint32_t)w_seg * (ry != 0 ? 2u : 1u);
+                RowInfo ri;
+                ri.row0 = 2 * lane * w_stride - w_seg_lo;  // table offsets are relative to the frame row
+                ri.row1 = ri.row0 + w_stride;
+                ri.wx = (float)(2 * oh - ry) * inv_all;
+                ri.wy = (float)ry * inv_all;
+                s_row[b][lane] = ri;
+            }
+            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+            fence_proxy_async();
+            __syncwarp();  // table, pass record and row data are written before the barrier is armed
+            if (lane == 0) mbar_expect_tx(&full[b], total);
+            __syncwarp();
+            if (lane < w_nr) {
+                unsigned char* dst = s_rows0 + (size_t)b * kCropRowBudget + (size_t)(2 * lane) * w_stride;
+                const uint8_t* src = fd.data + (size_t)(w_ry0 + y0) * (size_t)fd.pitch + w_seg_lo;
+                bulk_g2s(dst, src, (uint32_t)w_seg, &full[b]);
+                if (ry != 0) bulk_g2s(dst + w_stride, src + fd.pitch, (uint32_t)w_seg, &full[b]);
+            }
             advance();
-            publish_and_stage(buf ^ 1);  // in flight while cur is computed
         }
-        __syncthreads();  // table, next pass record, row data and armed barriers are visible
-
-        if (!failed && !mbar_wait_bounded(&bar[buf], phase[buf])) {
-            if (!mbar_wait_bounded(&bar[buf], phase[buf])) failed = true;
-        }
-        phase[buf] ^= 1u;
-
-        if (!failed) {
+    } else {
+        // =============================== consumer warps ==================================
+        __half* const out0 = out + (swap_rb ? 2 : 0) * plane;  // plane of input channel 0
+        __half* const out1 = out + plane;
+        __half* const out2 = out + (swap_rb ? 0 : 2) * plane;  // plane of input channel 2
+        uint32_t fphase[2] = {0u, 0u};
+        for (int k = 0;; ++k) {
+            const int b = k & 1;
+            if (!mbar_wait_bounded(&full[b], fphase[b]) && !mbar_wait_bounded(&full[b], fphase[b])) {
+                if (lane == 0) atomicOr(status, 0x4u);
+                break;
+            }
+            fphase[b] ^= 1u;
+            const CropPass cur = s_pass[b];
+            if (!cur.valid) break;
             // one warp per output row of the pass
-            const XEntry* const xt = s_xtab + cur.c0;
-            const unsigned char* const rows = s_rows0 + (size_t)buf * kCropRowBudget;
+            const XEntry* const xt = s_xtab0 + (size_t)cur.table * ow + cur.c0;
+            const unsigned char* const rows = s_rows0 + (size_t)b * kCropRowBudget;
             const size_t tile_off = (size_t)cur.slot * 3 * plane + (size_t)cur.r0 * ow + cur.c0;
             const int pairs = cur.ncols >> 1;
-            for (int r = warp; r < cur.nr; r += kCropThreads / 32) {
-                const RowInfo ri = s_row[buf][r];
+            for (int r = warp; r < cur.nr; r += kCropConsumerWarps) {
+                const RowInfo ri = s_row[b][r];
                 const size_t o = tile_off + (size_t)(r * ow);
                 if (ri.wy != 0.0f)
                     sample_row<true, false>(rows + ri.row0, rows + ri.row1, ri.wx, ri.wy, xt, pairs, lane, out0 + o,
@@ -295,11 +305,10 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
                     sample_row<false, false>(rows + ri.row0, rows + ri.row1, ri.wx, ri.wy, xt, pairs, lane, out0 + o,
                                              out1 + o, out2 + o, 0.0f);
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[b]);  // this warp is done with ring slot b
         }
-        __syncthreads();  // cur's rows, row data and pass record may now be overwritten
-        buf ^= 1;
     }
-    if (failed && threadIdx.x == 0) atomicOr(status, 0x4u);
 }
 
 template <int CAP>
@@ -324,15 +333,15 @@ static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     long long work = (long long)a.max_items * bands;
     long long cap = (long long)a.sm_count * kCropCtasPerSm;
     const int grid = (int)(work < cap ? work : cap);
-    const size_t smem = 2 * (size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w;
-    crop_kernel<CAP><<<grid, kCropThreads, smem, stream>>>(tab, a.d_items, a.d_n_items,
+    const size_t smem = 2 * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w);
+    crop_kernel<CAP><<<grid, kCropKernelThreads, smem, stream>>>(tab, a.d_items, a.d_n_items,
                                                           reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h,
                                                           band_rows, a.swap_rb, &a.d_ctr->status);
     return cudaGetLastError();
 }
 
 cudaError_t prepare_crop() {
-    const int smem = 2 * kCropRowBudget + (int)sizeof(XEntry) * 2048;
+    const int smem = 2 * (kCropRowBudget + (int)sizeof(XEntry) * 2048);
     cudaError_t e;
     e = cudaFuncSetAttribute(crop_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
