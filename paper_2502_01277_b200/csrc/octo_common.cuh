@@ -113,13 +113,27 @@ __device__ __forceinline__ XEntry make_xentry(int d, int src, int dst, float inv
     return e;
 }
 
-// Integer horizontal lerp of the three channels of one destination pixel.  `row` is the byte
-// address of a staged row (4-byte aligned, shared memory, at least 12 readable bytes past
-// any offset); `woff` = e.off & ~3 and `sh` = 8 * (e.off & 3) are shared by both rows.
-__device__ __forceinline__ void hsample(const unsigned char* __restrict__ row, uint32_t woff, uint32_t sh,
-                                        uint32_t wts, uint32_t& c0, uint32_t& c1, uint32_t& c2) {
-    const uint32_t* p = reinterpret_cast<const uint32_t*>(row + woff);
-    const uint32_t a = p[0], b = p[1], c = p[2];
+// Shared-memory loads through 32-bit shared-space addresses (no 64-bit generic pointer
+// arithmetic in the inner loops).
+__device__ __forceinline__ void lds32x3(uint32_t addr, uint32_t& a, uint32_t& b, uint32_t& c) {
+    asm volatile("ld.shared.u32 %0, [%3];\n\tld.shared.u32 %1, [%3+4];\n\tld.shared.u32 %2, [%3+8];"
+                 : "=r"(a), "=r"(b), "=r"(c)
+                 : "r"(addr));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// Integer horizontal lerp of the three channels of one destination pixel.  `addr` is the
+// shared-space address of the 4-byte aligned word that holds the left tap's first byte (the
+// staged rows keep at least 12 readable bytes past any tap); only the low five bits of `sh`
+// = 8 * byte offset matter (the funnel shift wraps).
+__device__ __forceinline__ void hsample(uint32_t addr, uint32_t sh, uint32_t wts, uint32_t& c0, uint32_t& c1,
+                                        uint32_t& c2) {
+    uint32_t a, b, c;
+    lds32x3(addr, a, b, c);
     const uint32_t lo = __funnelshift_r(a, b, sh);  // B0 G0 R0 B1
     const uint32_t hi = __funnelshift_r(b, c, sh);  // G1 R1 .. ..
     const uint32_t p01 = __byte_perm(lo, hi, 0x4130);  // B0 B1 G0 G1
@@ -129,21 +143,21 @@ __device__ __forceinline__ void hsample(const unsigned char* __restrict__ row, u
     c2 = __dp2a_lo(wts, p2, 0u);
 }
 
-// One destination pixel: horizontal integer lerp on one or two staged rows, then the
-// vertical lerp and all scaling in fp32 (wx / wy carry 1 / (255 * den_x * den_y)).
+// One destination pixel: horizontal integer lerp on one or two staged rows (shared-space
+// addresses row0, row0 + row_step), then the vertical lerp and all scaling in fp32 (wx / wy
+// carry 1 / (255 * den_x * den_y)).
 template <bool LERP_Y>
-__device__ __forceinline__ void sample_px(const unsigned char* __restrict__ row0,
-                                          const unsigned char* __restrict__ row1, const XEntry e, float wx,
-                                          float wy, float& f0, float& f1, float& f2) {
-    const uint32_t woff = e.off & ~3u, sh = (e.off & 3u) << 3;
+__device__ __forceinline__ void sample_px(uint32_t row0, uint32_t row_step, const uint32_t off, const uint32_t wts,
+                                          float wx, float wy, float& f0, float& f1, float& f2) {
+    const uint32_t addr = row0 + (off & ~3u), sh = off << 3;
     uint32_t a0, a1, a2;
-    hsample(row0, woff, sh, e.wts, a0, a1, a2);
+    hsample(addr, sh, wts, a0, a1, a2);
     f0 = __uint2float_rn(a0) * wx;
     f1 = __uint2float_rn(a1) * wx;
     f2 = __uint2float_rn(a2) * wx;
     if (LERP_Y) {
         uint32_t b0, b1, b2;
-        hsample(row1, woff, sh, e.wts, b0, b1, b2);
+        hsample(addr + row_step, sh, wts, b0, b1, b2);
         f0 = fmaf(__uint2float_rn(b0), wy, f0);
         f1 = fmaf(__uint2float_rn(b1), wy, f1);
         f2 = fmaf(__uint2float_rn(b2), wy, f2);
@@ -157,35 +171,34 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
 
 // One output row (or column tile of it) by one warp: lane l owns the pixel pairs l, l + 32, ...
 // so neighbouring lanes read neighbouring table entries and row words (no bank conflicts)
-// and the warp writes 128 contiguous bytes per plane and step.  o0 / o1 / o2 point at the
-// row's first pixel in the planes of input channels 0 / 1 / 2.  With FILL, columns whose
-// table entry has zero weights (canvas outside the image) receive fill_f.
+// and the warp writes 128 contiguous bytes per plane and step.  row0 / xt are shared-space
+// addresses of the first staged row and of the tile's first table entry; o0 / o1 / o2 point
+// at the row's first pixel in the planes of input channels 0 / 1 / 2.  With FILL, columns
+// whose table entry has zero weights (canvas outside the image) receive fill_f.
 template <bool LERP_Y, bool FILL>
-__device__ __forceinline__ void sample_row(const unsigned char* __restrict__ row0,
-                                           const unsigned char* __restrict__ row1, float wx, float wy,
-                                           const XEntry* __restrict__ xt, int pairs, int lane,
-                                           __half* __restrict__ o0, __half* __restrict__ o1,
+__device__ __forceinline__ void sample_row(uint32_t row0, uint32_t row_step, float wx, float wy, uint32_t xt,
+                                           int pairs, int lane, __half* __restrict__ o0, __half* __restrict__ o1,
                                            __half* __restrict__ o2, float fill_f) {
     for (int pair = lane; pair < pairs; pair += 32) {
-        const uint4 ee = *reinterpret_cast<const uint4*>(xt + 2 * pair);
-        const XEntry e0 = {ee.x, ee.y}, e1 = {ee.z, ee.w};
+        const uint4 ee = lds128(xt + 16u * (uint32_t)pair);  // two XEntry: {off, wts} x 2
         float a0, a1, a2, b0, b1, b2;
-        sample_px<LERP_Y>(row0, row1, e0, wx, wy, a0, a1, a2);
-        sample_px<LERP_Y>(row0, row1, e1, wx, wy, b0, b1, b2);
+        sample_px<LERP_Y>(row0, row_step, ee.x, ee.y, wx, wy, a0, a1, a2);
+        sample_px<LERP_Y>(row0, row_step, ee.z, ee.w, wx, wy, b0, b1, b2);
         if (FILL) {
-            if (e0.wts == 0u) { a0 = fill_f; a1 = fill_f; a2 = fill_f; }
-            if (e1.wts == 0u) { b0 = fill_f; b1 = fill_f; b2 = fill_f; }
+            if (ee.y == 0u) { a0 = fill_f; a1 = fill_f; a2 = fill_f; }
+            if (ee.w == 0u) { b0 = fill_f; b1 = fill_f; b2 = fill_f; }
         }
-        *reinterpret_cast<uint32_t*>(o0 + 2 * pair) = pack_half2(a0, b0);
-        *reinterpret_cast<uint32_t*>(o1 + 2 * pair) = pack_half2(a1, b1);
-        *reinterpret_cast<uint32_t*>(o2 + 2 * pair) = pack_half2(a2, b2);
+        const uint32_t o = 2u * (uint32_t)pair;
+        *reinterpret_cast<uint32_t*>(o0 + o) = pack_half2(a0, b0);
+        *reinterpret_cast<uint32_t*>(o1 + o) = pack_half2(a1, b1);
+        *reinterpret_cast<uint32_t*>(o2 + o) = pack_half2(a2, b2);
     }
 }
 
 // What a warp needs to know about one output row of a staged pass.
 struct RowInfo {
-    int32_t row0;  // byte offset of the first staged row inside the row buffer; < 0: canvas row
-    int32_t row1;  // byte offset of the second staged row (unused when wy == 0)
+    int32_t row0;  // byte offset of the first staged row relative to the row buffer
+    int32_t step;  // distance to the second staged row (unused when wy == 0); < 0: canvas row
     float wx, wy;  // vertical weights with all scaling folded in
 };
 

@@ -257,7 +257,7 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
                 bytes = (uint32_t)w_seg * (ry != 0 ? 2u : 1u);
                 RowInfo ri;
                 ri.row0 = 2 * lane * w_stride - w_seg_lo;  // table offsets are relative to the frame row
-                ri.row1 = ri.row0 + w_stride;
+                ri.step = w_stride;
                 ri.wx = (float)(2 * oh - ry) * inv_all;
                 ri.wy = (float)ry * inv_all;
                 s_row[b][lane] = ri;
@@ -291,19 +291,19 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
             const CropPass cur = s_pass[b];
             if (!cur.valid) break;
             // one warp per output row of the pass
-            const XEntry* const xt = s_xtab0 + (size_t)cur.table * ow + cur.c0;
-            const unsigned char* const rows = s_rows0 + (size_t)b * kCropRowBudget;
+            const uint32_t xt = smem_u32(s_xtab0) + (uint32_t)(cur.table * ow + cur.c0) * (uint32_t)sizeof(XEntry);
+            const uint32_t rows = smem_u32(s_rows0) + (uint32_t)b * kCropRowBudget;
             const size_t tile_off = (size_t)cur.slot * 3 * plane + (size_t)cur.r0 * ow + cur.c0;
             const int pairs = cur.ncols >> 1;
             for (int r = warp; r < cur.nr; r += kCropConsumerWarps) {
                 const RowInfo ri = s_row[b][r];
                 const size_t o = tile_off + (size_t)(r * ow);
                 if (ri.wy != 0.0f)
-                    sample_row<true, false>(rows + ri.row0, rows + ri.row1, ri.wx, ri.wy, xt, pairs, lane, out0 + o,
-                                            out1 + o, out2 + o, 0.0f);
+                    sample_row<true, false>(rows + (uint32_t)ri.row0, (uint32_t)ri.step, ri.wx, ri.wy, xt, pairs, lane,
+                                            out0 + o, out1 + o, out2 + o, 0.0f);
                 else
-                    sample_row<false, false>(rows + ri.row0, rows + ri.row1, ri.wx, ri.wy, xt, pairs, lane, out0 + o,
-                                             out1 + o, out2 + o, 0.0f);
+                    sample_row<false, false>(rows + (uint32_t)ri.row0, (uint32_t)ri.step, ri.wx, ri.wy, xt, pairs, lane,
+                                             out0 + o, out1 + o, out2 + o, 0.0f);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[b]);  // this warp is done with ring slot b

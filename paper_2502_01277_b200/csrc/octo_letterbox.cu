@@ -23,7 +23,7 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
                  int slot_bytes, uint32_t fill_h2, float fill_f, int swap_rb, unsigned int* __restrict__ status) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t bar;
-    __shared__ __align__(16) RowInfo s_row[kLbRows];  // per-row data; row0 < 0 marks a canvas (pad) row
+    __shared__ __align__(16) RowInfo s_row[kLbRows];  // per-row data; step < 0 marks a canvas (pad) row
 
     const FrameDesc& fd = tab.f[blockIdx.y];
     const int dy0 = blockIdx.x * band_rows;
@@ -63,12 +63,12 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
         for (int r = 0; r < nrows; ++r) {
             const int iy = dy0 + r - pad_t;
             RowInfo ri;
-            ri.row0 = -1; ri.row1 = 0; ri.wx = 0.0f; ri.wy = 0.0f;
+            ri.row0 = 0; ri.step = -1; ri.wx = 0.0f; ri.wy = 0.0f;
             if (iy < 0 || iy >= nh) { s_row[r] = ri; continue; }
             int y0, ry;
             src_coord(iy, h, nh, inv_dy, y0, ry);
             ri.row0 = slot * slot_bytes;
-            ri.row1 = ri.row0 + slot_bytes;
+            ri.step = slot_bytes;
             ri.wx = (float)(2 * nh - ry) * inv_all;
             ri.wy = (float)ry * inv_all;
             s_row[r] = ri;
@@ -107,24 +107,25 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
     // one warp per output row of the band
     const int pairs = S >> 1;
     const int lane = threadIdx.x & 31;
+    const uint32_t rows_s = smem_u32(s_rows), xtab_s = smem_u32(s_xtab);
     __half* const out0 = out_img + (swap_rb ? 2 : 0) * plane;  // plane of input channel 0
     __half* const out1 = out_img + plane;
     __half* const out2 = out_img + (swap_rb ? 0 : 2) * plane;  // plane of input channel 2
     for (int r = threadIdx.x >> 5; r < nrows; r += kLbThreads / 32) {
         const RowInfo ri = s_row[r];
         const size_t o = (size_t)(dy0 + r) * S;
-        if (ri.row0 < 0 || !copy_ok) {
+        if (ri.step < 0 || !copy_ok) {
             for (int pair = lane; pair < pairs; pair += 32) {
                 *reinterpret_cast<uint32_t*>(out0 + o + 2 * pair) = fill_h2;
                 *reinterpret_cast<uint32_t*>(out1 + o + 2 * pair) = fill_h2;
                 *reinterpret_cast<uint32_t*>(out2 + o + 2 * pair) = fill_h2;
             }
         } else if (ri.wy != 0.0f) {
-            sample_row<true, true>(s_rows + ri.row0, s_rows + ri.row1, ri.wx, ri.wy, s_xtab, pairs, lane, out0 + o,
-                                   out1 + o, out2 + o, fill_f);
+            sample_row<true, true>(rows_s + (uint32_t)ri.row0, (uint32_t)ri.step, ri.wx, ri.wy, xtab_s, pairs, lane,
+                                   out0 + o, out1 + o, out2 + o, fill_f);
         } else {
-            sample_row<false, true>(s_rows + ri.row0, s_rows + ri.row1, ri.wx, ri.wy, s_xtab, pairs, lane, out0 + o,
-                                    out1 + o, out2 + o, fill_f);
+            sample_row<false, true>(rows_s + (uint32_t)ri.row0, (uint32_t)ri.step, ri.wx, ri.wy, xtab_s, pairs, lane,
+                                    out0 + o, out1 + o, out2 + o, fill_f);
         }
     }
 }
