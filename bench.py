@@ -39,7 +39,14 @@ UNIT = "frames/s"
 # source the capture was taken from.  An entry whose hash no longer matches the source is
 # reported as null.
 NCU_TRAFFIC = {
-    # kernel: (source file, sha256[:16] of that file at capture time, bytes per unit, unit)
+    # kernel: (source files, sha256[:16] of their concatenation at capture time, bytes per unit, unit)
+    # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md)
+    "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
+             "8f85268299fbeb73", 498201.0, "crop"),
+    "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
+                  "e18d17f81bd349de", 3705548.0, "frame"),
+    "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
+               "14bf76fbde1bde9e", 3295584.0, "frame"),
 }
 
 
@@ -97,16 +104,19 @@ def decode_bytes(n: int, a: int, c: int, candidates: int, logits: bool) -> int:
     return int(scan + candidates * (row + 8))
 
 
-def file_hash(path: str) -> str:
-    return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
+def files_hash(paths) -> str:
+    h = hashlib.sha256()
+    for p in paths:
+        h.update(open(os.path.join(ROOT, p), "rb").read())
+    return h.hexdigest()[:16]
 
 
 def traffic_for(kernel: str, units: float):
     ent = NCU_TRAFFIC.get(kernel)
     if not ent:
         return None
-    src, digest, per_unit, _unit = ent
-    if file_hash(os.path.join(ROOT, src)) != digest:
+    srcs, digest, per_unit, _unit = ent
+    if files_hash(srcs) != digest:
         return None
     return per_unit * units
 
