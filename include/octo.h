@@ -214,7 +214,8 @@ OCTO_API int octo_stage_item_table(octo_stage_t* st, int32_t branch, const octo_
 OCTO_API int octo_stage_copy_items(octo_stage_t* st, int32_t branch, octo_item_t* items_out, int32_t count,
                                    void* cuda_stream);
 
-/* Kernel order used by octo_kernel_times_t. */
+/* Kernel order used by octo_kernel_times_t.  OCTO_K_ASSEMBLE stays zero: the batch assembler
+ * runs inside the crop kernel. */
 enum { OCTO_K_LETTERBOX = 0, OCTO_K_DECODE = 1, OCTO_K_NMS = 2, OCTO_K_ASSEMBLE = 3, OCTO_K_CROP = 4,
        OCTO_K_COUNT = 5 };
 

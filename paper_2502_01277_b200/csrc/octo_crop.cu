@@ -1,99 +1,27 @@
-// Batch assembler and ROI crop-resize for one downstream branch.
+// Batch assembler and ROI crop-resize for one downstream branch, in one kernel.
 //
-// assemble_kernel (one CTA): exclusive prefix sum of the per-frame class-filtered detection
-// counts -> offsets[n+1]; then the item table of the requested window (frame, detection,
-// integer crop rectangle).  Integer work only.
+// Assembler (integer work only).  Every CTA scans the per-frame class-filtered detection
+// counts of the branch (at most 512 integers) into shared memory: offsets[n+1], total and
+// the number of items packed into the caller's window.  CTA 0 writes offsets / n_items.  An
+// item is resolved where it is needed: slot -> frame by binary search in the offsets, ->
+// detection through the branch's index list, -> outward-rounded integer rectangle.  The item
+// table entry of a slot is written by the CTA that processes the slot's first row band.
 //
-// crop_kernel: HBM-bound (the fp16 output is as large as the source rectangles).  A
-// persistent grid strides over (slot, row band) tiles; the number of packed items is read
-// from device memory, so no host synchronisation sits between NMS and cropping.  Per tile the
-// CTA builds a table of horizontal taps (byte offset + exact integer weights per column),
-// one thread has the bulk-copy engine stage the 16-byte aligned segments of the source rows
-// the band taps into shared memory (mbarrier, bounded wait), and every thread then produces
-// pixel pairs (lane l of a warp takes pixels 2l, 2l+1 of a 64-pixel run, so table and row
-// reads of neighbouring lanes fall into neighbouring banks): the horizontal lerp is an exact
-// integer two-way dot product per channel, the vertical lerp and all scaling are two fp32
-// operations, and each warp writes 128 contiguous bytes per plane straight into the
-// downstream slot.
+// Crop-resize: bound by instruction issue, then HBM (the fp16 output is as large as the
+// source rectangles).  A persistent grid strides over (slot, row band) tiles, so no host
+// synchronisation sits between NMS and cropping.  Inside a CTA one producer warp walks the
+// tiles: it resolves the item, builds the table of horizontal taps (byte offset + exact
+// integer weights per output column) and has the bulk-copy engine stage the 16-byte aligned
+// segments of the source rows a pass taps into one of two shared-memory buffers (mbarrier
+// "full" / "empty" ring, every wait bounded).  Eight consumer warps take one output row
+// each: lane l owns pixel pairs l, l+32, ... so neighbouring lanes read neighbouring table
+// entries and row words; the horizontal lerp is an exact integer two-way dot product per
+// channel, the vertical lerp and all scaling are two fp32 operations, and a warp writes 128
+// contiguous bytes per plane straight into the downstream slot.
 #include "octo_common.cuh"
 #include "octo_kernels.h"
 
 namespace octo {
-
-constexpr int kAsmThreads = 1024;
-
-template <int CAP>
-__global__ void __launch_bounds__(kAsmThreads)
-assemble_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int first_item, int max_items,
-                const int* __restrict__ bcount, const int* __restrict__ bidx,
-                const octo_det_t* __restrict__ dets, int* __restrict__ offsets, int* __restrict__ n_items,
-                octo_item_t* __restrict__ items, StageCounters* __restrict__ ctr) {
-    __shared__ int s_off[CAP + 1];
-    __shared__ int s_warp[kAsmThreads / 32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-
-    // exclusive scan of up to CAP (<= 1024) counts: one element per thread
-    static_assert(CAP <= kAsmThreads, "one count per thread");
-    {
-        const int v = threadIdx.x < n ? bcount[threadIdx.x] : 0;
-        int inc = v;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, inc, off);
-            if (lane >= off) inc += t;
-        }
-        if (lane == 31) s_warp[warp] = inc;
-        __syncthreads();
-        if (warp == 0) {
-            int w = s_warp[lane];
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, w, off);
-                if (lane >= off) w += t;
-            }
-            s_warp[lane] = w;  // inclusive over warps
-        }
-        __syncthreads();
-        const int base = warp > 0 ? s_warp[warp - 1] : 0;
-        if (threadIdx.x < n) s_off[threadIdx.x] = base + inc - v;
-        if (threadIdx.x == n - 1) s_off[n] = base + inc;
-    }
-    __syncthreads();
-    const int total = s_off[n];
-    for (int i = threadIdx.x; i <= n; i += kAsmThreads) offsets[i] = s_off[i];
-    if (threadIdx.x == 0) {
-        long long rest = (long long)total - (long long)first_item;
-        int packed = rest < 0 ? 0 : (rest > max_items ? max_items : (int)rest);
-        n_items[0] = packed;
-        n_items[1] = total;
-        ctr->packed = packed;
-        ctr->total_items = total;
-        if ((long long)total > (long long)first_item + (long long)max_items) atomicOr(&ctr->status, 0x2u);
-    }
-    // item table of the window; one warp per frame
-    for (int f = warp; f < n; f += kAsmThreads / 32) {
-        const int o = s_off[f], m = s_off[f + 1] - o;
-        const FrameDesc& fd = tab.f[f];
-        for (int j = lane; j < m; j += 32) {
-            const long long slot = (long long)o + j - first_item;
-            if (slot < 0 || slot >= max_items) continue;
-            const int det = bidx[(size_t)f * max_det + j];
-            const octo_det_t d = dets[(size_t)f * max_det + det];
-            // outward-rounded rectangle, clamped so that it is never empty
-            int rx0 = (int)floorf(d.x1), ry0 = (int)floorf(d.y1);
-            int rx1 = (int)ceilf(d.x2), ry1 = (int)ceilf(d.y2);
-            rx0 = min(max(rx0, 0), fd.w - 1);
-            ry0 = min(max(ry0, 0), fd.h - 1);
-            rx1 = min(max(rx1, rx0 + 1), fd.w);
-            ry1 = min(max(ry1, ry0 + 1), fd.h);
-            octo_item_t it;
-            it.frame = f; it.det = det;
-            it.rx0 = rx0; it.ry0 = ry0; it.rx1 = rx1; it.ry1 = ry1;
-            it._pad[0] = 0; it._pad[1] = 0;
-            items[slot] = it;
-        }
-    }
-}
 
 // Shared memory for staged source rows.  A pass stages two row segments per output row; a
 // segment longer than kCropMaxStride - 16 bytes (a rectangle wider than about 4000 pixels)
@@ -118,22 +46,39 @@ struct __align__(16) CropPass {
 
 template <int CAP>
 __global__ void __launch_bounds__(kCropKernelThreads, kCropCtasPerSm)
-crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __restrict__ items,
-            const int* __restrict__ n_items, __half* __restrict__ out, int ow, int oh, int band_rows,
-            int swap_rb, unsigned int* __restrict__ status) {
+crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int first_item, int max_items,
+            const int* __restrict__ bcount, const int* __restrict__ bidx, const octo_det_t* __restrict__ dets,
+            int* __restrict__ offsets, int* __restrict__ n_items, octo_item_t* __restrict__ items,
+            __half* __restrict__ out, int ow, int oh, int band_rows, int swap_rb, StageCounters* __restrict__ ctr) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t full[2], empty[2];
     __shared__ CropPass s_pass[2];
     __shared__ __align__(16) RowInfo s_row[2][kCropMaxPassRows];  // per-row data of the staged passes
+    __shared__ int s_off[CAP + 1];                                // exclusive scan of the frame counts
 
     unsigned char* const s_rows0 = smem;
     XEntry* const s_xtab0 = reinterpret_cast<XEntry*>(smem + 2 * kCropRowBudget);  // two tables of ow entries
+    unsigned int* const status = &ctr->status;
 
-    const int packed = n_items[0];
-    const int bands = (oh + band_rows - 1) / band_rows;
-    const size_t plane = (size_t)ow * (size_t)oh;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
+    // ---- assembler: offsets of the branch's items per frame ------------------------------------
+    if (warp == 0) {
+        int run = 0;
+        for (int base = 0; base < n; base += 32) {
+            const int i = base + lane;
+            const int v = i < n ? bcount[i] : 0;
+            int inc = v;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, inc, off);
+                if (lane >= off) inc += t;
+            }
+            if (i < n) s_off[i] = run + inc - v;
+            run += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (lane == 0) s_off[n] = run;
+    }
     if (threadIdx.x == 0) {
         mbar_init(&full[0], 1);
         mbar_init(&full[1], 1);
@@ -142,15 +87,34 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
         mbar_fence_init();
     }
     __syncthreads();
+    const int total = s_off[n];
+    const long long rest = (long long)total - (long long)first_item;
+    const int packed = rest < 0 ? 0 : (rest > max_items ? max_items : (int)rest);
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i <= n; i += kCropKernelThreads) offsets[i] = s_off[i];
+        if (threadIdx.x == 0) {
+            n_items[0] = packed;
+            n_items[1] = total;
+            ctr->packed = packed;
+            ctr->total_items = total;
+            if ((long long)total > (long long)first_item + (long long)max_items) atomicOr(status, 0x2u);
+        }
+    }
+
+    const int bands = (oh + band_rows - 1) / band_rows;
+    const size_t plane = (size_t)ow * (size_t)oh;
 
     if (warp == kCropConsumerWarps) {
         // =============================== producer warp ===================================
         const float inv_dx = 1.0f / (float)(2 * ow), inv_dy = 1.0f / (float)(2 * oh);
         // every scale factor folded into the vertical weights: 1 / (255 * den_x * den_y)
         const float inv_all = 1.0f / (255.0f * (float)(2 * ow) * (float)(2 * oh));
-        // tile index = slot * bands + band, advanced by gridDim.x per tile without divisions
-        const int step_slot = (int)(gridDim.x / (unsigned)bands), step_band = (int)(gridDim.x % (unsigned)bands);
-        int w_slot = (int)(blockIdx.x / (unsigned)bands), w_band = (int)(blockIdx.x % (unsigned)bands);
+        // Tiles of this CTA: index blockIdx.x + t * gridDim.x = slot * bands + band, t = 0, 1, ...
+        // Items are resolved 32 tiles at a time, one per lane (q_* registers), so the dependent
+        // loads slot -> detection index -> detection cost one round trip per 32 tiles.
+        int w_tiles = 0;  // tiles opened so far
+        int q_slot = 0, q_band = 0, q_frame = 0, q_rx0 = 0, q_ry0 = 0, q_rx1 = 1, q_ry1 = 1;
+        int w_slot = 0, w_band = 0;
         int w_frame = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
         int w_row_lo = 0, w_row_hi = 0, w_tile_cols = ow;
         int w_c0 = 0, w_ncols = 0, w_r0 = 0, w_nr = 0;
@@ -178,14 +142,54 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
             if (pr >= kCropConsumerWarps) pr &= ~(kCropConsumerWarps - 1);
             w_pass_rows = max(1, min(pr, band_rows));
         };
-        // first pass of the tile (w_slot, w_band), if there is one
+        // lane l resolves the item of tile w_tiles + l
+        auto resolve_batch = [&]() {
+            const long long tile = (long long)blockIdx.x + (long long)(w_tiles + lane) * (long long)gridDim.x;
+            q_slot = (int)min(tile / bands, (long long)packed);  // >= packed: no such tile
+            q_band = (int)(tile % bands);
+            if (q_slot >= packed) return;
+            const int item = first_item + q_slot;
+            int lo = 0, hi = n;  // largest f with s_off[f] <= item (frames without items are skipped)
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (s_off[mid] <= item) lo = mid; else hi = mid;
+            }
+            const int f = lo;
+            const int det = bidx[(size_t)f * max_det + (item - s_off[f])];
+            const octo_det_t d = dets[(size_t)f * max_det + det];
+            const FrameDesc& fd = tab.f[f];
+            // outward-rounded rectangle, clamped so that it is never empty
+            int rx0 = (int)floorf(d.x1), ry0 = (int)floorf(d.y1);
+            int rx1 = (int)ceilf(d.x2), ry1 = (int)ceilf(d.y2);
+            rx0 = min(max(rx0, 0), fd.w - 1);
+            ry0 = min(max(ry0, 0), fd.h - 1);
+            rx1 = min(max(rx1, rx0 + 1), fd.w);
+            ry1 = min(max(ry1, ry0 + 1), fd.h);
+            if (q_band == 0) {  // the tile of a slot's first band records the item
+                octo_item_t it;
+                it.frame = f; it.det = det;
+                it.rx0 = rx0; it.ry0 = ry0; it.rx1 = rx1; it.ry1 = ry1;
+                it._pad[0] = 0; it._pad[1] = 0;
+                items[q_slot] = it;
+            }
+            q_frame = f; q_rx0 = rx0; q_ry0 = ry0; q_rx1 = rx1; q_ry1 = ry1;
+        };
+        // first pass of the next tile, if there is one
         auto open_tile = [&]() {
+            const int src = w_tiles & 31;
+            if (src == 0) resolve_batch();
+            __syncwarp();
+            w_tiles += 1;
+            w_slot = __shfl_sync(0xffffffffu, q_slot, src);
+            w_band = __shfl_sync(0xffffffffu, q_band, src);
+            const int f = __shfl_sync(0xffffffffu, q_frame, src);
+            const int rx0 = __shfl_sync(0xffffffffu, q_rx0, src), ry0 = __shfl_sync(0xffffffffu, q_ry0, src);
+            const int rx1 = __shfl_sync(0xffffffffu, q_rx1, src), ry1 = __shfl_sync(0xffffffffu, q_ry1, src);
             w_valid = w_slot < packed;
             if (!w_valid) return;
-            const octo_item_t it = items[w_slot];
-            w_frame = it.frame;
-            w_rx0 = it.rx0; w_ry0 = it.ry0; w_cw = it.rx1 - it.rx0; w_ch = it.ry1 - it.ry0;
-            const int full_seg = ((3 * it.rx1 + 15) & ~15) - ((3 * it.rx0) & ~15);
+            w_frame = f;
+            w_rx0 = rx0; w_ry0 = ry0; w_cw = rx1 - rx0; w_ch = ry1 - ry0;
+            const int full_seg = ((3 * rx1 + 15) & ~15) - ((3 * rx0) & ~15);
             w_tile_cols =
                 (full_seg + 16 > kCropMaxStride) ? max(2, (int)((long long)kCropTilePx * ow / w_cw) & ~1) : ow;
             w_c0 = 0;
@@ -205,9 +209,6 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
                 set_tile();
                 w_r0 = w_row_lo;
             } else {
-                w_slot += step_slot;
-                w_band += step_band;
-                if (w_band >= bands) { w_band -= bands; w_slot += 1; }
                 open_tile();
                 return;
             }
@@ -312,31 +313,22 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const octo_item_t* __re
 }
 
 template <int CAP>
-static cudaError_t launch_assemble_cap(const CropArgs& a, cudaStream_t stream) {
-    static FrameTable<CAP> tab;
-    for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
-    assemble_kernel<CAP><<<1, kAsmThreads, 0, stream>>>(tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount,
-                                                       a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items, a.d_items,
-                                                       a.d_ctr);
-    return cudaGetLastError();
-}
-
-template <int CAP>
 static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     static FrameTable<CAP> tab;
     for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
-    // rows per (slot, band) tile: about 4096 pixels, a multiple of the warp count
+    // rows per (slot, band) tile: about 4096 pixels, a multiple of the consumer warp count
     int band_rows = (4096 / a.out_w) & ~7;
     band_rows = band_rows < 8 ? 8 : band_rows;
     band_rows = band_rows > a.out_h ? a.out_h : band_rows;
     const int bands = (a.out_h + band_rows - 1) / band_rows;
     long long work = (long long)a.max_items * bands;
     long long cap = (long long)a.sm_count * kCropCtasPerSm;
-    const int grid = (int)(work < cap ? work : cap);
+    int grid = (int)(work < cap ? work : cap);
+    if (grid < 1) grid = 1;  // a zero-slot window still gets its offsets and totals
     const size_t smem = 2 * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w);
-    crop_kernel<CAP><<<grid, kCropKernelThreads, smem, stream>>>(tab, a.d_items, a.d_n_items,
-                                                          reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h,
-                                                          band_rows, a.swap_rb, &a.d_ctr->status);
+    crop_kernel<CAP><<<grid, kCropKernelThreads, smem, stream>>>(
+        tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
+        a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, band_rows, a.swap_rb, a.d_ctr);
     return cudaGetLastError();
 }
 
@@ -350,13 +342,7 @@ cudaError_t prepare_crop() {
     return cudaFuncSetAttribute(crop_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 
-cudaError_t launch_assemble(const CropArgs& a, cudaStream_t stream) {
-    if (a.n <= 8) return launch_assemble_cap<8>(a, stream);
-    if (a.n <= 64) return launch_assemble_cap<64>(a, stream);
-    return launch_assemble_cap<512>(a, stream);
-}
-
-// Requires a.max_items > 0.
+// Assembler + crop-resize of one branch window (a.max_items may be 0).
 cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream) {
     if (a.n <= 8) return launch_crop_cap<8>(a, stream);
     if (a.n <= 64) return launch_crop_cap<64>(a, stream);

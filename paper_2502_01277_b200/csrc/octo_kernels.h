@@ -61,8 +61,7 @@ cudaError_t launch_decode(const float* d_head, int n, int A, int C, int logits, 
                           unsigned long long* d_keys, int* d_cand_count, unsigned int* d_status,
                           cudaStream_t stream);
 cudaError_t launch_nms(const NmsArgs& a, cudaStream_t stream);
-cudaError_t launch_assemble(const CropArgs& a, cudaStream_t stream);
-cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream);  // needs a.max_items > 0
+cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream);  // batch assembler + crop-resize
 
 constexpr int kLetterboxMaxWidth = 8192;  // widest frame the row staging supports
 

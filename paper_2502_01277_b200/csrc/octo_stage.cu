@@ -313,15 +313,10 @@ extern "C" int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_i
     OCTO_CUDA(cudaSetDevice(c.device));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     {
-        ScopedKernelTimer t(st, OCTO_K_ASSEMBLE, stream);
-        OCTO_CUDA(launch_assemble(a, stream));
-    }
-    st->launches += 1;
-    if (max_items > 0) {
         ScopedKernelTimer t(st, OCTO_K_CROP, stream);
         OCTO_CUDA(launch_crop(a, stream));
-        st->launches += 1;
     }
+    st->launches += 1;
     return OCTO_OK;
 }
 
