@@ -286,16 +286,37 @@ __device__ __forceinline__ float4 box_corners(float cx, float cy, float bw, floa
 }
 
 // IoU, operation by operation: inter / ((area_a + area_b) - inter), 0 if the union is empty.
-__device__ __forceinline__ float iou_fixed(const float4 a, const float4 b) {
+__device__ __forceinline__ void iou_terms(const float4 a, const float4 b, float& inter, float& uni) {
     float iw = __fsub_rn(fminf(a.z, b.z), fmaxf(a.x, b.x));
     float ih = __fsub_rn(fminf(a.w, b.w), fmaxf(a.y, b.y));
     iw = fmaxf(iw, 0.0f);
     ih = fmaxf(ih, 0.0f);
-    const float inter = __fmul_rn(iw, ih);
+    inter = __fmul_rn(iw, ih);
     const float area_a = __fmul_rn(__fsub_rn(a.z, a.x), __fsub_rn(a.w, a.y));
     const float area_b = __fmul_rn(__fsub_rn(b.z, b.x), __fsub_rn(b.w, b.y));
-    const float uni = __fsub_rn(__fadd_rn(area_a, area_b), inter);
+    uni = __fsub_rn(__fadd_rn(area_a, area_b), inter);
+}
+__device__ __forceinline__ float iou_fixed(const float4 a, const float4 b) {
+    float inter, uni;
+    iou_terms(a, b, inter, uni);
     return uni > 0.0f ? __fdiv_rn(inter, uni) : 0.0f;
+}
+
+// The test fl(inter / uni) > thr without the division.  The binary32 quotient rounds to a
+// value above thr exactly when the real quotient lies above the midpoint `mid` of thr and the
+// next float up (or on it, when that next float has an even mantissa and so wins the tie).
+// inter, uni and mid have 24, 24 and 25 significant bits, so mid * uni is exact in binary64
+// and the comparison is exact.  Non-finite operands compare false, like the quotient would.
+struct IouTest {
+    double mid;
+    int tie_up;
+};
+__device__ __forceinline__ bool iou_above(const float4 a, const float4 b, const IouTest t) {
+    float inter, uni;
+    iou_terms(a, b, inter, uni);
+    if (!(uni > 0.0f)) return false;
+    const double lhs = (double)inter, rhs = __dmul_rn(t.mid, (double)uni);
+    return t.tie_up ? lhs >= rhs : lhs > rhs;
 }
 
 }  // namespace octo

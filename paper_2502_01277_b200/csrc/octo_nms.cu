@@ -1,40 +1,67 @@
 // Per-image ordering + class-aware greedy NMS + cap + scale-back (one CTA per image).
 //
-// Latency / shared-memory bound; bytes are negligible.  The candidate keys of an image
-// (class | inverted score bits | anchor) are sorted in shared memory with a bitonic network,
-// which groups classes and orders each class by score (ties: lower anchor).  Boxes are
-// gathered once from the head by anchor.  Classes are independent under class-aware NMS, so
-// each warp runs the greedy scan of whole classes: 32 candidates at a time are tested
-// against the class's survivors so far (broadcast reads of shared memory), then resolved
-// among themselves with ballots and register shuffles.  Survivors are compacted in place,
-// re-keyed to (inverted score | anchor | class) and sorted once more to obtain the global
-// score order; the first max_det are mapped back to frame pixels and written out, together
-// with each downstream branch's class-filtered index list.
+// Latency / shared-memory bound; bytes are negligible.  Classes are independent under
+// class-aware NMS, so the image's candidate keys (class | inverted score bits | anchor) are
+// first bucketed by class in shared memory (histogram, scan, scatter).  Each warp then owns
+// whole classes: it sorts the class's keys with a warp-level bitonic network (score
+// descending, ties by lower anchor), gathers the boxes from the head by anchor and runs the
+// greedy scan: 32 candidates at a time are tested against the class's survivors so far
+// (broadcast reads of shared memory), then resolved among themselves with ballots and
+// register shuffles.  Survivors are compacted in place and re-keyed to (inverted score |
+// anchor | class).  The global score order is a merge of the per-class survivor lists: the
+// rank of a survivor is its index in its own list plus, for every other class, the number of
+// that class's survivors that precede it (binary search).  The first max_det in that order
+// are mapped back to frame pixels and written out, together with each downstream branch's
+// class-filtered index list.
 //
 // Images with more candidates than fit in shared memory take the same code path with the
-// arrays in a global-memory workspace.
+// arrays in a global-memory workspace; classes with more than kWarpSortMax candidates are
+// sorted by the whole CTA.
 #include "octo_common.cuh"
+#include <cmath>
+#include <cstring>
+
 #include "octo_kernels.h"
 
 namespace octo {
 
 constexpr int kNmsThreads = 1024;
-constexpr int kNmsSmemCap = 8192;  // candidates sorted on chip: 8 B key + 16 B box each
+constexpr int kNmsSmemCap = 8192;   // candidates handled on chip: 8 B key + 16 B box each
+constexpr int kWarpSortMax = 2048;  // largest class segment a single warp sorts
 
-__device__ __forceinline__ void bitonic_sort(unsigned long long* __restrict__ k, int np2) {
+__device__ __forceinline__ void cmp_swap(unsigned long long* __restrict__ k, int i, int j) {
+    const unsigned long long a = k[i], b = k[j];
+    if (a > b) { k[i] = b; k[j] = a; }
+}
+
+// Ascending bitonic sort of k[0, m) for any m, by `nthreads` cooperating threads (a warp or
+// the whole CTA).  Every comparator puts the smaller key at the lower index (the first stage
+// of each merge pairs mirrored positions), so positions >= m can stand for +infinity and are
+// simply skipped.
+template <bool BLOCK>
+__device__ __forceinline__ void bitonic_range(unsigned long long* __restrict__ k, int m, int tid, int nthreads) {
+    int np2 = 2;
+    while (np2 < m) np2 <<= 1;
+    const int half = np2 >> 1;
     for (int size = 2; size <= np2; size <<= 1) {
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            __syncthreads();
-            for (int t = threadIdx.x; t < (np2 >> 1); t += kNmsThreads) {
-                const int lo = 2 * t - (t & (stride - 1));  // index with bit `stride` clear
-                const int hi = lo + stride;
-                const unsigned long long a = k[lo], b = k[hi];
-                const bool up = (lo & size) == 0;
-                if ((a > b) == up) { k[lo] = b; k[hi] = a; }
+        if (BLOCK) __syncthreads(); else __syncwarp();
+        const int h = size >> 1;
+        for (int t = tid; t < half; t += nthreads) {
+            const int off = t & (h - 1);
+            const int i = 2 * t - off;           // block start + off
+            const int j = i + size - 1 - 2 * off;  // mirrored position in the block
+            if (j < m) cmp_swap(k, i, j);
+        }
+        for (int stride = size >> 2; stride > 0; stride >>= 1) {
+            if (BLOCK) __syncthreads(); else __syncwarp();
+            for (int t = tid; t < half; t += nthreads) {
+                const int i = 2 * t - (t & (stride - 1));
+                const int j = i + stride;
+                if (j < m) cmp_swap(k, i, j);
             }
         }
     }
-    __syncthreads();
+    if (BLOCK) __syncthreads(); else __syncwarp();
 }
 
 __device__ __forceinline__ float4 gather_box(const float* __restrict__ hrow) {
@@ -42,15 +69,16 @@ __device__ __forceinline__ float4 gather_box(const float* __restrict__ hrow) {
 }
 
 template <int CAP>
-__global__ void __launch_bounds__(kNmsThreads)
+__global__ void __launch_bounds__(kNmsThreads, 1)
 nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict__ head, int A, int C,
-           float iou_thr, int max_det, int key_stride, unsigned long long* __restrict__ gkeys,
+           const IouTest iou_test, int max_det, int key_stride, unsigned long long* __restrict__ gkeys,
            float4* __restrict__ gboxes, int* __restrict__ cand_count, octo_det_rec* __restrict__ dets,
            int* __restrict__ counts, int num_branches, const __grid_constant__ BranchMasks masks,
            int* __restrict__ bcount, int* __restrict__ bidx, int max_batch, StageCounters* __restrict__ ctr) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ int seg_start[128], seg_end[128];
-    __shared__ int s_total;
+    __shared__ int seg_start[128], seg_cnt[128], cursor[128], nkept[128];
+    __shared__ int live[128];  // classes with survivors
+    __shared__ int s_total, s_live, s_big;
 
     const int img = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -59,103 +87,202 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
 
     int cnt = cand_count[img];
     cnt = min(cnt, min(A, key_stride));
+    if (threadIdx.x < 128) { seg_cnt[threadIdx.x] = 0; nkept[threadIdx.x] = 0; }
     __syncthreads();
     if (threadIdx.x == 0) {
         cand_count[img] = 0;  // ready for the next batch's decode
         atomicAdd(&ctr->candidates, (unsigned long long)cnt);
         atomicMax(&ctr->max_cand, cnt);
         s_total = 0;
+        s_live = 0;
+        s_big = 0;
     }
-    if (threadIdx.x < 128) { seg_start[threadIdx.x] = 0; seg_end[threadIdx.x] = 0; }
 
-    int np2 = 2;
-    while (np2 < cnt) np2 <<= 1;
-
+    unsigned long long* const gk = gkeys + (size_t)img * key_stride;
+    const bool on_chip = cnt <= kNmsSmemCap;
     unsigned long long* keys;
     float4* boxes;
-    unsigned long long* const gk = gkeys + (size_t)img * key_stride;
-    if (np2 <= kNmsSmemCap) {
-        keys = reinterpret_cast<unsigned long long*>(smem_raw + (size_t)kNmsSmemCap * sizeof(float4));
+    if (on_chip) {
         boxes = reinterpret_cast<float4*>(smem_raw);
-        for (int i = threadIdx.x; i < np2; i += kNmsThreads) keys[i] = i < cnt ? gk[i] : kKeySentinel;
+        keys = reinterpret_cast<unsigned long long*>(smem_raw + (size_t)kNmsSmemCap * sizeof(float4));
     } else {
-        keys = gk;  // key_stride is a power of two >= A, so the padded length fits
         boxes = gboxes + (size_t)img * key_stride;
-        for (int i = cnt + threadIdx.x; i < np2; i += kNmsThreads) keys[i] = kKeySentinel;
+        keys = gk;
         if (threadIdx.x == 0) atomicOr(&ctr->status, 0x8u);
     }
 
-    if (cnt > 0) {
-        // ---- class-major order: class, then score descending, then anchor ascending ----
-        bitonic_sort(keys, np2);
-
-        // ---- class segments and boxes ----
-        for (int p = threadIdx.x; p < cnt; p += kNmsThreads) {
-            const unsigned long long k = keys[p];
-            const int cls = (int)(k >> 57);
-            if (p == 0 || (int)(keys[p - 1] >> 57) != cls) seg_start[cls] = p;
-            if (p == cnt - 1 || (int)(keys[p + 1] >> 57) != cls) seg_end[cls] = p + 1;
-            const int anchor = (int)(k & ((1ull << kKeyAnchorBits) - 1));
-            boxes[p] = gather_box(hbase + (size_t)anchor * row_len);
+    // ---- bucket the keys by class: histogram, scan, scatter ----
+    for (int i = threadIdx.x; i < cnt; i += kNmsThreads) atomicAdd(&seg_cnt[(int)(gk[i] >> 57)], 1);
+    __syncthreads();
+    if (warp == 0) {
+        int run = 0;
+#pragma unroll
+        for (int base = 0; base < 128; base += 32) {
+            const int v = seg_cnt[base + lane];
+            int inc = v;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, inc, off);
+                if (lane >= off) inc += t;
+            }
+            seg_start[base + lane] = run + inc - v;
+            cursor[base + lane] = run + inc - v;
+            run += __shfl_sync(0xffffffffu, inc, 31);
+            if (__any_sync(0xffffffffu, v > kWarpSortMax) && lane == 0) s_big = 1;
+        }
+    }
+    __syncthreads();
+    {
+        // off chip the scatter goes through the box workspace and back into the key array
+        unsigned long long* const dst = on_chip ? keys : reinterpret_cast<unsigned long long*>(boxes);
+        for (int i = threadIdx.x; i < cnt; i += kNmsThreads) {
+            const unsigned long long k = gk[i];
+            dst[atomicAdd(&cursor[(int)(k >> 57)], 1)] = k;
         }
         __syncthreads();
-
-        // ---- greedy NMS, one warp per class ----
-        for (int cls = warp; cls < 128; cls += kNmsThreads / 32) {
-            const int s = seg_start[cls], e = seg_end[cls];
-            int nk = 0;  // survivors of this class, compacted at [s, s + nk)
-            for (int c0 = s; c0 < e && nk < max_det; c0 += 32) {
-                const int p = c0 + lane;
-                const bool valid = p < e;
-                float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-                unsigned long long k = kKeySentinel;
-                if (valid) { b = boxes[p]; k = keys[p]; }
-                bool alive = valid;
-                for (int t = 0; t < nk; ++t) {
-                    if (!__any_sync(0xffffffffu, alive)) break;
-                    const float4 kb = boxes[s + t];
-                    if (alive && iou_fixed(kb, b) > iou_thr) alive = false;
-                }
-                unsigned rem = __ballot_sync(0xffffffffu, alive);
-                unsigned keptmask = 0;
-                while (rem) {
-                    const int l = __ffs(rem) - 1;
-                    keptmask |= 1u << l;
-                    float4 lb;
-                    lb.x = __shfl_sync(0xffffffffu, b.x, l);
-                    lb.y = __shfl_sync(0xffffffffu, b.y, l);
-                    lb.z = __shfl_sync(0xffffffffu, b.z, l);
-                    lb.w = __shfl_sync(0xffffffffu, b.w, l);
-                    if (alive && lane > l && iou_fixed(lb, b) > iou_thr) alive = false;
-                    rem = __ballot_sync(0xffffffffu, alive) & ~((2u << l) - 1u);
-                }
-                __syncwarp();
-                const int allowed = min(__popc(keptmask), max_det - nk);
-                if ((keptmask >> lane) & 1u) {
-                    const int r = __popc(keptmask & ((1u << lane) - 1u));
-                    if (r < allowed) {
-                        boxes[s + nk + r] = b;
-                        // re-key for the global order: inverted score | anchor | class
-                        keys[s + nk + r] = ((k & ((1ull << 57) - 1)) << 7) | (k >> 57);
-                    }
-                }
-                __syncwarp();
-                nk += allowed;
-            }
-            for (int p = s + nk + lane; p < e; p += 32) keys[p] = kKeySentinel;
-            if (lane == 0 && nk > 0) atomicAdd(&s_total, nk);
+        if (!on_chip) {
+            for (int i = threadIdx.x; i < cnt; i += kNmsThreads) keys[i] = dst[i];
+            __syncthreads();
         }
+    }
 
-        // ---- global order of the survivors ----
-        bitonic_sort(keys, np2);
+    // ---- very large classes are sorted by the whole CTA ----
+    if (s_big) {
+        for (int cls = 0; cls < 128; ++cls) {
+            const int m = seg_cnt[cls];
+            if (m > kWarpSortMax) bitonic_range<true>(keys + seg_start[cls], m, threadIdx.x, kNmsThreads);
+        }
+    }
+
+    // ---- one warp per class: sort, gather boxes, greedy NMS ----
+    for (int cls = warp; cls < 128; cls += kNmsThreads / 32) {
+        const int m = seg_cnt[cls];
+        if (m == 0) continue;
+        const int s = seg_start[cls], e = s + m;
+        if (m > 1 && m <= kWarpSortMax) bitonic_range<false>(keys + s, m, lane, 32);
+        for (int p = s + lane; p < e; p += 32) {
+            const int anchor = (int)(keys[p] & ((1ull << kKeyAnchorBits) - 1));
+            boxes[p] = gather_box(hbase + (size_t)anchor * row_len);
+        }
+        __syncwarp();
+        int nk = 0;  // survivors of this class, compacted at [s, s + nk)
+        for (int c0 = s; c0 < e && nk < max_det; c0 += 32) {
+            const int p = c0 + lane;
+            const bool valid = p < e;
+            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+            unsigned long long k = kKeySentinel;
+            if (valid) { b = boxes[p]; k = keys[p]; }
+            bool alive = valid;
+            for (int t = 0; t < nk; ++t) {
+                if (!__any_sync(0xffffffffu, alive)) break;
+                const float4 kb = boxes[s + t];
+                if (alive && iou_above(kb, b, iou_test)) alive = false;
+            }
+            unsigned rem = __ballot_sync(0xffffffffu, alive);
+            unsigned keptmask = 0;
+            while (rem) {
+                const int l = __ffs(rem) - 1;
+                keptmask |= 1u << l;
+                float4 lb;
+                lb.x = __shfl_sync(0xffffffffu, b.x, l);
+                lb.y = __shfl_sync(0xffffffffu, b.y, l);
+                lb.z = __shfl_sync(0xffffffffu, b.z, l);
+                lb.w = __shfl_sync(0xffffffffu, b.w, l);
+                if (alive && lane > l && iou_above(lb, b, iou_test)) alive = false;
+                rem = __ballot_sync(0xffffffffu, alive) & ~((2u << l) - 1u);
+            }
+            __syncwarp();
+            const int allowed = min(__popc(keptmask), max_det - nk);
+            if ((keptmask >> lane) & 1u) {
+                const int r = __popc(keptmask & ((1u << lane) - 1u));
+                if (r < allowed) {
+                    boxes[s + nk + r] = b;
+                    // re-key for the global order: inverted score | anchor | class
+                    keys[s + nk + r] = ((k & ((1ull << 57) - 1)) << 7) | (k >> 57);
+                }
+            }
+            __syncwarp();
+            nk += allowed;
+        }
+        for (int p = s + nk + lane; p < e; p += 32) keys[p] = kKeySentinel;
+        if (lane == 0 && nk > 0) {
+            nkept[cls] = nk;
+            atomicAdd(&s_total, nk);
+            live[atomicAdd(&s_live, 1)] = cls;
+        }
     }
     __syncthreads();
 
+    // ---- global score order: merge of the per-class survivor lists by rank ----
     const int nout = min(s_total, max_det);
+    const int nlive = s_live;
+    if (warp == 0) {
+        // exclusive scan of the survivor counts over the live classes -> cursor[q]
+        int run = 0;
+        for (int base = 0; base < nlive; base += 32) {
+            const int q = base + lane;
+            const int v = q < nlive ? nkept[live[q]] : 0;
+            int inc = v;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, inc, off);
+                if (lane >= off) inc += t;
+            }
+            if (q < nlive) cursor[q] = run + inc - v;
+            run += __shfl_sync(0xffffffffu, inc, 31);
+        }
+    }
+    __syncthreads();
+    // boxes are no longer needed: their memory holds the ordered survivors and the ranks
+    unsigned long long* const ordered = reinterpret_cast<unsigned long long*>(boxes);
+    int* const rank = reinterpret_cast<int*>(ordered + min(max_det, cnt));
+    const int total = s_total;
+    // survivor e (dense numbering over the live classes): rank starts as the index in its own list
+    for (int e = threadIdx.x; e < total; e += kNmsThreads) {
+        int lo = 0, hi = nlive;  // live class q with cursor[q] <= e < cursor[q + 1]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (cursor[mid] <= e) lo = mid; else hi = mid;
+        }
+        rank[e] = e - cursor[lo];
+    }
+    __syncthreads();
+    // every (survivor, other live class) pair adds the number of that class's survivors that
+    // precede the survivor; pairs are independent, so the searches run in parallel
+    for (int i = threadIdx.x; i < total * nlive; i += kNmsThreads) {
+        const int e = i / nlive, q = i - e * nlive;
+        int lo = 0, hi = nlive;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (cursor[mid] <= e) lo = mid; else hi = mid;
+        }
+        if (lo == q) continue;
+        const unsigned long long g = keys[seg_start[live[lo]] + (e - cursor[lo])];
+        const unsigned long long* const list = keys + seg_start[live[q]];
+        int l2 = 0, h2 = nkept[live[q]];
+        while (l2 < h2) {
+            const int mid = (l2 + h2) >> 1;
+            if (list[mid] < g) l2 = mid + 1; else h2 = mid;
+        }
+        if (l2) atomicAdd(&rank[e], l2);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < total; e += kNmsThreads) {
+        const int r = rank[e];
+        if (r >= max_det) continue;
+        int lo = 0, hi = nlive;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (cursor[mid] <= e) lo = mid; else hi = mid;
+        }
+        ordered[r] = keys[seg_start[live[lo]] + (e - cursor[lo])];
+    }
+    __syncthreads();
+
     const FrameDesc& fd = tab.f[img];
     const float fw = (float)fd.w, fh = (float)fd.h, fpl = (float)fd.pad_l, fpt = (float)fd.pad_t;
     for (int r = threadIdx.x; r < nout; r += kNmsThreads) {
-        const unsigned long long g = keys[r];
+        const unsigned long long g = ordered[r];
         const int cls = (int)(g & 127u);
         const int anchor = (int)((g >> 7) & ((1ull << kKeyAnchorBits) - 1));
         const float score = __uint_as_float(~(unsigned)(g >> 32));
@@ -183,7 +310,7 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
             const int r = r0 + lane;
             bool take = false;
             if (r < nout) {
-                const unsigned cls = (unsigned)(keys[r] & 127u);
+                const unsigned cls = (unsigned)(ordered[r] & 127u);
                 take = (masks.m[warp][cls >> 5] >> (cls & 31u)) & 1u;
             }
             const unsigned bal = __ballot_sync(0xffffffffu, take);
@@ -210,7 +337,14 @@ static cudaError_t launch_cap(const NmsArgs& a, cudaStream_t stream) {
     static FrameTable<CAP> tab;
     for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
     const size_t smem = kNmsSmemBytes;
-    nms_kernel<CAP><<<a.n, kNmsThreads, smem, stream>>>(tab, a.d_head, a.A, a.C, a.iou_thr, a.max_det, a.key_stride,
+    // rounding boundary of the IoU test (see iou_above)
+    const float up = nextafterf(a.iou_thr, INFINITY);
+    IouTest iou_test;
+    iou_test.mid = 0.5 * ((double)a.iou_thr + (double)up);
+    unsigned int up_bits;
+    memcpy(&up_bits, &up, sizeof(up_bits));
+    iou_test.tie_up = (up_bits & 1u) == 0u ? 1 : 0;
+    nms_kernel<CAP><<<a.n, kNmsThreads, smem, stream>>>(tab, a.d_head, a.A, a.C, iou_test, a.max_det, a.key_stride,
                                                        a.d_keys, a.d_boxes, a.d_cand_count,
                                                        reinterpret_cast<octo_det_rec*>(a.d_dets), a.d_counts,
                                                        a.num_branches, a.masks, a.d_bcount, a.d_bidx, a.max_batch,
