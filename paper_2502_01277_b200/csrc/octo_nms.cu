@@ -28,6 +28,7 @@ namespace octo {
 constexpr int kNmsThreads = 1024;
 constexpr int kNmsSmemCap = 8192;   // candidates handled on chip: 8 B key + 16 B box each
 constexpr int kWarpSortMax = 2048;  // largest class segment a single warp sorts
+constexpr int kRankSortMax = 512;   // up to here the warp sorts by counting instead of a network
 
 __device__ __forceinline__ void cmp_swap(unsigned long long* __restrict__ k, int i, int j) {
     const unsigned long long a = k[i], b = k[j];
@@ -159,7 +160,32 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
         const int m = seg_cnt[cls];
         if (m == 0) continue;
         const int s = seg_start[cls], e = s + m;
-        if (m > 1 && m <= kWarpSortMax) bitonic_range<false>(keys + s, m, lane, 32);
+        if (m > 1 && m <= kRankSortMax) {
+            // small class: every key counts the keys below it and moves to that position, staged
+            // in the (not yet used) box slots of the segment
+            unsigned long long* const tmp = reinterpret_cast<unsigned long long*>(boxes + s);
+            for (int i0 = lane; i0 < m; i0 += 128) {
+                // up to four keys per lane share one pass over the segment
+                const unsigned long long k0 = keys[s + i0];
+                const unsigned long long k1 = i0 + 32 < m ? keys[s + i0 + 32] : kKeySentinel;
+                const unsigned long long k2 = i0 + 64 < m ? keys[s + i0 + 64] : kKeySentinel;
+                const unsigned long long k3 = i0 + 96 < m ? keys[s + i0 + 96] : kKeySentinel;
+                int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+                for (int j = 0; j < m; ++j) {
+                    const unsigned long long kj = keys[s + j];
+                    r0 += kj < k0; r1 += kj < k1; r2 += kj < k2; r3 += kj < k3;
+                }
+                tmp[r0] = k0;
+                if (i0 + 32 < m) tmp[r1] = k1;
+                if (i0 + 64 < m) tmp[r2] = k2;
+                if (i0 + 96 < m) tmp[r3] = k3;
+            }
+            __syncwarp();
+            for (int p = lane; p < m; p += 32) keys[s + p] = tmp[p];
+            __syncwarp();
+        } else if (m > 1 && m <= kWarpSortMax) {
+            bitonic_range<false>(keys + s, m, lane, 32);
+        }
         for (int p = s + lane; p < e; p += 32) {
             const int anchor = (int)(keys[p] & ((1ull << kKeyAnchorBits) - 1));
             boxes[p] = gather_box(hbase + (size_t)anchor * row_len);
@@ -249,8 +275,10 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
     __syncthreads();
     // every (survivor, other live class) pair adds the number of that class's survivors that
     // precede the survivor; pairs are independent, so the searches run in parallel
+    // (neighbouring threads take neighbouring survivors against the same class, so the list reads
+    // broadcast and the rank updates hit different addresses)
     for (int i = threadIdx.x; i < total * nlive; i += kNmsThreads) {
-        const int e = i / nlive, q = i - e * nlive;
+        const int q = i / total, e = i - q * total;
         int lo = 0, hi = nlive;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
