@@ -316,13 +316,18 @@ template <int CAP>
 static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     static FrameTable<CAP> tab;
     for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
-    // rows per (slot, band) tile: about 4096 pixels, a multiple of the consumer warp count
-    int band_rows = (4096 / a.out_w) & ~7;
-    band_rows = band_rows < 8 ? 8 : band_rows;
+    // Tiles are (slot, row band).  One band per crop amortises the per-tile work (item lookup,
+    // tap table) best; crops are only cut into bands when there are too few of them to fill
+    // the grid about eight times over (the slots are usually provisioned generously).  Bands are multiples of the consumer warp count.
+    const long long cap = (long long)a.sm_count * kCropCtasPerSm;
+    const long long slots = a.max_items > 0 ? a.max_items : 1;
+    long long bands_want = (8 * cap + slots - 1) / slots;
+    const int max_bands = (a.out_h + 7) / 8;
+    const int bands_req = (int)(bands_want < 1 ? 1 : (bands_want > max_bands ? max_bands : bands_want));
+    int band_rows = ((a.out_h + bands_req - 1) / bands_req + 7) & ~7;
     band_rows = band_rows > a.out_h ? a.out_h : band_rows;
     const int bands = (a.out_h + band_rows - 1) / band_rows;
     long long work = (long long)a.max_items * bands;
-    long long cap = (long long)a.sm_count * kCropCtasPerSm;
     int grid = (int)(work < cap ? work : cap);
     if (grid < 1) grid = 1;  // a zero-slot window still gets its offsets and totals
     const size_t smem = 2 * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w);
