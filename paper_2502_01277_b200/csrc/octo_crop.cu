@@ -13,25 +13,27 @@
 // tiles: it resolves the item, builds the table of horizontal taps (byte offset + exact
 // integer weights per output column) and has the bulk-copy engine stage the 16-byte aligned
 // segments of the source rows a pass taps into one of two shared-memory buffers (mbarrier
-// "full" / "empty" ring, every wait bounded).  Eight consumer warps take one output row
-// each: lane l owns pixel pairs l, l+32, ... so neighbouring lanes read neighbouring table
-// entries and row words; the horizontal lerp is an exact integer two-way dot product per
-// channel, the vertical lerp and all scaling are two fp32 operations, and a warp writes 128
-// contiguous bytes per plane straight into the downstream slot.
+// "full" / "empty" ring, every wait bounded).  The 256 threads of the eight consumer warps
+// walk a pass as a flat, row-major list of pixel pairs, so every lane is busy and
+// neighbouring lanes read neighbouring table entries and row words; the horizontal lerp is
+// an exact integer two-way dot product per channel, the vertical lerp and all scaling are two
+// fp32 operations, and a warp writes up to 128 contiguous bytes per plane straight into the
+// downstream slot.  Measured: large passes matter more than occupancy (2 x 32 KB buffers at
+// 3 CTAs/SM beat 2 x 24 KB at 4 and 4 x 12 KB at 4).
 #include "octo_common.cuh"
 #include "octo_kernels.h"
 
 namespace octo {
 
 // Shared memory for staged source rows.  A pass stages two row segments per output row; a
-// segment longer than kCropMaxStride - 16 bytes (a rectangle wider than about 4000 pixels)
+// segment longer than kCropMaxStride - 16 bytes (a rectangle wider than about 5300 pixels)
 // is split into column tiles, so one row pair always fits.  Two buffers form a ring between
 // the producer warp and the consumer warps.
-constexpr int kCropRowBudget = 24576;
+constexpr int kCropRowBudget = 32768;
 constexpr int kCropMaxStride = kCropRowBudget / 2;
-constexpr int kCropTilePx = 4000;
+constexpr int kCropTilePx = 5300;
 constexpr int kCropMaxPassRows = 32;
-constexpr int kCropCtasPerSm = 4;
+constexpr int kCropCtasPerSm = 3;
 constexpr int kCropConsumerWarps = 8;
 constexpr int kCropKernelThreads = 32 * (kCropConsumerWarps + 1);  // + one producer warp
 
@@ -137,10 +139,7 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             w_seg_lo = lo;
             w_seg = hi - lo;
             w_stride = w_seg + 16;
-            // whole multiples of the consumer warp count keep every warp busy (one warp per row)
-            int pr = min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows);
-            if (pr >= kCropConsumerWarps) pr &= ~(kCropConsumerWarps - 1);
-            w_pass_rows = max(1, min(pr, band_rows));
+            w_pass_rows = max(1, min(min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows), band_rows));
         };
         // lane l resolves the item of tile w_tiles + l
         auto resolve_batch = [&]() {
@@ -291,20 +290,37 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             fphase[b] ^= 1u;
             const CropPass cur = s_pass[b];
             if (!cur.valid) break;
-            // one warp per output row of the pass
+            // flat list of pixel pairs (row-major); thread t of the consumers owns pairs t, t+256, ...
             const uint32_t xt = smem_u32(s_xtab0) + (uint32_t)(cur.table * ow + cur.c0) * (uint32_t)sizeof(XEntry);
             const uint32_t rows = smem_u32(s_rows0) + (uint32_t)b * kCropRowBudget;
+            const uint32_t rinfo = smem_u32(&s_row[b][0]);
             const size_t tile_off = (size_t)cur.slot * 3 * plane + (size_t)cur.r0 * ow + cur.c0;
+            __half* const t0 = out0 + tile_off;
+            __half* const t1 = out1 + tile_off;
+            __half* const t2 = out2 + tile_off;
             const int pairs = cur.ncols >> 1;
-            for (int r = warp; r < cur.nr; r += kCropConsumerWarps) {
-                const RowInfo ri = s_row[b][r];
-                const size_t o = tile_off + (size_t)(r * ow);
-                if (ri.wy != 0.0f)
-                    sample_row<true, false>(rows + (uint32_t)ri.row0, (uint32_t)ri.step, ri.wx, ri.wy, xt, pairs, lane,
-                                            out0 + o, out1 + o, out2 + o, 0.0f);
-                else
-                    sample_row<false, false>(rows + (uint32_t)ri.row0, (uint32_t)ri.step, ri.wx, ri.wy, xt, pairs, lane,
-                                             out0 + o, out1 + o, out2 + o, 0.0f);
+            const int npairs = cur.nr * pairs;
+            const float inv_pairs = 1.0f / (float)pairs;
+            for (int idx = threadIdx.x; idx < npairs; idx += 32 * kCropConsumerWarps) {
+                int r = __float2int_rz(__int2float_rn(idx) * inv_pairs);
+                int pair = idx - r * pairs;
+                if (pair >= pairs) { pair -= pairs; ++r; }
+                else if (pair < 0) { pair += pairs; --r; }
+                const uint4 rw = lds128(rinfo + 16u * (uint32_t)r);
+                const uint4 ee = lds128(xt + 16u * (uint32_t)pair);
+                const float wx = __uint_as_float(rw.z), wy = __uint_as_float(rw.w);
+                float a0, a1, a2, b0, b1, b2;
+                if (wy != 0.0f) {
+                    sample_px<true>(rows + rw.x, rw.y, ee.x, ee.y, wx, wy, a0, a1, a2);
+                    sample_px<true>(rows + rw.x, rw.y, ee.z, ee.w, wx, wy, b0, b1, b2);
+                } else {
+                    sample_px<false>(rows + rw.x, rw.y, ee.x, ee.y, wx, wy, a0, a1, a2);
+                    sample_px<false>(rows + rw.x, rw.y, ee.z, ee.w, wx, wy, b0, b1, b2);
+                }
+                const uint32_t o = (uint32_t)(r * ow + 2 * pair);
+                *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(a0, b0);
+                *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(a1, b1);
+                *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(a2, b2);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[b]);  // this warp is done with ring slot b
