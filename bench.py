@@ -1,5 +1,5 @@
 #!/usr/bin/env python
-"""Benchmark of the cascade-stage hot path (letterbox -> decode/NMS -> assemble -> crop).
+"""Benchmark of the cascade-stage hot path (letterbox -> decode -> NMS -> assemble + crop).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload sweep] [--batch 256]
     python bench.py --impl reference ...        # the CPU oracle on the host cores
@@ -42,11 +42,11 @@ NCU_TRAFFIC = {
     # kernel: (source files, sha256[:16] of their concatenation at capture time, bytes per unit, unit)
     # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md)
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "8f85268299fbeb73", 498201.0, "crop"),
+             "e242c302f30bc941", 493304.0, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                  "e18d17f81bd349de", 3705548.0, "frame"),
+                  "b85159dddf9a967d", 3692384.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "14bf76fbde1bde9e", 3295584.0, "frame"),
+               "c2b06f79f1b032c4", 1697652.0, "frame"),
 }
 
 
