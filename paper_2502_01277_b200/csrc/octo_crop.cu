@@ -19,7 +19,7 @@
 // an exact integer two-way dot product per channel, the vertical lerp and all scaling are two
 // fp32 operations, and a warp writes up to 128 contiguous bytes per plane straight into the
 // downstream slot.  Measured: large passes matter more than occupancy (2 x 32 KB buffers at
-// 3 CTAs/SM beat 2 x 24 KB at 4 and 4 x 12 KB at 4).
+// 3 CTAs/SM beat 2 x 24 KB at 4, 3 x 22 KB at 3 and 4 x 12 KB at 4).
 #include "octo_common.cuh"
 #include "octo_kernels.h"
 
@@ -29,7 +29,8 @@ namespace octo {
 // segment longer than kCropMaxStride - 16 bytes (a rectangle wider than about 5300 pixels)
 // is split into column tiles, so one row pair always fits.  Two buffers form a ring between
 // the producer warp and the consumer warps.
-constexpr int kCropRowBudget = 32768;
+constexpr int kCropStages = 2;         // ring depth (row buffers and tap tables)
+constexpr int kCropRowBudget = 32768;  // bytes per ring buffer
 constexpr int kCropMaxStride = kCropRowBudget / 2;
 constexpr int kCropTilePx = 5300;
 constexpr int kCropMaxPassRows = 32;
@@ -53,13 +54,13 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             int* __restrict__ offsets, int* __restrict__ n_items, octo_item_t* __restrict__ items,
             __half* __restrict__ out, int ow, int oh, int band_rows, int swap_rb, StageCounters* __restrict__ ctr) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t full[2], empty[2];
-    __shared__ CropPass s_pass[2];
-    __shared__ __align__(16) RowInfo s_row[2][kCropMaxPassRows];  // per-row data of the staged passes
+    __shared__ __align__(8) uint64_t full[kCropStages], empty[kCropStages];
+    __shared__ CropPass s_pass[kCropStages];
+    __shared__ __align__(16) RowInfo s_row[kCropStages][kCropMaxPassRows];  // per-row data of the staged passes
     __shared__ int s_off[CAP + 1];                                // exclusive scan of the frame counts
 
     unsigned char* const s_rows0 = smem;
-    XEntry* const s_xtab0 = reinterpret_cast<XEntry*>(smem + 2 * kCropRowBudget);  // two tables of ow entries
+    XEntry* const s_xtab0 = reinterpret_cast<XEntry*>(smem + kCropStages * kCropRowBudget);  // kCropStages tables of ow entries
     unsigned int* const status = &ctr->status;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -82,10 +83,10 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         if (lane == 0) s_off[n] = run;
     }
     if (threadIdx.x == 0) {
-        mbar_init(&full[0], 1);
-        mbar_init(&full[1], 1);
-        mbar_init(&empty[0], kCropConsumerWarps);
-        mbar_init(&empty[1], kCropConsumerWarps);
+        for (int b = 0; b < kCropStages; ++b) {
+            mbar_init(&full[b], 1);
+            mbar_init(&empty[b], kCropConsumerWarps);
+        }
         mbar_fence_init();
     }
     __syncthreads();
@@ -215,23 +216,25 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         };
 
         open_tile();
-        uint32_t ephase[2] = {0u, 0u};
-        int tb = 1;
+        uint32_t ephase = 0u;  // bit b: parity of empty[b] to wait for
+        int tb = kCropStages - 1;
         for (int k = 0;; ++k) {
-            const int b = k & 1;
-            if (k >= 2) {
+            const int b = k % kCropStages;
+            if (k >= kCropStages) {
+                const uint32_t par = (ephase >> b) & 1u;
                 // the consumers have finished the pass that used ring slot b
-                if (!mbar_wait_bounded(&empty[b], ephase[b]) && !mbar_wait_bounded(&empty[b], ephase[b])) {
+                if (!mbar_wait_bounded(&empty[b], par) && !mbar_wait_bounded(&empty[b], par)) {
                     if (lane == 0) atomicOr(status, 0x4u);
                     break;
                 }
-                ephase[b] ^= 1u;
+                ephase ^= 1u << b;
             }
             if (w_valid && w_new) {
                 // taps of every output column: byte offset inside a frame row + integer weights.
-                // The other table is still in use by at most the previous pass; this one was last
-                // used two tiles ago, i.e. by passes the wait above has seen finished.
-                tb ^= 1;
+                // Tables rotate with the tiles: this one belonged to the tile kCropStages tiles
+                // back, all of whose passes the wait above has seen finished (every tile in
+                // between has at least one pass).
+                tb = (tb + 1) % kCropStages;
                 XEntry* const xt = s_xtab0 + (size_t)tb * ow;
                 for (int dx = lane; dx < ow; dx += 32) xt[dx] = make_xentry(dx, w_cw, ow, inv_dx, 3 * w_rx0);
             }
@@ -280,14 +283,15 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         __half* const out0 = out + (swap_rb ? 2 : 0) * plane;  // plane of input channel 0
         __half* const out1 = out + plane;
         __half* const out2 = out + (swap_rb ? 0 : 2) * plane;  // plane of input channel 2
-        uint32_t fphase[2] = {0u, 0u};
+        uint32_t fphase = 0u;  // bit b: parity of full[b] to wait for
         for (int k = 0;; ++k) {
-            const int b = k & 1;
-            if (!mbar_wait_bounded(&full[b], fphase[b]) && !mbar_wait_bounded(&full[b], fphase[b])) {
+            const int b = k % kCropStages;
+            const uint32_t par = (fphase >> b) & 1u;
+            if (!mbar_wait_bounded(&full[b], par) && !mbar_wait_bounded(&full[b], par)) {
                 if (lane == 0) atomicOr(status, 0x4u);
                 break;
             }
-            fphase[b] ^= 1u;
+            fphase ^= 1u << b;
             const CropPass cur = s_pass[b];
             if (!cur.valid) break;
             // flat list of pixel pairs (row-major); thread t of the consumers owns pairs t, t+256, ...
@@ -346,7 +350,7 @@ static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     long long work = (long long)a.max_items * bands;
     int grid = (int)(work < cap ? work : cap);
     if (grid < 1) grid = 1;  // a zero-slot window still gets its offsets and totals
-    const size_t smem = 2 * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w);
+    const size_t smem = (size_t)kCropStages * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w);
     crop_kernel<CAP><<<grid, kCropKernelThreads, smem, stream>>>(
         tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
         a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, band_rows, a.swap_rb, a.d_ctr);
@@ -354,7 +358,7 @@ static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
 }
 
 cudaError_t prepare_crop() {
-    const int smem = 2 * (kCropRowBudget + (int)sizeof(XEntry) * 2048);
+    const int smem = kCropStages * (kCropRowBudget + (int)sizeof(XEntry) * 2048);
     cudaError_t e;
     e = cudaFuncSetAttribute(crop_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
