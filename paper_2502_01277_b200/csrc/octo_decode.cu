@@ -14,8 +14,6 @@
 namespace octo {
 
 constexpr int kDecThreads = 256;
-constexpr int kDecPerThread = 4;  // anchors per thread
-constexpr int kDecPerCta = kDecThreads * kDecPerThread;
 
 // Read-only load that asks L2 to fetch 64 bytes around the address instead of the default
 // 128: the obj scan touches 4 bytes per 340-byte row, so the smaller fill granularity cuts
@@ -26,6 +24,9 @@ __device__ __forceinline__ float ld_obj(const float* p) {
     return v;
 }
 
+// kDecPerThread anchors per thread: 4 for large batches, 1 when the grid would otherwise be
+// too small to cover the SMs.
+template <int kDecPerThread>
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(const float* __restrict__ head, int A, int C, int logits, float conf, int key_stride,
               unsigned long long* __restrict__ keys, int* __restrict__ cand_count,
@@ -36,7 +37,7 @@ decode_kernel(const float* __restrict__ head, int A, int C, int logits, float co
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     // each warp owns kDecPerThread consecutive groups of 32 anchors
-    const int a_warp = blockIdx.x * kDecPerCta + warp * (32 * kDecPerThread);
+    const int a_warp = blockIdx.x * (kDecThreads * kDecPerThread) + warp * (32 * kDecPerThread);
 
     float obj[kDecPerThread];
 #pragma unroll
@@ -109,9 +110,16 @@ cudaError_t launch_decode(const float* d_head, int n, int A, int C, int logits, 
                           unsigned long long* d_keys, int* d_cand_count, unsigned int* d_status,
                           cudaStream_t stream) {
     // d_cand_count is zero on entry: zeroed at stage creation and re-zeroed by the NMS kernel.
-    dim3 grid((A + kDecPerCta - 1) / kDecPerCta, n);
-    decode_kernel<<<grid, kDecThreads, 0, stream>>>(d_head, A, C, logits, conf, key_stride, d_keys, d_cand_count,
-                                                   d_status);
+    const int per_cta4 = kDecThreads * 4;
+    if ((long long)n * ((A + per_cta4 - 1) / per_cta4) >= 296) {
+        dim3 grid((A + per_cta4 - 1) / per_cta4, n);
+        decode_kernel<4><<<grid, kDecThreads, 0, stream>>>(d_head, A, C, logits, conf, key_stride, d_keys,
+                                                          d_cand_count, d_status);
+    } else {
+        dim3 grid((A + kDecThreads - 1) / kDecThreads, n);
+        decode_kernel<1><<<grid, kDecThreads, 0, stream>>>(d_head, A, C, logits, conf, key_stride, d_keys,
+                                                          d_cand_count, d_status);
+    }
     return cudaGetLastError();
 }
 

@@ -157,6 +157,8 @@ static cudaError_t launch_cap(const FrameDesc* frames, int n, void* d_out, int S
     const long long room = 56 * 1024 - (long long)lb_smem_bytes(S, 0, slot_bytes);
     int band_rows = (int)(room / per_row);
     band_rows = band_rows < 1 ? 1 : (band_rows > kLbRows ? kLbRows : band_rows);
+    // small batches: fewer rows per CTA so that the grid still covers the SMs about twice
+    while (band_rows > 2 && (long long)n * ((S + band_rows - 1) / band_rows) < 296) band_rows >>= 1;
     const size_t smem = lb_smem_bytes(S, band_rows * slots_per_row(frames, n), slot_bytes);
     const __half hf = __double2half((double)pad_value / 255.0);  // one rounding, nearest even
     const uint32_t fb = *reinterpret_cast<const unsigned short*>(&hf);
