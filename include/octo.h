@@ -150,6 +150,32 @@ OCTO_API int octo_stage_destroy(octo_stage_t* st);
 OCTO_API int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frames, int32_t n,
                           void* d_out_f16_nchw, void* cuda_stream);
 
+/* One input of a chained (second-level) stage: the rectangle [rx0, rx1) x [ry0, ry1) of a source
+ * frame, as reported in an upstream stage's item table. */
+typedef struct {
+    const uint8_t* d_data;                 /* the ORIGINAL frame (same rules as octo_frame_t) */
+    int32_t width, height, pitch_bytes;
+    int32_t rx0, ry0, rx1, ry1;
+    int32_t _pad;
+} octo_region_t;
+
+/*
+ * Chained stage (the paper's cascades continue below the first detector, e.g. vehicle crop ->
+ * plate detector, person crop -> face detector; Section I and Section III-B, Observation 1).
+ * Declares that this stage's current batch consists of n regions which an upstream stage has
+ * already cropped and stretched to net_size x net_size: the upstream octo_crop_batch output
+ * (a branch with out_w = out_h = net_size) IS this stage's detector input, so no kernel runs
+ * here.  The call records the table that the next octo_postprocess_batch and octo_crop_batch
+ * use: head boxes, given on the net_size x net_size grid, are mapped back into the rectangle of
+ * the original frame, X = rx0 + x * fl((rx1 - rx0) / net_size), clamped to the rectangle, and
+ * this stage's own crops are resampled from the original frame pixels.
+ *   regions  host array of n entries, normally filled from octo_stage_copy_items of the
+ *            upstream stage plus that stage's frame descriptors.
+ * Errors: OCTO_E_INVALID_ARG (null, n < 1, rectangle empty or outside its frame, pitch < 3 *
+ * width), OCTO_E_CAPACITY (n > max_batch), OCTO_E_ALIGNMENT.
+ */
+OCTO_API int octo_adopt_regions(octo_stage_t* st, const octo_region_t* regions, int32_t n, void* cuda_stream);
+
 /*
  * Decode the detector head of the batch last given to octo_preprocess_batch (n must match)
  * into detections (stage output Out_m of Table II; the per-frame count is what drives the

@@ -7,6 +7,6 @@ the CUDA package, and it imports nothing from it.
 """
 from .oracle import (  # noqa: F401
     DET_DTYPE, build, letterbox_geometry, resize_f64, f64_to_half, letterbox, sigmoid,
-    decode, sort_candidates, iou, nms, scale_back, postprocess_image, crop_rect, crop,
+    decode, sort_candidates, iou, nms, scale_back, postprocess_image, postprocess_region, crop_rect, crop,
     assemble, StageResult, run_stage,
 )

@@ -252,19 +252,29 @@ int32_t orc_nms(const orc_det_t* c, int32_t n, float thr, int32_t max_det, int32
     return k;
 }
 
-/* R6: letterbox pixels -> frame pixels in binary32: X = fl(fl(x - pad) * g), g = fl(w / nw),
- * clamped to [0, w] (and [0, h]). */
+/* R6: detector-input pixels -> source-frame pixels in binary32.  The detector input shows a
+ * region [ox, ox+rw) x [oy, oy+rh) of the source frame (the whole frame for a first-level
+ * stage; the upstream crop rectangle for a chained stage), scaled to nw x nh and placed at
+ * (pad_l, pad_t) on the canvas:  X = fl(fl(fl(x - pad_l) * g) + ox), g = fl(rw / nw), clamped
+ * to [ox, ox + rw]; likewise in y.  With ox = 0 the last addition changes nothing. */
+void orc_scale_back_region(orc_det_t* d, int32_t nw, int32_t nh, int32_t pad_l, int32_t pad_t,
+                           int32_t ox, int32_t oy, int32_t rw, int32_t rh) {
+    float gx = (float)rw / (float)nw, gy = (float)rh / (float)nh;
+    float fpl = (float)pad_l, fpt = (float)pad_t;
+    float xlo = (float)ox, ylo = (float)oy, xhi = (float)(ox + rw), yhi = (float)(oy + rh);
+    float X1 = (d->x1 - fpl) * gx + xlo, X2 = (d->x2 - fpl) * gx + xlo;
+    float Y1 = (d->y1 - fpt) * gy + ylo, Y2 = (d->y2 - fpt) * gy + ylo;
+    d->x1 = fminf(fmaxf(X1, xlo), xhi);
+    d->x2 = fminf(fmaxf(X2, xlo), xhi);
+    d->y1 = fminf(fmaxf(Y1, ylo), yhi);
+    d->y2 = fminf(fmaxf(Y2, ylo), yhi);
+}
+
+/* R6 for a first-level stage: the region is the whole w x h frame, letterboxed by R1. */
 void orc_scale_back(orc_det_t* d, int32_t w, int32_t h, int32_t S) {
     int32_t nw, nh, pl, pt;
     orc_letterbox_geometry(w, h, S, &nw, &nh, &pl, &pt);
-    float gx = (float)w / (float)nw, gy = (float)h / (float)nh;
-    float fw = (float)w, fh = (float)h, fpl = (float)pl, fpt = (float)pt;
-    float X1 = (d->x1 - fpl) * gx, X2 = (d->x2 - fpl) * gx;
-    float Y1 = (d->y1 - fpt) * gy, Y2 = (d->y2 - fpt) * gy;
-    d->x1 = fminf(fmaxf(X1, 0.0f), fw);
-    d->x2 = fminf(fmaxf(X2, 0.0f), fw);
-    d->y1 = fminf(fmaxf(Y1, 0.0f), fh);
-    d->y2 = fminf(fmaxf(Y2, 0.0f), fh);
+    orc_scale_back_region(d, nw, nh, pl, pt, 0, 0, w, h);
 }
 
 /* R3..R6 for one image: head -> dets[<= max_det] in frame pixels.  Returns kept count;
@@ -280,6 +290,27 @@ int32_t orc_postprocess_image(const float* head, int32_t A, int32_t C, int32_t l
     for (int32_t t = 0; t < k; ++t) {
         dets[t] = cand[keep[t]];
         orc_scale_back(&dets[t], w, h, S);
+    }
+    if (n_cand) *n_cand = n;
+    free(cand);
+    free(keep);
+    return k;
+}
+
+/* R3..R6 for one item of a chained (second-level) stage.  Its detector input is the upstream
+ * crop of the rectangle [ox, ox+rw) x [oy, oy+rh), stretched to S x S (no padding), so the
+ * head's boxes live on that S x S grid and map back into the rectangle of the ORIGINAL frame. */
+int32_t orc_postprocess_region(const float* head, int32_t A, int32_t C, int32_t logits, float conf,
+                               float iou_thr, int32_t max_det, int32_t S, int32_t ox, int32_t oy,
+                               int32_t rw, int32_t rh, orc_det_t* dets, int32_t* n_cand) {
+    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * (size_t)(A > 0 ? A : 1));
+    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
+    int32_t n = orc_decode(head, A, C, logits, conf, cand);
+    orc_sort(cand, n);
+    int32_t k = orc_nms(cand, n, iou_thr, max_det, keep);
+    for (int32_t t = 0; t < k; ++t) {
+        dets[t] = cand[keep[t]];
+        orc_scale_back_region(&dets[t], S, S, 0, 0, ox, oy, rw, rh);
     }
     if (n_cand) *n_cand = n;
     free(cand);

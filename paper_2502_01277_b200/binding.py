@@ -41,6 +41,7 @@ EXPORTS = (
     "octo_stage_item_table", "octo_stage_copy_items", "octo_stage_set_timing", "octo_stage_kernel_times",
     "octo_stage_workspace_bytes", "octo_stage_launch_count",
     "octo_strerror", "octo_last_cuda_error", "octo_version", "octo_postprocess_frame_static",
+    "octo_adopt_regions",
 )
 
 
@@ -62,6 +63,12 @@ class StageConfig(ctypes.Structure):
 class Frame(ctypes.Structure):
     _fields_ = [("d_data", ctypes.c_void_p), ("width", ctypes.c_int32), ("height", ctypes.c_int32),
                 ("pitch_bytes", ctypes.c_int32), ("_pad", ctypes.c_int32)]
+
+
+class Region(ctypes.Structure):
+    _fields_ = [("d_data", ctypes.c_void_p), ("width", ctypes.c_int32), ("height", ctypes.c_int32),
+                ("pitch_bytes", ctypes.c_int32), ("rx0", ctypes.c_int32), ("ry0", ctypes.c_int32),
+                ("rx1", ctypes.c_int32), ("ry1", ctypes.c_int32), ("_pad", ctypes.c_int32)]
 
 
 class StageStats(ctypes.Structure):
@@ -112,6 +119,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_stage_destroy.argtypes = [vp]
     lib.octo_preprocess_batch.argtypes = [vp, ctypes.POINTER(Frame), i32, vp, vp]
     lib.octo_postprocess_batch.argtypes = [vp, vp, i32, vp, vp, vp]
+    lib.octo_adopt_regions.argtypes = [vp, ctypes.POINTER(Region), i32, vp]
+    lib.octo_adopt_regions.restype = ctypes.c_int
     lib.octo_crop_batch.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.octo_stage_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     lib.octo_stage_clear_status.argtypes = [vp, vp]
@@ -289,6 +298,23 @@ class Stage:
             self._frames_keepalive = keepalive
         self.n = n
         return out
+
+    def adopt_regions(self, frames, sizes, items, stream=None):
+        """Chained stage: this batch = the upstream items (ITEM_DTYPE records: frame index +
+        rectangle) of the upstream frames (CUDA tensors [h, pitch]) with their (w, h) sizes."""
+        n = len(items)
+        arr = (Region * max(n, 1))()
+        for i, it in enumerate(items):
+            f = frames[int(it["frame"])]
+            w, h = sizes[int(it["frame"])]
+            arr[i].d_data, arr[i].width, arr[i].height, arr[i].pitch_bytes = f.data_ptr(), w, h, f.stride(0)
+            arr[i].rx0, arr[i].ry0, arr[i].rx1, arr[i].ry1 = (int(it["rx0"]), int(it["ry0"]), int(it["rx1"]),
+                                                              int(it["ry1"]))
+        rc = load_library().octo_adopt_regions(self.handle, arr, n, self._stream(stream))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_adopt_regions")
+        self._frames_keepalive = list(frames)
+        self.n = n
 
     def postprocess(self, head, dets=None, counts=None, stream=None):
         """head: float32 CUDA tensor [n, A, 5+C].  Returns (dets uint8 [n, max_det, 32], counts int32 [n])."""

@@ -14,10 +14,13 @@ struct FrameDesc {
     const uint8_t* data;
     int32_t w, h, pitch;
     int32_t nw, nh, pad_l, pad_t;
-    float gx, gy;  // fl(w / nw), fl(h / nh): scale-back gains
-    int32_t _pad;
+    float gx, gy;  // fl(region width / nw), fl(region height / nh): scale-back gains
+    // Region of the source frame that the detector input shows: the whole frame for a
+    // first-level stage, the upstream crop rectangle for a chained stage.  Boxes are mapped
+    // back into it and clamped to it.
+    uint16_t ox, oy, rw, rh;
 };
-static_assert(sizeof(FrameDesc) == 48, "FrameDesc layout");
+static_assert(sizeof(FrameDesc) == 56, "FrameDesc layout");
 
 template <int CAP>
 struct FrameTable {

@@ -308,7 +308,10 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
     __syncthreads();
 
     const FrameDesc& fd = tab.f[img];
-    const float fw = (float)fd.w, fh = (float)fd.h, fpl = (float)fd.pad_l, fpt = (float)fd.pad_t;
+    // region of the source frame shown by the detector input: x in [x_lo, x_hi], y likewise
+    const float fpl = (float)fd.pad_l, fpt = (float)fd.pad_t;
+    const float x_lo = (float)fd.ox, y_lo = (float)fd.oy;
+    const float x_hi = (float)(fd.ox + fd.rw), y_hi = (float)(fd.oy + fd.rh);
     for (int r = threadIdx.x; r < nout; r += kNmsThreads) {
         const unsigned long long g = ordered[r];
         const int cls = (int)(g & 127u);
@@ -316,10 +319,11 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
         const float score = __uint_as_float(~(unsigned)(g >> 32));
         const float4 b = gather_box(hbase + (size_t)anchor * row_len);
         octo_det_rec d;
-        d.x1 = fminf(fmaxf(__fmul_rn(__fsub_rn(b.x, fpl), fd.gx), 0.0f), fw);
-        d.y1 = fminf(fmaxf(__fmul_rn(__fsub_rn(b.y, fpt), fd.gy), 0.0f), fh);
-        d.x2 = fminf(fmaxf(__fmul_rn(__fsub_rn(b.z, fpl), fd.gx), 0.0f), fw);
-        d.y2 = fminf(fmaxf(__fmul_rn(__fsub_rn(b.w, fpt), fd.gy), 0.0f), fh);
+        // X = fl(fl(fl(x - pad) * gain) + origin), clamped to the region
+        d.x1 = fminf(fmaxf(__fadd_rn(__fmul_rn(__fsub_rn(b.x, fpl), fd.gx), x_lo), x_lo), x_hi);
+        d.y1 = fminf(fmaxf(__fadd_rn(__fmul_rn(__fsub_rn(b.y, fpt), fd.gy), y_lo), y_lo), y_hi);
+        d.x2 = fminf(fmaxf(__fadd_rn(__fmul_rn(__fsub_rn(b.z, fpl), fd.gx), x_lo), x_lo), x_hi);
+        d.y2 = fminf(fmaxf(__fadd_rn(__fmul_rn(__fsub_rn(b.w, fpt), fd.gy), y_lo), y_lo), y_hi);
         d.score = score;
         d.cls = cls;
         d.anchor = anchor;

@@ -86,7 +86,10 @@ void frame_geometry(int w, int h, int S, FrameDesc* fd) {
     fd->pad_t = (int)((S - nh) / 2);
     fd->gx = (float)w / (float)fd->nw;
     fd->gy = (float)h / (float)fd->nh;
-    fd->_pad = 0;
+    fd->ox = 0;
+    fd->oy = 0;
+    fd->rw = (uint16_t)w;
+    fd->rh = (uint16_t)h;
 }
 
 }  // namespace

@@ -183,6 +183,10 @@ static void letterbox_geometry(int w, int h, int S, FrameDesc* fd) {
     fd->pad_t = (int)((S - nh) / 2);
     fd->gx = (float)w / (float)fd->nw;
     fd->gy = (float)h / (float)fd->nh;
+    fd->ox = 0;
+    fd->oy = 0;
+    fd->rw = (uint16_t)w;
+    fd->rh = (uint16_t)h;
 }
 
 extern "C" int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frames, int32_t n,
@@ -208,7 +212,6 @@ extern "C" int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frame
         fd.w = frames[i].width;
         fd.h = frames[i].height;
         fd.pitch = frames[i].pitch_bytes;
-        fd._pad = 0;
         letterbox_geometry(fd.w, fd.h, st->cfg.net_size, &fd);
     }
     st->max_w = max_w;
@@ -219,6 +222,45 @@ extern "C" int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frame
                                    st->cfg.swap_rb, &st->d_ctr->status, static_cast<cudaStream_t>(cuda_stream)));
     }
     st->launches += 1;
+    st->n_frames = n;
+    return OCTO_OK;
+}
+
+extern "C" int octo_adopt_regions(octo_stage_t* st, const octo_region_t* regions, int32_t n, void* cuda_stream) {
+    (void)cuda_stream;  // nothing is enqueued: the table travels with the next kernel launches
+    if (!st || !regions || n < 1) return OCTO_E_INVALID_ARG;
+    if (n > st->cfg.max_batch) return OCTO_E_CAPACITY;
+    const int S = st->cfg.net_size;
+    for (int i = 0; i < n; ++i) {
+        const octo_region_t& r = regions[i];
+        if (!r.d_data || r.width < 1 || r.height < 1) return OCTO_E_INVALID_ARG;
+        if (r.width > 16384 || r.height > 16384) return OCTO_E_CAPACITY;
+        if ((long long)r.pitch_bytes < 3LL * r.width) return OCTO_E_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(r.d_data) & 15) || (r.pitch_bytes & 15)) return OCTO_E_ALIGNMENT;
+        if (r.rx0 < 0 || r.ry0 < 0 || r.rx1 <= r.rx0 || r.ry1 <= r.ry0 || r.rx1 > r.width || r.ry1 > r.height)
+            return OCTO_E_INVALID_ARG;
+    }
+    st->n_frames = 0;
+    st->have_dets = false;
+    for (int i = 0; i < n; ++i) {
+        const octo_region_t& r = regions[i];
+        FrameDesc& fd = st->frames[i];
+        fd.data = r.d_data;
+        fd.w = r.width;
+        fd.h = r.height;
+        fd.pitch = r.pitch_bytes;
+        fd.nw = S;  // the upstream crop is a plain stretch to S x S: no padding
+        fd.nh = S;
+        fd.pad_l = 0;
+        fd.pad_t = 0;
+        fd.ox = (uint16_t)r.rx0;
+        fd.oy = (uint16_t)r.ry0;
+        fd.rw = (uint16_t)(r.rx1 - r.rx0);
+        fd.rh = (uint16_t)(r.ry1 - r.ry0);
+        fd.gx = (float)(r.rx1 - r.rx0) / (float)S;
+        fd.gy = (float)(r.ry1 - r.ry0) / (float)S;
+    }
+    st->max_w = 0;
     st->n_frames = n;
     return OCTO_OK;
 }

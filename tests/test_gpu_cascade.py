@@ -1,0 +1,115 @@
+"""Second-level cascade on the GPU against the oracle: a first-level detector stage crops its
+survivors to 256x256 (the plate-detector branch of the traffic pipeline); a chained stage
+adopts those crops as its detector input, decodes its own synthetic head, maps the boxes back
+into the ORIGINAL frame through the upstream rectangles and crops again from the original
+pixels.  Indices, counts, packing, rectangles, scores and box coordinates must be bit-exact;
+fp16 pixels within 2e-3."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2502_01277_b200 as octo
+import workloads
+from gpu_harness import half_absdiff
+from oracle import DET_DTYPE
+
+pytestmark = pytest.mark.gpu
+
+
+def test_two_level_cascade_matches_oracle():
+    wl = replace(workloads.WORKLOADS["traffic_1080p"], branches=((256, 256),))
+    b = workloads.make_batch(wl, batch=3, seed=31)
+    s2, c2, max_det2 = 256, 6, 12
+    a2 = workloads.num_anchors(s2)
+    # ---- level 1 on the GPU
+    st1 = octo.Stage(net_size=wl.net_size, max_batch=b.n, num_anchors=wl.num_anchors, num_classes=wl.num_classes,
+                     max_det=wl.max_det, branches=wl.branches)
+    st2 = None
+    try:
+        frames = [torch.from_numpy(f).cuda() for f in b.frames]
+        st1.preprocess(frames, b.sizes)
+        st1.postprocess(torch.from_numpy(b.head).cuda())
+        crops1, off1, ni1 = st1.crop(0, 256)
+        torch.cuda.synchronize()
+        n1 = int(ni1[0])
+        items1 = st1.item_table(0, n1)
+        ref1 = oracle.run_stage(b.frames, b.sizes, b.head, wl.net_size, wl.branches, max_det=wl.max_det,
+                                do_letterbox=False)
+        assert n1 == len(ref1.items[0]) and n1 > 20
+        assert np.array_equal(np.stack([items1["rx0"], items1["ry0"], items1["rx1"], items1["ry1"]], 1),
+                              ref1.rects[0])
+        # ---- level 2: the 256x256 crops are the detector input; heads are synthetic
+        head2 = workloads.make_heads(77, n1, s2, num_classes=c2, n_raised=14, n_groups=4)
+        st2 = octo.Stage(net_size=s2, max_batch=n1, num_anchors=a2, num_classes=c2, max_det=max_det2,
+                         branches=((64, 32),))
+        st2.adopt_regions(frames, b.sizes, items1)
+        dets2, counts2 = st2.postprocess(torch.from_numpy(head2).cuda())
+        cap2 = n1 * max_det2
+        buf = torch.full((cap2, 3, 32, 64), 0x7BFF, dtype=torch.int16, device="cuda")
+        _, off2, ni2 = st2.crop(0, cap2, out=buf.view(torch.float16))
+        torch.cuda.synchronize()
+        d2, c2n = octo.dets_to_numpy(dets2, counts2)
+        packed2, total2 = (int(v) for v in ni2.cpu())
+        items2 = st2.item_table(0, packed2)
+        got = buf.cpu().numpy().view(np.uint16)
+        assert st2.status() == 0
+        # ---- oracle chain
+        ref_d = np.zeros((n1, max_det2), dtype=DET_DTYPE)
+        ref_c = np.zeros(n1, dtype=np.int32)
+        for i in range(n1):
+            r = ref1.rects[0][i]
+            d, _ = oracle.postprocess_region(head2[i], tuple(int(v) for v in r), s2, max_det=max_det2)
+            ref_d[i, : len(d)] = d
+            ref_c[i] = len(d)
+        assert np.array_equal(c2n, ref_c) and int(ref_c.sum()) > n1
+        for i in range(n1):
+            k = ref_c[i]
+            assert d2[i, :k].tobytes() == ref_d[i, :k].tobytes(), f"item {i}: detections differ"
+            rx0, ry0, rx1, ry1 = ref1.rects[0][i]
+            assert np.all((ref_d[i, :k]["x1"] >= rx0) & (ref_d[i, :k]["x2"] <= rx1))
+            assert np.all((ref_d[i, :k]["y1"] >= ry0) & (ref_d[i, :k]["y2"] <= ry1))
+        offs, its, (pk, tot) = oracle.assemble(ref_d, ref_c, max_det2)
+        assert (packed2, total2) == (pk, tot) and np.array_equal(off2.cpu().numpy(), offs)
+        assert np.array_equal(np.stack([items2["frame"], items2["det"]], 1), its)
+        for k, (i, j) in enumerate(its):
+            f = int(items1["frame"][i])  # the ORIGINAL frame behind upstream item i
+            w, h = b.sizes[f]
+            rect = oracle.crop_rect(ref_d[i, j], w, h)
+            assert (int(items2["rx0"][k]), int(items2["ry0"][k]), int(items2["rx1"][k]), int(items2["ry1"][k])) == rect
+            want = oracle.crop(b.frames[f], w, h, ref_d[i, j], 64, 32)
+            assert half_absdiff(got[k], want) <= 2e-3
+        assert np.all(got[packed2:] == 0x7BFF)
+    finally:
+        st1.close()
+        if st2 is not None:
+            st2.close()
+
+
+def test_adopt_regions_argument_errors():
+    from paper_2502_01277_b200 import binding as B
+    st = octo.Stage(net_size=64, max_batch=2, num_anchors=252, num_classes=4, max_det=10, branches=((16, 16),))
+    try:
+        f = torch.zeros((30, 128), dtype=torch.uint8, device="cuda")
+        lib = octo.load_library()
+
+        def call(rects, n=None):
+            arr = (B.Region * max(len(rects), 1))()
+            for i, (ptr, w, h, p, r) in enumerate(rects):
+                arr[i].d_data, arr[i].width, arr[i].height, arr[i].pitch_bytes = ptr, w, h, p
+                arr[i].rx0, arr[i].ry0, arr[i].rx1, arr[i].ry1 = r
+            return lib.octo_adopt_regions(st.handle, arr, len(rects) if n is None else n, None)
+
+        ok = (f.data_ptr(), 40, 30, 128, (2, 3, 20, 25))
+        assert call([ok]) == B.OCTO_OK
+        assert call([ok], n=0) == B.OCTO_E_INVALID_ARG
+        assert call([ok] * 3) == B.OCTO_E_CAPACITY
+        assert call([(f.data_ptr(), 40, 30, 128, (5, 3, 5, 25))]) == B.OCTO_E_INVALID_ARG   # empty
+        assert call([(f.data_ptr(), 40, 30, 128, (5, 3, 41, 25))]) == B.OCTO_E_INVALID_ARG  # outside the frame
+        assert call([(f.data_ptr(), 40, 30, 112, (2, 3, 20, 25))]) == B.OCTO_E_INVALID_ARG  # pitch < 3 w
+        assert call([(f.data_ptr() + 4, 40, 30, 128, (2, 3, 20, 25))]) == B.OCTO_E_ALIGNMENT
+        assert call([(0, 40, 30, 128, (2, 3, 20, 25))]) == B.OCTO_E_INVALID_ARG
+    finally:
+        st.close()

@@ -358,3 +358,22 @@ def test_scale_back_portrait_and_inexact_gain():
             (float(d["x2"][0]) - pl) * 1366 / nw, (float(d["y2"][0]) - pt) * 768 / nh]
     got = [float(out[k]) for k in ("x1", "y1", "x2", "y2")]
     assert np.allclose(got, want, rtol=1e-6)
+
+
+def test_chained_stage_maps_boxes_into_the_upstream_rectangle():
+    """Second-level stage: a 180x180 rectangle at (300, 180) stretched to 256x256; gain 180/256 =
+    0.703125 is a binary32 number, so the hand values are exact."""
+    C = 4
+    head = np.stack([_head_row(C, cx=128, cy=192, w=128, h=128, obj=3.0, cls={2: 3.0}),   # (64,128)-(192,256)
+                     _head_row(C, cx=10, cy=250, w=60, h=40, obj=2.0, cls={1: 2.0})])     # pokes out left / bottom
+    dets, ncand = oracle.postprocess_region(head, (300, 180, 480, 360), 256)
+    assert ncand == 2 and len(dets) == 2
+    a, b = dets[0], dets[1]
+    assert (a["x1"], a["y1"], a["x2"], a["y2"]) == (345.0, 270.0, 435.0, 360.0)
+    # (-20,230)-(40,270) -> x: 300 - 14.06 -> clamped to 300 ; 300 + 28.125 ; y: 180 + 161.71875 ; clamped to 360
+    assert (b["x1"], b["x2"], b["y2"]) == (300.0, 328.125, 360.0)
+    assert float(b["y1"]) == 180.0 + 230 * 0.703125
+    # the region of a first-level stage is the whole frame: same numbers as scale_back
+    d1, _ = oracle.postprocess_image(head, 256, 256, 256)
+    d2, _ = oracle.postprocess_region(head, (0, 0, 256, 256), 256)
+    assert d1.tobytes() == d2.tobytes()

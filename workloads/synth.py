@@ -164,6 +164,22 @@ def make_batch(name_or_workload, batch: Optional[int] = None, first_frame: int =
     return Batch(wl, frames, sizes, head, first_frame)
 
 
+def make_heads(seed: int, n: int, net_size: int, num_classes: int = 80, n_raised: int = 10, n_groups: int = 4,
+               size_range: Tuple[float, float] = (30.0, 120.0), jitter: float = 0.15,
+               scale_range: Tuple[float, float] = (0.8, 1.25), first: int = 0, logits: bool = True) -> np.ndarray:
+    """Heads [n, A, 5 + C] of a chained (second-level) detector whose input is an upstream crop
+    stretched to net_size x net_size: same recipe as the frame heads, boxes anywhere on the grid."""
+    lib = _load()
+    a = num_anchors(net_size)
+    head = np.empty((n, a, 5 + num_classes), dtype=np.float32)
+    f32p = ctypes.POINTER(ctypes.c_float)
+    for i in range(n):
+        lib.wl_head(seed, first + i, net_size, a, num_classes, n_raised, n_groups, 0.0, float(net_size),
+                    size_range[0], size_range[1], jitter, scale_range[0], scale_range[1], -4.0, 2.0, 0.5,
+                    1 if logits else 0, head[i].ctypes.data_as(f32p))
+    return head
+
+
 def shard_range(total: int, rank: int, world: int) -> Tuple[int, int]:
     """Contiguous [begin, end) slice of `total` frames owned by `rank` of `world`."""
     base, rem = divmod(total, world)
