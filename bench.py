@@ -55,7 +55,7 @@ def parse_args():
     p.add_argument("--gpus", type=int, default=1)
     p.add_argument("--steps", type=int, default=30)
     p.add_argument("--warmup", type=int, default=5)
-    p.add_argument("--workload", default="sweep", choices=sorted(workloads.WORKLOADS))
+    p.add_argument("--workload", default="sweep", choices=sorted(workloads.WORKLOADS) + ["two_level"])
     p.add_argument("--batch", type=int, default=None, help="frames per GPU per step")
     p.add_argument("--impl", default="octo", choices=["octo", "reference"])
     p.add_argument("--e2e-steps", type=int, default=None)
@@ -65,6 +65,8 @@ def parse_args():
 
 
 def default_batch(name: str) -> int:
+    if name == "two_level":
+        return 64
     return 256 if name == "sweep" else workloads.WORKLOADS[name].batch
 
 
@@ -198,6 +200,9 @@ def run_reference(args):
     if rank != 0:
         return
     name = args.workload
+    if name == "two_level":
+        print(json.dumps({"impl": "reference", "unavailable": "the reference arm covers the single-stage workloads"}))
+        return
     bsz = args.batch or default_batch(name)
     cores = len(os.sched_getaffinity(0))
     sample = cpu_sample_frames(bsz, cores)
@@ -517,10 +522,113 @@ def run_octo(args):
         dist.destroy_process_group()
 
 
+def run_two_level(args):
+    """Two-level cascade (frames -> detector stage -> 256x256 crops -> chained detector stage ->
+    64x32 crops).  One step = level-1 pass, host hand-off of the item table, level-2 pass.  The
+    hand-off synchronises, as it does between two serving containers.  Single GPU."""
+    import torch
+    from dataclasses import replace
+
+    import paper_2502_01277_b200 as octo
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    n = args.batch or default_batch("two_level")
+    wl = replace(workloads.WORKLOADS["traffic_1080p"], branches=((256, 256),))
+    batch = workloads.make_batch(wl, batch=n, seed=5)
+    s2, c2, max_det2 = 256, 8, 16
+    a2 = workloads.num_anchors(s2)
+    st1 = octo.Stage(net_size=wl.net_size, max_batch=n, num_anchors=wl.num_anchors, num_classes=wl.num_classes,
+                     max_det=wl.max_det, branches=wl.branches)
+    stream = torch.cuda.Stream(dev)
+    cap1 = n * wl.items_per_frame
+    with torch.cuda.stream(stream):
+        frames = [torch.from_numpy(f).to(dev) for f in batch.frames]
+        head1 = torch.from_numpy(batch.head).to(dev)
+        det_in = torch.empty((n, 3, wl.net_size, wl.net_size), dtype=torch.float16, device=dev)
+        dets1 = torch.zeros((n, wl.max_det, 32), dtype=torch.uint8, device=dev)
+        counts1 = torch.zeros((n,), dtype=torch.int32, device=dev)
+        crops1 = torch.empty((cap1, 3, 256, 256), dtype=torch.float16, device=dev)
+        off1 = torch.zeros((n + 1,), dtype=torch.int32, device=dev)
+        ni1 = torch.zeros((2,), dtype=torch.int32, device=dev)
+        desc = st1.frame_array(frames, batch.sizes)
+        # one dry pass to learn the number of level-1 items, which sizes level 2
+        st1.preprocess_array(desc, n, det_in, stream=stream, keepalive=frames)
+        st1.postprocess(head1, dets=dets1, counts=counts1, stream=stream)
+        st1.crop(0, cap1, out=crops1, offsets=off1, n_items=ni1, stream=stream)
+    stream.synchronize()
+    n1 = int(ni1[0])
+    head2_h = workloads.make_heads(9, n1, s2, num_classes=c2, n_raised=12, n_groups=3)
+    st2 = octo.Stage(net_size=s2, max_batch=min(n1, 512), num_anchors=a2, num_classes=c2, max_det=max_det2,
+                     branches=((64, 32),))
+    c2n = min(n1, 512)  # level-2 batches of at most 512 upstream items
+    with torch.cuda.stream(stream):
+        head2 = torch.from_numpy(head2_h).to(dev)
+        dets2 = torch.zeros((c2n, max_det2, 32), dtype=torch.uint8, device=dev)
+        counts2 = torch.zeros((c2n,), dtype=torch.int32, device=dev)
+        crops2 = torch.empty((c2n * max_det2, 3, 32, 64), dtype=torch.float16, device=dev)
+        off2 = torch.zeros((c2n + 1,), dtype=torch.int32, device=dev)
+        ni2 = torch.zeros((2,), dtype=torch.int32, device=dev)
+    items2_total = [0]
+
+    def step(_i):
+        st1.preprocess_array(desc, n, det_in, stream=stream, keepalive=frames)
+        st1.postprocess(head1, dets=dets1, counts=counts1, stream=stream)
+        st1.crop(0, cap1, out=crops1, offsets=off1, n_items=ni1, stream=stream)
+        stream.synchronize()  # hand-off: the downstream stage learns its inputs from the host
+        m = int(ni1[0])
+        items = st1.item_table(0, m)
+        tot = 0
+        for lo in range(0, m, c2n):
+            hi = min(lo + c2n, m)
+            st2.adopt_regions(frames, batch.sizes, items[lo:hi], stream=stream)
+            st2.postprocess(head2[lo:hi], dets=dets2[: hi - lo], counts=counts2[: hi - lo], stream=stream)
+            st2.crop(0, (hi - lo) * max_det2, out=crops2, offsets=off2[: hi - lo + 1], n_items=ni2, stream=stream)
+            tot += hi - lo
+        items2_total[0] = tot
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    l0 = st1.launch_count + st2.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / args.steps
+    launches = st1.launch_count + st2.launch_count - l0
+    clocks = sampler.stop()
+    for st in (st1, st2):
+        if st.status(stream) & ~0xA:
+            raise SystemExit(f"device status word {st.status(stream):#x}")
+    line = {
+        "metric": METRIC, "value": n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"two_level B={n}", "level1": "1920x1080 -> 640, crops 256x256",
+                   "level1_items": n1, "level2": f"head [{n1}, {a2}, {5 + c2}], crops 64x32",
+                   "level2_items_last_batch": int(ni2[1]), "handoff": "host (item table read back, stream sync)",
+                   "l2": f"working set {(sum(f.numel() for f in frames) + head1.numel() * 4 + crops1.numel() * 2) / 2**20:.0f} MiB"},
+        "e2e": None, "gpu_launches": int(launches), "clocks": clocks, "roofline": None, "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+    st1.close()
+    st2.close()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "two_level":
+        run_two_level(args)
     else:
         run_octo(args)
 

@@ -77,6 +77,9 @@ class StageStats(ctypes.Structure):
                 ("max_candidates_per_image", ctypes.c_int32)]
 
 
+REGION_DTYPE = np.dtype([("d_data", "<u8"), ("width", "<i4"), ("height", "<i4"), ("pitch_bytes", "<i4"),
+                         ("rx0", "<i4"), ("ry0", "<i4"), ("rx1", "<i4"), ("ry1", "<i4"), ("pad", "<i4")])
+
 KERNEL_NAMES = ("letterbox", "decode", "nms", "assemble", "crop")
 
 
@@ -303,13 +306,17 @@ class Stage:
         """Chained stage: this batch = the upstream items (ITEM_DTYPE records: frame index +
         rectangle) of the upstream frames (CUDA tensors [h, pitch]) with their (w, h) sizes."""
         n = len(items)
-        arr = (Region * max(n, 1))()
-        for i, it in enumerate(items):
-            f = frames[int(it["frame"])]
-            w, h = sizes[int(it["frame"])]
-            arr[i].d_data, arr[i].width, arr[i].height, arr[i].pitch_bytes = f.data_ptr(), w, h, f.stride(0)
-            arr[i].rx0, arr[i].ry0, arr[i].rx1, arr[i].ry1 = (int(it["rx0"]), int(it["ry0"]), int(it["rx1"]),
-                                                              int(it["ry1"]))
+        fr = np.asarray(items["frame"], dtype=np.int64)
+        ptrs = np.array([f.data_ptr() for f in frames], dtype=np.uint64)
+        pitches = np.array([f.stride(0) for f in frames], dtype=np.int32)
+        wh = np.asarray(sizes, dtype=np.int32).reshape(-1, 2)
+        reg = np.zeros(max(n, 1), dtype=REGION_DTYPE)
+        if n:
+            reg["d_data"][:n] = ptrs[fr]
+            reg["width"][:n], reg["height"][:n], reg["pitch_bytes"][:n] = wh[fr, 0], wh[fr, 1], pitches[fr]
+            for k in ("rx0", "ry0", "rx1", "ry1"):
+                reg[k][:n] = items[k]
+        arr = reg.ctypes.data_as(ctypes.POINTER(Region))
         rc = load_library().octo_adopt_regions(self.handle, arr, n, self._stream(stream))
         if rc != OCTO_OK:
             raise OctoError(rc, "octo_adopt_regions")
