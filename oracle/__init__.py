@@ -8,5 +8,5 @@ the CUDA package, and it imports nothing from it.
 from .oracle import (  # noqa: F401
     DET_DTYPE, build, letterbox_geometry, resize_f64, f64_to_half, letterbox, sigmoid,
     decode, sort_candidates, iou, nms, scale_back, postprocess_image, postprocess_region, crop_rect, crop,
-    assemble, StageResult, run_stage,
+    assemble, StageResult, run_stage, margin_report,
 )

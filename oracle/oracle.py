@@ -297,3 +297,39 @@ def run_stage(frames: Sequence[np.ndarray], sizes: Sequence[Tuple[int, int]], he
         res.rects.append(rects)
         res.crops.append(crops)
     return res
+
+
+def margin_report(head: np.ndarray, logits: bool = True, conf: float = 0.25, iou_thr: float = 0.45) -> dict:
+    """Margin certificate of one image in double precision: how close any decision of the stage
+    comes to flipping.  Returns the smallest |score - conf| over all anchors, the smallest gap
+    between neighbouring scores of the ordered candidates, and the smallest |IoU - iou_thr| over
+    all same-class candidate pairs (a superset of the pairs the greedy scan tests)."""
+    h = np.asarray(head, dtype=np.float64)
+    cls_v = h[:, 5:].max(axis=1)
+    if logits:
+        score = 1.0 / (1.0 + np.exp(-h[:, 4])) / (1.0 + np.exp(-cls_v))
+    else:
+        score = h[:, 4] * cls_v
+    ok = np.isfinite(h).all(axis=1) & (h[:, 2] > 0) & (h[:, 3] > 0)
+    cand = np.nonzero(ok & (score > conf))[0]
+    s = np.sort(score[cand])[::-1]
+    out = {"candidates": int(len(cand)),
+           "min_abs_score_minus_conf": float(np.min(np.abs(score[ok] - conf))) if ok.any() else float("inf"),
+           "min_score_gap": float(np.min(-np.diff(s))) if len(s) > 1 else float("inf"),
+           "min_abs_iou_minus_thr": float("inf")}
+    k = h[cand, 5:].argmax(axis=1)
+    x1, y1 = h[cand, 0] - 0.5 * h[cand, 2], h[cand, 1] - 0.5 * h[cand, 3]
+    x2, y2 = h[cand, 0] + 0.5 * h[cand, 2], h[cand, 1] + 0.5 * h[cand, 3]
+    for c in np.unique(k):
+        m = np.nonzero(k == c)[0]
+        if len(m) < 2:
+            continue
+        iw = np.clip(np.minimum(x2[m, None], x2[None, m]) - np.maximum(x1[m, None], x1[None, m]), 0, None)
+        ih = np.clip(np.minimum(y2[m, None], y2[None, m]) - np.maximum(y1[m, None], y1[None, m]), 0, None)
+        inter = iw * ih
+        area = (x2[m] - x1[m]) * (y2[m] - y1[m])
+        uni = area[:, None] + area[None, :] - inter
+        iou = np.where(uni > 0, inter / np.where(uni > 0, uni, 1.0), 0.0)
+        iu = np.triu_indices(len(m), 1)
+        out["min_abs_iou_minus_thr"] = min(out["min_abs_iou_minus_thr"], float(np.min(np.abs(iou[iu] - iou_thr))))
+    return out

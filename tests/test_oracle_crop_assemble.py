@@ -155,3 +155,20 @@ def test_stage_two_branch_packing_consistent():
     for (f, j), rect in zip(r.items[0], r.rects[0]):
         w, h = b.sizes[f]
         assert 0 <= rect[0] < rect[2] <= w and 0 <= rect[1] < rect[3] <= h
+
+
+def test_margin_report_on_the_workloads(capsys):
+    """How close the synthetic workloads come to a flipped decision (double precision).  Bit
+    exactness of the CUDA path rests on the fixed binary32 formulas, not on wide margins: in
+    the dense scene neighbouring scores are a few ulps apart."""
+    rows = []
+    for name in ("tiny", "traffic_1080p", "dense_nms", "sweep"):
+        b = workloads.make_batch(name, batch=1)
+        r = oracle.margin_report(b.head[0])
+        rows.append((name, r))
+        assert r["candidates"] > 0 and r["min_abs_score_minus_conf"] > 0 and r["min_score_gap"] >= 0
+        assert np.isfinite(r["min_abs_iou_minus_thr"])
+    with capsys.disabled():
+        for name, r in rows:
+            print(f"\n  margins {name}: cand={r['candidates']} |score-conf|>={r['min_abs_score_minus_conf']:.3e} "
+                  f"score gap>={r['min_score_gap']:.3e} |IoU-thr|>={r['min_abs_iou_minus_thr']:.3e}", end="")
