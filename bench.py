@@ -42,11 +42,11 @@ NCU_TRAFFIC = {
     # kernel: (source files, sha256[:16] of their concatenation at capture time, bytes per unit, unit)
     # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md)
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "e242c302f30bc941", 493304.0, "crop"),
+             "871dcab23b897b84", 493693.0, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                  "b85159dddf9a967d", 3692384.0, "frame"),
+                  "bc1f87af93a7ce97", 3705012.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "c2b06f79f1b032c4", 1697652.0, "frame"),
+               "933edd2128942e38", 1696520.0, "frame"),
 }
 
 
