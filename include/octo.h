@@ -221,6 +221,47 @@ OCTO_API int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int32
 OCTO_API int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_item, int32_t max_items,
                     void* d_out_f16, int32_t* d_offsets, int32_t* d_n_items, void* cuda_stream);
 
+/* ---- device-side dynamic-batch queue -------------------------------------------------------
+ * Downstream models take batches of the size bz the scheduler chose (Algorithm 1), while the
+ * number of objects per frame varies and arrives in bursts; requests wait in a queue until a
+ * batch fills, the first one waiting longest (Section II, Eq. 1 discussion; Section III-B,
+ * Observation 1).  An octo_queue_t keeps such pending items of ONE downstream branch on the
+ * device across successive detector batches: octo_queue_push appends the items of a stage's
+ * current batch, octo_queue_pop crops the oldest bz of them into a downstream batch.  Order
+ * is first in, first out: pushes in call order, inside a push the branch's item order.  Items
+ * that do not fit are dropped (newest first) and counted.  Queued items refer to their source
+ * frames by pointer: the caller keeps those frames alive and unchanged until the items are
+ * popped.  Not re-entrant; use one stream at a time.
+ */
+typedef struct octo_queue octo_queue_t;
+
+/* One queued item as reported by octo_queue_pop (48 bytes). */
+typedef struct {
+    const uint8_t* d_data;              /* source frame                                   */
+    int32_t width, height, pitch_bytes;
+    int32_t rx0, ry0, rx1, ry1;         /* crop rectangle                                 */
+    int32_t seq;                        /* number of the push that queued it (from 0)     */
+    int32_t frame, det;                 /* position in that push's batch                  */
+} octo_qitem_t;
+
+/* capacity: items the ring holds; out_w (multiple of 8) x out_h: crop size; max_bz: largest bz. */
+OCTO_API int octo_queue_create(int32_t device, int32_t capacity, int32_t out_w, int32_t out_h, int32_t swap_rb,
+                               int32_t max_bz, octo_queue_t** out);
+OCTO_API int octo_queue_destroy(octo_queue_t* q);
+
+/* Append the items of `branch` of the stage's current batch (after octo_postprocess_batch;
+ * same item order and rectangles as octo_crop_batch would use).  Enqueues one kernel.
+ * Errors: OCTO_E_INVALID_ARG, OCTO_E_NO_PREPROCESS, OCTO_E_NO_POSTPROCESS, OCTO_E_CUDA. */
+OCTO_API int octo_queue_push(octo_queue_t* q, octo_stage_t* st, int32_t branch, void* cuda_stream);
+
+/* Crop the oldest min(bz, pending) items into d_out_f16 [bz, 3, out_h, out_w] (slot i = i-th
+ * oldest; slots >= popped untouched) and remove them.  d_items_out (may be NULL): [bz] records
+ * of the popped items.  d_info: [4] int32 = {popped, pending after the pop, items dropped so far,
+ * seq of the oldest item still pending or -1}.  Enqueues two kernels; nothing synchronises.
+ * Errors: OCTO_E_INVALID_ARG (bz < 1 or > max_bz, null pointers), OCTO_E_ALIGNMENT, OCTO_E_CUDA. */
+OCTO_API int octo_queue_pop(octo_queue_t* q, int32_t bz, void* d_out_f16, octo_qitem_t* d_items_out,
+                            int32_t* d_info, void* cuda_stream);
+
 /* Synchronise `cuda_stream`, then read (and keep) the device status word. */
 OCTO_API int octo_stage_status(octo_stage_t* st, uint32_t* status_word, void* cuda_stream);
 

@@ -10,3 +10,4 @@ from .oracle import (  # noqa: F401
     decode, sort_candidates, iou, nms, scale_back, postprocess_image, postprocess_region, crop_rect, crop,
     assemble, StageResult, run_stage, margin_report,
 )
+from .queue import OracleQueue  # noqa: F401,E402

@@ -41,7 +41,7 @@ EXPORTS = (
     "octo_stage_item_table", "octo_stage_copy_items", "octo_stage_set_timing", "octo_stage_kernel_times",
     "octo_stage_workspace_bytes", "octo_stage_launch_count",
     "octo_strerror", "octo_last_cuda_error", "octo_version", "octo_postprocess_frame_static",
-    "octo_adopt_regions",
+    "octo_adopt_regions", "octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop",
 )
 
 
@@ -79,6 +79,10 @@ class StageStats(ctypes.Structure):
 
 REGION_DTYPE = np.dtype([("d_data", "<u8"), ("width", "<i4"), ("height", "<i4"), ("pitch_bytes", "<i4"),
                          ("rx0", "<i4"), ("ry0", "<i4"), ("rx1", "<i4"), ("ry1", "<i4"), ("pad", "<i4")])
+
+QITEM_DTYPE = np.dtype([("d_data", "<u8"), ("width", "<i4"), ("height", "<i4"), ("pitch_bytes", "<i4"),
+                        ("rx0", "<i4"), ("ry0", "<i4"), ("rx1", "<i4"), ("ry1", "<i4"), ("seq", "<i4"),
+                        ("frame", "<i4"), ("det", "<i4")])
 
 KERNEL_NAMES = ("letterbox", "decode", "nms", "assemble", "crop")
 
@@ -138,6 +142,12 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_postprocess_frame_static.argtypes = [i32, vp, i32, i32, i32, ctypes.c_float, ctypes.c_float,
                                                   i32, i32, i32, i32, vp, vp, vp]
     lib.octo_postprocess_frame_static.restype = ctypes.c_int
+    lib.octo_queue_create.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(vp)]
+    lib.octo_queue_destroy.argtypes = [vp]
+    lib.octo_queue_push.argtypes = [vp, vp, i32, vp]
+    lib.octo_queue_pop.argtypes = [vp, i32, vp, vp, vp, vp]
+    for name in ("octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop"):
+        getattr(lib, name).restype = ctypes.c_int
     lib.octo_stage_workspace_bytes.argtypes = [vp]
     lib.octo_stage_workspace_bytes.restype = ctypes.c_int64
     lib.octo_stage_launch_count.argtypes = [vp]
@@ -389,6 +399,55 @@ class Stage:
     @property
     def workspace_bytes(self) -> int:
         return int(load_library().octo_stage_workspace_bytes(self.handle))
+
+
+class Queue:
+    """Device-side dynamic-batch queue of one downstream branch (octo_queue_* in octo.h)."""
+
+    def __init__(self, capacity: int, out_w: int, out_h: int, max_bz: int, device: int = 0, swap_rb: bool = True):
+        import torch
+        self._torch = torch
+        self.out_w, self.out_h, self.max_bz = out_w, out_h, max_bz
+        self.device = torch.device("cuda", device)
+        h = ctypes.c_void_p()
+        rc = load_library().octo_queue_create(device, capacity, out_w, out_h, 1 if swap_rb else 0, max_bz,
+                                              ctypes.byref(h))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_queue_create")
+        self.handle = h
+        self._keepalive = []
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            load_library().octo_queue_destroy(self.handle)
+            self.handle = None
+
+    def _stream(self, stream) -> int:
+        if stream is None:
+            stream = self._torch.cuda.current_stream(self.device)
+        return int(stream.cuda_stream)
+
+    def push(self, stage: "Stage", branch: int = 0, stream=None) -> None:
+        rc = load_library().octo_queue_push(self.handle, stage.handle, branch, self._stream(stream))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_queue_push")
+        self._keepalive.append(list(stage._frames_keepalive))  # frames stay alive while queued
+        self._keepalive = self._keepalive[-64:]
+
+    def pop(self, bz: int, out=None, items=None, info=None, stream=None):
+        """Returns (crops fp16 [bz, 3, oh, ow], items uint8 [bz, 48], info int32 [4])."""
+        t = self._torch
+        if out is None:
+            out = t.empty((bz, 3, self.out_h, self.out_w), dtype=t.float16, device=self.device)
+        if items is None:
+            items = t.zeros((bz, QITEM_DTYPE.itemsize), dtype=t.uint8, device=self.device)
+        if info is None:
+            info = t.zeros((4,), dtype=t.int32, device=self.device)
+        rc = load_library().octo_queue_pop(self.handle, bz, out.data_ptr(), items.data_ptr(), info.data_ptr(),
+                                           self._stream(stream))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_queue_pop")
+        return out, items, info
 
 
 def dets_to_numpy(dets, counts) -> Tuple[np.ndarray, np.ndarray]:

@@ -27,6 +27,17 @@ struct FrameTable {
     FrameDesc f[CAP];
 };
 
+// One queued item of a device-side dynamic-batch queue: everything needed to crop it later,
+// independent of the stage batch it came from.
+struct QRecord {
+    const uint8_t* data;  // source frame
+    int32_t w, h, pitch;
+    int32_t rx0, ry0, rx1, ry1;
+    int32_t seq;          // number of the push that queued it
+    int32_t frame, det;   // position in that push's batch
+};
+static_assert(sizeof(QRecord) == 48, "QRecord layout");
+
 struct BranchDesc {
     int32_t out_w, out_h;
     uint32_t class_mask[4];

@@ -47,12 +47,16 @@ struct __align__(16) CropPass {
     int32_t _pad;
 };
 
-template <int CAP>
+// QUEUE = false: items come from the stage's current batch through the assembler above.
+// QUEUE = true: items are self-contained records popped from a device queue (qrec[0, *qpacked));
+// the assembler is skipped and nothing but the crops is written.
+template <int CAP, bool QUEUE>
 __global__ void __launch_bounds__(kCropKernelThreads, kCropCtasPerSm)
 crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int first_item, int max_items,
             const int* __restrict__ bcount, const int* __restrict__ bidx, const octo_det_t* __restrict__ dets,
             int* __restrict__ offsets, int* __restrict__ n_items, octo_item_t* __restrict__ items,
-            __half* __restrict__ out, int ow, int oh, int band_rows, int swap_rb, StageCounters* __restrict__ ctr) {
+            __half* __restrict__ out, int ow, int oh, int band_rows, int swap_rb, StageCounters* __restrict__ ctr,
+            const QRecord* __restrict__ qrec, const int* __restrict__ qpacked, unsigned int* __restrict__ qstatus) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t full[kCropStages], empty[kCropStages];
     __shared__ CropPass s_pass[kCropStages];
@@ -61,12 +65,12 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
 
     unsigned char* const s_rows0 = smem;
     XEntry* const s_xtab0 = reinterpret_cast<XEntry*>(smem + kCropStages * kCropRowBudget);  // kCropStages tables of ow entries
-    unsigned int* const status = &ctr->status;
+    unsigned int* const status = QUEUE ? qstatus : &ctr->status;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     // ---- assembler: offsets of the branch's items per frame ------------------------------------
-    if (warp == 0) {
+    if (!QUEUE && warp == 0) {
         int run = 0;
         for (int base = 0; base < n; base += 32) {
             const int i = base + lane;
@@ -90,10 +94,10 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         mbar_fence_init();
     }
     __syncthreads();
-    const int total = s_off[n];
+    const int total = QUEUE ? 0 : s_off[n];
     const long long rest = (long long)total - (long long)first_item;
-    const int packed = rest < 0 ? 0 : (rest > max_items ? max_items : (int)rest);
-    if (blockIdx.x == 0) {
+    const int packed = QUEUE ? min(*qpacked, max_items) : (rest < 0 ? 0 : (rest > max_items ? max_items : (int)rest));
+    if (!QUEUE && blockIdx.x == 0) {
         for (int i = threadIdx.x; i <= n; i += kCropKernelThreads) offsets[i] = s_off[i];
         if (threadIdx.x == 0) {
             n_items[0] = packed;
@@ -116,9 +120,11 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         // Items are resolved 32 tiles at a time, one per lane (q_* registers), so the dependent
         // loads slot -> detection index -> detection cost one round trip per 32 tiles.
         int w_tiles = 0;  // tiles opened so far
-        int q_slot = 0, q_band = 0, q_frame = 0, q_rx0 = 0, q_ry0 = 0, q_rx1 = 1, q_ry1 = 1;
+        int q_slot = 0, q_band = 0, q_pitch = 0, q_rx0 = 0, q_ry0 = 0, q_rx1 = 1, q_ry1 = 1;
+        const uint8_t* q_data = nullptr;
         int w_slot = 0, w_band = 0;
-        int w_frame = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
+        int w_pitch = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
+        const uint8_t* w_data = nullptr;
         int w_row_lo = 0, w_row_hi = 0, w_tile_cols = ow;
         int w_c0 = 0, w_ncols = 0, w_r0 = 0, w_nr = 0;
         int w_seg_lo = 0, w_seg = 0, w_stride = 16, w_pass_rows = 1;
@@ -148,6 +154,12 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             q_slot = (int)min(tile / bands, (long long)packed);  // >= packed: no such tile
             q_band = (int)(tile % bands);
             if (q_slot >= packed) return;
+            if (QUEUE) {
+                const QRecord rec = qrec[q_slot];
+                q_data = rec.data; q_pitch = rec.pitch;
+                q_rx0 = rec.rx0; q_ry0 = rec.ry0; q_rx1 = rec.rx1; q_ry1 = rec.ry1;
+                return;
+            }
             const int item = first_item + q_slot;
             int lo = 0, hi = n;  // largest f with s_off[f] <= item (frames without items are skipped)
             while (hi - lo > 1) {
@@ -172,7 +184,8 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 it._pad[0] = 0; it._pad[1] = 0;
                 items[q_slot] = it;
             }
-            q_frame = f; q_rx0 = rx0; q_ry0 = ry0; q_rx1 = rx1; q_ry1 = ry1;
+            q_data = fd.data; q_pitch = fd.pitch;
+            q_rx0 = rx0; q_ry0 = ry0; q_rx1 = rx1; q_ry1 = ry1;
         };
         // first pass of the next tile, if there is one
         auto open_tile = [&]() {
@@ -182,12 +195,14 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             w_tiles += 1;
             w_slot = __shfl_sync(0xffffffffu, q_slot, src);
             w_band = __shfl_sync(0xffffffffu, q_band, src);
-            const int f = __shfl_sync(0xffffffffu, q_frame, src);
+            const unsigned long long dptr = __shfl_sync(0xffffffffu, (unsigned long long)q_data, src);
+            const int pitch = __shfl_sync(0xffffffffu, q_pitch, src);
             const int rx0 = __shfl_sync(0xffffffffu, q_rx0, src), ry0 = __shfl_sync(0xffffffffu, q_ry0, src);
             const int rx1 = __shfl_sync(0xffffffffu, q_rx1, src), ry1 = __shfl_sync(0xffffffffu, q_ry1, src);
             w_valid = w_slot < packed;
             if (!w_valid) return;
-            w_frame = f;
+            w_data = reinterpret_cast<const uint8_t*>(dptr);
+            w_pitch = pitch;
             w_rx0 = rx0; w_ry0 = ry0; w_cw = rx1 - rx0; w_ch = ry1 - ry0;
             const int full_seg = ((3 * rx1 + 15) & ~15) - ((3 * rx0) & ~15);
             w_tile_cols =
@@ -252,7 +267,6 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 break;
             }
             // lane r owns output row w_r0 + r of the pass
-            const FrameDesc& fd = tab.f[w_frame];
             int y0 = 0, ry = 0;
             uint32_t bytes = 0;
             if (lane < w_nr) {
@@ -272,9 +286,9 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             __syncwarp();
             if (lane < w_nr) {
                 unsigned char* dst = s_rows0 + (size_t)b * kCropRowBudget + (size_t)(2 * lane) * w_stride;
-                const uint8_t* src = fd.data + (size_t)(w_ry0 + y0) * (size_t)fd.pitch + w_seg_lo;
+                const uint8_t* src = w_data + (size_t)(w_ry0 + y0) * (size_t)w_pitch + w_seg_lo;
                 bulk_g2s(dst, src, (uint32_t)w_seg, &full[b]);
-                if (ry != 0) bulk_g2s(dst + w_stride, src + fd.pitch, (uint32_t)w_seg, &full[b]);
+                if (ry != 0) bulk_g2s(dst + w_stride, src + w_pitch, (uint32_t)w_seg, &full[b]);
             }
             advance();
         }
@@ -351,20 +365,23 @@ static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     int grid = (int)(work < cap ? work : cap);
     if (grid < 1) grid = 1;  // a zero-slot window still gets its offsets and totals
     const size_t smem = (size_t)kCropStages * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w);
-    crop_kernel<CAP><<<grid, kCropKernelThreads, smem, stream>>>(
+    crop_kernel<CAP, false><<<grid, kCropKernelThreads, smem, stream>>>(
         tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
-        a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, band_rows, a.swap_rb, a.d_ctr);
+        a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, band_rows, a.swap_rb, a.d_ctr, nullptr,
+        nullptr, nullptr);
     return cudaGetLastError();
 }
 
 cudaError_t prepare_crop() {
     const int smem = kCropStages * (kCropRowBudget + (int)sizeof(XEntry) * 2048);
     cudaError_t e;
-    e = cudaFuncSetAttribute(crop_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(crop_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(crop_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(crop_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(crop_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(crop_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(crop_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 
 // Assembler + crop-resize of one branch window (a.max_items may be 0).
@@ -372,6 +389,26 @@ cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream) {
     if (a.n <= 8) return launch_crop_cap<8>(a, stream);
     if (a.n <= 64) return launch_crop_cap<64>(a, stream);
     return launch_crop_cap<512>(a, stream);
+}
+
+// Crop the records staged by a queue pop (at most bz of them) into the downstream batch.
+cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int bz, void* d_out, int out_w,
+                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, cudaStream_t stream) {
+    static FrameTable<8> tab;  // unused in queue mode
+    const long long cap = (long long)sm_count * kCropCtasPerSm;
+    long long bands_want = (8 * cap + bz - 1) / bz;
+    const int max_bands = (out_h + 7) / 8;
+    const int bands_req = (int)(bands_want < 1 ? 1 : (bands_want > max_bands ? max_bands : bands_want));
+    int band_rows = ((out_h + bands_req - 1) / bands_req + 7) & ~7;
+    band_rows = band_rows > out_h ? out_h : band_rows;
+    const int bands = (out_h + band_rows - 1) / band_rows;
+    const long long work = (long long)bz * bands;
+    const int grid = (int)(work < cap ? work : cap);
+    const size_t smem = (size_t)kCropStages * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)out_w);
+    crop_kernel<8, true><<<grid, kCropKernelThreads, smem, stream>>>(
+        tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
+        out_w, out_h, band_rows, swap_rb, nullptr, d_staged, d_qpacked, d_status);
+    return cudaGetLastError();
 }
 
 }  // namespace octo

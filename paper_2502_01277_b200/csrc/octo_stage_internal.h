@@ -1,0 +1,36 @@
+// Internal definition of the stage object, shared by the files that implement the C ABI.
+#pragma once
+
+#include "octo.h"
+#include "octo_kernels.h"
+
+constexpr int kEventPairs = 2048;
+
+struct octo_stage {
+    octo_stage_config_t cfg;
+    int sm_count;
+    int key_stride;  // candidate slots per image: next power of two >= A
+    // device workspace
+    unsigned long long* d_keys;
+    float4* d_boxes;
+    int* d_cand_count;
+    int* d_bcount;  // [branches][max_batch]
+    int* d_bidx;    // [branches][max_batch][max_det]
+    octo_item_t* d_items[OCTO_MAX_BRANCHES];
+    octo::StageCounters* d_ctr;
+    int64_t workspace_bytes;
+    // host state of the current batch
+    octo::FrameDesc frames[OCTO_MAX_BATCH];
+    int n_frames;
+    int max_w;
+    bool have_dets;
+    const octo_det_t* d_dets;
+    int64_t launches;
+    // optional per-kernel timing
+    bool timing;
+    cudaEvent_t ev[2 * kEventPairs];
+    int ev_kernel[kEventPairs];
+    int ev_used;
+    int64_t ev_dropped;
+};
+

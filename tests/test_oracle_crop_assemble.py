@@ -172,3 +172,19 @@ def test_margin_report_on_the_workloads(capsys):
         for name, r in rows:
             print(f"\n  margins {name}: cand={r['candidates']} |score-conf|>={r['min_abs_score_minus_conf']:.3e} "
                   f"score gap>={r['min_score_gap']:.3e} |IoU-thr|>={r['min_abs_iou_minus_thr']:.3e}", end="")
+
+
+def test_queue_hand_case():
+    """FIFO across pushes, newest dropped at capacity, oldest-pending stamp: worked by hand."""
+    q = oracle.OracleQueue(capacity=5)
+    q.push([(0, 0), (0, 1), (2, 0)], [(0, 0, 1, 1)] * 3, ["a", "b", "c"])          # seq 0: 3 items
+    q.push([(1, 0), (1, 1), (1, 2)], [(0, 0, 2, 2)] * 3, ["d", "e", "f"])          # seq 1: 2 fit, 1 dropped
+    recs, info = q.pop(2)
+    assert [(r[0], r[1], r[2]) for r in recs] == [(0, 0, 0), (0, 0, 1)] and info == (2, 3, 1, 0)
+    q.push([(0, 0)], [(1, 1, 3, 3)], ["g"])                                         # seq 2
+    recs, info = q.pop(3)
+    assert [(r[0], r[1], r[2], r[4]) for r in recs] == [(0, 2, 0, "c"), (1, 1, 0, "e"), (1, 1, 1, "e")]
+    assert info == (3, 1, 1, 2)
+    recs, info = q.pop(4)
+    assert [(r[0], r[3]) for r in recs] == [(2, (1, 1, 3, 3))] and info == (1, 0, 1, -1)
+    assert q.pop(2) == ([], (0, 0, 1, -1))
