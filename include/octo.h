@@ -89,6 +89,7 @@ typedef struct {
     int32_t pad_value;      /* canvas fill, 0..255 (114)                                    */
     int32_t swap_rb;        /* 1: output plane 0 = input channel 2 (BGR -> RGB)             */
     int32_t num_branches;   /* 1..OCTO_MAX_BRANCHES                                         */
+    int32_t class_agnostic; /* 1: NMS suppresses across classes (one class for NMS only)    */
     octo_branch_cfg_t branch[OCTO_MAX_BRANCHES];
 } octo_stage_config_t;
 

@@ -239,17 +239,22 @@ float orc_iou(const orc_det_t* a, const orc_det_t* b) {
 /* R5: greedy class-aware NMS over a list already in R4 order.  Element i is kept iff no
  * earlier KEPT element of the same class has IoU(j, i) > thr (strict); stops after max_det
  * kept.  keep[] receives the kept positions in order; returns their number. */
-int32_t orc_nms(const orc_det_t* c, int32_t n, float thr, int32_t max_det, int32_t* keep) {
+int32_t orc_nms_ex(const orc_det_t* c, int32_t n, float thr, int32_t max_det, int32_t agnostic, int32_t* keep) {
     int32_t k = 0;
     for (int32_t i = 0; i < n && k < max_det; ++i) {
         int alive = 1;
         for (int32_t t = 0; t < k; ++t) {
             const orc_det_t* j = &c[keep[t]];
-            if (j->cls == c[i].cls && orc_iou(j, &c[i]) > thr) { alive = 0; break; }
+            if ((agnostic || j->cls == c[i].cls) && orc_iou(j, &c[i]) > thr) { alive = 0; break; }
         }
         if (alive) keep[k++] = i;
     }
     return k;
+}
+/* Class-aware form (the default); with agnostic != 0 orc_nms_ex ignores the class test, i.e.
+ * boxes of different classes suppress each other (decode variant, classes kept for output). */
+int32_t orc_nms(const orc_det_t* c, int32_t n, float thr, int32_t max_det, int32_t* keep) {
+    return orc_nms_ex(c, n, thr, max_det, 0, keep);
 }
 
 /* R6: detector-input pixels -> source-frame pixels in binary32.  The detector input shows a
@@ -279,14 +284,22 @@ void orc_scale_back(orc_det_t* d, int32_t w, int32_t h, int32_t S) {
 
 /* R3..R6 for one image: head -> dets[<= max_det] in frame pixels.  Returns kept count;
  * *n_cand receives the candidate count before NMS. */
+int32_t orc_postprocess_image_ex(const float* head, int32_t A, int32_t C, int32_t logits,
+                                 float conf, float iou_thr, int32_t max_det, int32_t w, int32_t h,
+                                 int32_t S, int32_t agnostic, orc_det_t* dets, int32_t* n_cand);
 int32_t orc_postprocess_image(const float* head, int32_t A, int32_t C, int32_t logits,
                               float conf, float iou_thr, int32_t max_det, int32_t w, int32_t h,
                               int32_t S, orc_det_t* dets, int32_t* n_cand) {
+    return orc_postprocess_image_ex(head, A, C, logits, conf, iou_thr, max_det, w, h, S, 0, dets, n_cand);
+}
+int32_t orc_postprocess_image_ex(const float* head, int32_t A, int32_t C, int32_t logits,
+                                 float conf, float iou_thr, int32_t max_det, int32_t w, int32_t h,
+                                 int32_t S, int32_t agnostic, orc_det_t* dets, int32_t* n_cand) {
     orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * (size_t)(A > 0 ? A : 1));
     int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
     int32_t n = orc_decode(head, A, C, logits, conf, cand);
     orc_sort(cand, n);
-    int32_t k = orc_nms(cand, n, iou_thr, max_det, keep);
+    int32_t k = orc_nms_ex(cand, n, iou_thr, max_det, agnostic, keep);
     for (int32_t t = 0; t < k; ++t) {
         dets[t] = cand[keep[t]];
         orc_scale_back(&dets[t], w, h, S);

@@ -56,6 +56,10 @@ def _load():
     lib.orc_iou.restype = f32
     lib.orc_nms.argtypes = [vp, i32, f32, i32, vp]
     lib.orc_nms.restype = i32
+    lib.orc_nms_ex.argtypes = [vp, i32, f32, i32, i32, vp]
+    lib.orc_nms_ex.restype = i32
+    lib.orc_postprocess_image_ex.argtypes = [vp, i32, i32, i32, f32, f32, i32, i32, i32, i32, i32, vp, vp]
+    lib.orc_postprocess_image_ex.restype = i32
     lib.orc_scale_back.argtypes = [vp, i32, i32, i32]
     lib.orc_scale_back.restype = None
     lib.orc_postprocess_image.argtypes = [vp, i32, i32, i32, f32, f32, i32, i32, i32, i32, vp, vp]
@@ -150,11 +154,11 @@ def iou(a: np.ndarray, b: np.ndarray) -> float:
     return float(_load().orc_iou(_ptr(aa), _ptr(bb)))
 
 
-def nms(sorted_cand: np.ndarray, thr: float = 0.45, max_det: int = 300) -> np.ndarray:
+def nms(sorted_cand: np.ndarray, thr: float = 0.45, max_det: int = 300, agnostic: bool = False) -> np.ndarray:
     """Positions (int32) of the kept elements of an already ordered candidate list."""
     c = np.ascontiguousarray(sorted_cand, dtype=DET_DTYPE)
     keep = np.zeros(max(max_det, 1), dtype=np.int32)
-    k = _load().orc_nms(_ptr(c), len(c), np.float32(thr), max_det, _ptr(keep))
+    k = _load().orc_nms_ex(_ptr(c), len(c), np.float32(thr), max_det, 1 if agnostic else 0, _ptr(keep))
     return keep[:k].copy()
 
 
@@ -167,14 +171,15 @@ def scale_back(dets: np.ndarray, w: int, h: int, s: int) -> np.ndarray:
 
 
 def postprocess_image(head: np.ndarray, w: int, h: int, s: int, logits: bool = True,
-                      conf: float = 0.25, iou_thr: float = 0.45, max_det: int = 300):
+                      conf: float = 0.25, iou_thr: float = 0.45, max_det: int = 300, agnostic: bool = False):
     """head [A, 5+C] -> (dets in frame pixels [kept], candidate count)."""
     hd = np.ascontiguousarray(head, dtype=np.float32)
     a, row = hd.shape
     dets = np.zeros(max(max_det, 1), dtype=DET_DTYPE)
     ncand = np.zeros(1, dtype=np.int32)
-    k = _load().orc_postprocess_image(_ptr(hd), a, row - 5, 1 if logits else 0, np.float32(conf),
-                                      np.float32(iou_thr), max_det, w, h, s, _ptr(dets), _ptr(ncand))
+    k = _load().orc_postprocess_image_ex(_ptr(hd), a, row - 5, 1 if logits else 0, np.float32(conf),
+                                         np.float32(iou_thr), max_det, w, h, s, 1 if agnostic else 0,
+                                         _ptr(dets), _ptr(ncand))
     return dets[:k].copy(), int(ncand[0])
 
 
@@ -246,7 +251,7 @@ def run_stage(frames: Sequence[np.ndarray], sizes: Sequence[Tuple[int, int]], he
               conf: float = 0.25, iou_thr: float = 0.45, max_det: int = 300, pad_value: int = 114,
               swap_rb: bool = True, class_masks: Optional[Sequence[Sequence[int]]] = None,
               do_letterbox: bool = True, do_crops: bool = True, max_crops: Optional[int] = None,
-              threads: int = 1) -> StageResult:
+              threads: int = 1, agnostic: bool = False) -> StageResult:
     """Whole stage over one batch, frame by frame (optionally a thread per frame; the C
     routines release the GIL).  max_crops bounds the crops rendered per branch."""
     n = len(frames)
@@ -260,7 +265,7 @@ def run_stage(frames: Sequence[np.ndarray], sizes: Sequence[Tuple[int, int]], he
         w, h = sizes[i]
         if do_letterbox:
             det_in[i] = letterbox(frames[i], w, h, s, pad_value, swap_rb)
-        d, nc = postprocess_image(head[i], w, h, s, logits, conf, iou_thr, max_det)
+        d, nc = postprocess_image(head[i], w, h, s, logits, conf, iou_thr, max_det, agnostic)
         dets[i, : len(d)] = d
         counts[i] = len(d)
         ncand[i] = nc

@@ -55,7 +55,7 @@ class StageConfig(ctypes.Structure):
         ("num_anchors", ctypes.c_int32), ("num_classes", ctypes.c_int32),
         ("head_is_logits", ctypes.c_int32), ("conf_thresh", ctypes.c_float),
         ("iou_thresh", ctypes.c_float), ("max_det", ctypes.c_int32), ("pad_value", ctypes.c_int32),
-        ("swap_rb", ctypes.c_int32), ("num_branches", ctypes.c_int32),
+        ("swap_rb", ctypes.c_int32), ("num_branches", ctypes.c_int32), ("class_agnostic", ctypes.c_int32),
         ("branch", BranchCfg * OCTO_MAX_BRANCHES),
     ]
 
@@ -168,7 +168,8 @@ def make_config(*, device: int = 0, net_size: int = 640, max_batch: int = 8, num
                 num_classes: int = 80, head_is_logits: bool = True, conf_thresh: float = 0.25,
                 iou_thresh: float = 0.45, max_det: int = 300, pad_value: int = 114, swap_rb: bool = True,
                 branches: Sequence[Tuple[int, int]] = ((224, 224),),
-                class_masks: Optional[Sequence[Sequence[int]]] = None) -> StageConfig:
+                class_masks: Optional[Sequence[Sequence[int]]] = None,
+                class_agnostic: bool = False) -> StageConfig:
     cfg = StageConfig()
     cfg.device, cfg.net_size, cfg.max_batch = device, net_size, max_batch
     cfg.num_anchors, cfg.num_classes = num_anchors, num_classes
@@ -176,6 +177,7 @@ def make_config(*, device: int = 0, net_size: int = 640, max_batch: int = 8, num
     cfg.conf_thresh, cfg.iou_thresh = conf_thresh, iou_thresh
     cfg.max_det, cfg.pad_value, cfg.swap_rb = max_det, pad_value, 1 if swap_rb else 0
     cfg.num_branches = len(branches)
+    cfg.class_agnostic = 1 if class_agnostic else 0
     for b, (ow, oh) in enumerate(branches[:OCTO_MAX_BRANCHES]):
         cfg.branch[b].out_w, cfg.branch[b].out_h = ow, oh
         mask = class_masks[b] if class_masks is not None else (0xFFFFFFFF,) * 4

@@ -28,9 +28,12 @@ __device__ __forceinline__ float ld_obj(const float* p) {
 // too small to cover the SMs.
 template <int kDecPerThread>
 __global__ void __launch_bounds__(kDecThreads)
-decode_kernel(const float* __restrict__ head, int A, int C, int logits, float conf, int key_stride,
+decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf, int key_stride,
               unsigned long long* __restrict__ keys, int* __restrict__ cand_count,
               unsigned int* __restrict__ status) {
+    // mode bit 0: obj / class values are logits; bit 1: class-agnostic NMS (key class field 0)
+    const int logits = mode & 1;
+    const bool agnostic = (mode & 2) != 0;
     const int img = blockIdx.y;
     const int row_len = 5 + C;
     const float* __restrict__ hbase = head + (size_t)img * (size_t)A * (size_t)row_len;
@@ -95,7 +98,7 @@ decode_kernel(const float* __restrict__ head, int A, int C, int logits, float co
                                            : __fmul_rn(ob, best);
                 if (score > conf) {
                     const int slot = atomicAdd(cand_count + img, 1);
-                    const unsigned long long key = ((unsigned long long)(unsigned)best_k << 57) |
+                    const unsigned long long key = ((unsigned long long)(unsigned)(agnostic ? 0 : best_k) << 57) |
                                                    ((unsigned long long)(~__float_as_uint(score)) << kKeyAnchorBits) |
                                                    (unsigned long long)(unsigned)ra;
                     if (slot < key_stride) keys[(size_t)img * key_stride + slot] = key;

@@ -28,6 +28,7 @@ struct NmsArgs {
     octo_det_t* d_dets;
     int* d_counts;
     int num_branches;
+    int class_agnostic;  // NMS across classes; the class of a survivor is recomputed for the output
     BranchMasks masks;
     int* d_bcount;
     int* d_bidx;

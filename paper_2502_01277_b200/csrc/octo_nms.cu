@@ -74,7 +74,8 @@ __global__ void __launch_bounds__(kNmsThreads, 1)
 nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict__ head, int A, int C,
            const IouTest iou_test, int max_det, int key_stride, unsigned long long* __restrict__ gkeys,
            float4* __restrict__ gboxes, int* __restrict__ cand_count, octo_det_rec* __restrict__ dets,
-           int* __restrict__ counts, int num_branches, const __grid_constant__ BranchMasks masks,
+           int* __restrict__ counts, int num_branches, int class_agnostic,
+           const __grid_constant__ BranchMasks masks,
            int* __restrict__ bcount, int* __restrict__ bidx, int max_batch, StageCounters* __restrict__ ctr) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int seg_start[128], seg_cnt[128], cursor[128], nkept[128];
@@ -314,10 +315,20 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
     const float x_hi = (float)(fd.ox + fd.rw), y_hi = (float)(fd.oy + fd.rh);
     for (int r = threadIdx.x; r < nout; r += kNmsThreads) {
         const unsigned long long g = ordered[r];
-        const int cls = (int)(g & 127u);
+        int cls = (int)(g & 127u);
         const int anchor = (int)((g >> 7) & ((1ull << kKeyAnchorBits) - 1));
         const float score = __uint_as_float(~(unsigned)(g >> 32));
         const float4 b = gather_box(hbase + (size_t)anchor * row_len);
+        if (class_agnostic) {
+            // NMS ran with every candidate in class 0: recover the real class (first maximum)
+            const float* __restrict__ cv = hbase + (size_t)anchor * row_len + 5;
+            float best = __ldg(cv);
+            cls = 0;
+            for (int k = 1; k < C; ++k) {
+                const float v = __ldg(cv + k);
+                if (v > best) { best = v; cls = k; }
+            }
+        }
         octo_det_rec d;
         // X = fl(fl(fl(x - pad) * gain) + origin), clamped to the region
         d.x1 = fminf(fmaxf(__fadd_rn(__fmul_rn(__fsub_rn(b.x, fpl), fd.gx), x_lo), x_lo), x_hi);
@@ -329,7 +340,9 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
         d.anchor = anchor;
         d._pad = 0;
         dets[(size_t)img * max_det + r] = d;
+        if (class_agnostic) ordered[r] = (g & ~127ull) | (unsigned long long)cls;  // for the branch lists
     }
+    __syncthreads();
     if (threadIdx.x == 0) {
         counts[img] = nout;
         atomicAdd(&ctr->kept, (unsigned long long)nout);
@@ -379,7 +392,7 @@ static cudaError_t launch_cap(const NmsArgs& a, cudaStream_t stream) {
     nms_kernel<CAP><<<a.n, kNmsThreads, smem, stream>>>(tab, a.d_head, a.A, a.C, iou_test, a.max_det, a.key_stride,
                                                        a.d_keys, a.d_boxes, a.d_cand_count,
                                                        reinterpret_cast<octo_det_rec*>(a.d_dets), a.d_counts,
-                                                       a.num_branches, a.masks, a.d_bcount, a.d_bidx, a.max_batch,
+                                                       a.num_branches, a.class_agnostic, a.masks, a.d_bcount, a.d_bidx, a.max_batch,
                                                        a.d_ctr);
     return cudaGetLastError();
 }

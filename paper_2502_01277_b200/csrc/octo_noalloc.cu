@@ -157,6 +157,7 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
     a.d_dets = d_dets;
     a.d_counts = d_count;
     a.num_branches = 0;  // no downstream branch lists here
+    a.class_agnostic = 0;
     memset(&a.masks, 0, sizeof(a.masks));
     a.d_bcount = d_bcount;
     a.d_bidx = d_bidx;

@@ -53,6 +53,7 @@ static int validate_config(const octo_stage_config_t* c) {
     if (c->pad_value < 0 || c->pad_value > 255) return OCTO_E_INVALID_ARG;
     if (c->swap_rb != 0 && c->swap_rb != 1) return OCTO_E_INVALID_ARG;
     if (c->num_branches < 1 || c->num_branches > OCTO_MAX_BRANCHES) return OCTO_E_INVALID_ARG;
+    if (c->class_agnostic != 0 && c->class_agnostic != 1) return OCTO_E_INVALID_ARG;
     for (int b = 0; b < c->num_branches; ++b) {
         const octo_branch_cfg_t& br = c->branch[b];
         if (br.out_w < 8 || br.out_w > 2048 || (br.out_w & 7)) return OCTO_E_INVALID_ARG;
@@ -250,7 +251,7 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     OCTO_CUDA(cudaSetDevice(c.device));
     {
         ScopedKernelTimer t(st, OCTO_K_DECODE, stream);
-        OCTO_CUDA(launch_decode(d_head, n, c.num_anchors, c.num_classes, c.head_is_logits, c.conf_thresh,
+        OCTO_CUDA(launch_decode(d_head, n, c.num_anchors, c.num_classes, c.head_is_logits | (c.class_agnostic << 1), c.conf_thresh,
                                 st->key_stride, st->d_keys, st->d_cand_count, &st->d_ctr->status, stream));
     }
     st->launches += 1;
@@ -269,6 +270,7 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     a.d_dets = d_dets;
     a.d_counts = d_counts;
     a.num_branches = c.num_branches;
+    a.class_agnostic = c.class_agnostic;
     memset(&a.masks, 0, sizeof(a.masks));
     for (int b = 0; b < c.num_branches; ++b) memcpy(a.masks.m[b], c.branch[b].class_mask, sizeof(uint32_t) * 4);
     a.d_bcount = st->d_bcount;

@@ -370,3 +370,20 @@ def test_crop_of_very_wide_rectangles_is_tiled_by_columns():
             assert res.status == 0
         finally:
             st.close()
+
+
+def test_class_agnostic_nms_variant():
+    """Decode variant: suppression across classes; the survivors keep their own class."""
+    b = _small_case(400, 60, batch=3)
+    wl = b.workload
+    st = make_stage(wl, b.n, class_agnostic=True)
+    try:
+        ref = _oracle(b, agnostic=True)
+        ref_aware = _oracle(b, do_letterbox=False, do_crops=False)
+        res = run_stage_gpu(st, b.frames, b.sizes, b.head, max_items=[400])
+        _check_dets(res, ref)
+        _check_branch(res, ref, 0, max_items=400)
+        assert int(ref.counts.sum()) < int(ref_aware.counts.sum())
+        assert len(set(ref.dets[0, : ref.counts[0]]["cls"].tolist())) > 3
+    finally:
+        st.close()

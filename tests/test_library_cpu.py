@@ -41,7 +41,7 @@ def test_version_and_strerror():
 
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(binding.BranchCfg) == 24
-    assert ctypes.sizeof(binding.StageConfig) == 12 * 4 + 4 * 24
+    assert ctypes.sizeof(binding.StageConfig) == 13 * 4 + 4 * 24
     assert ctypes.sizeof(binding.Frame) == 24
     assert binding.DET_DTYPE.itemsize == 32 and binding.ITEM_DTYPE.itemsize == 32
     assert ctypes.sizeof(binding.StageStats) == 40

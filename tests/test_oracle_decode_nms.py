@@ -377,3 +377,31 @@ def test_chained_stage_maps_boxes_into_the_upstream_rectangle():
     d1, _ = oracle.postprocess_image(head, 256, 256, 256)
     d2, _ = oracle.postprocess_region(head, (0, 0, 256, 256), 256)
     assert d1.tobytes() == d2.tobytes()
+
+
+def test_class_agnostic_variant_worked_example_and_library():
+    """Decode variant: NMS across classes.  In the worked example D (class 1) has B's box, which
+    overlaps A by 0.681, so it dies as soon as classes are ignored: kept A, F, E."""
+    names, d = _load_worked()
+    s = oracle.sort_candidates(d)
+    assert [names[a] for a in s["anchor"][oracle.nms(s, 0.45, 300, agnostic=True)]] == ["A", "F", "E"]
+    assert [names[a] for a in s["anchor"][oracle.nms(s, 0.45, 300)]] == ["A", "F", "D", "E"]
+    rng = np.random.default_rng(15)
+    for trial in range(10):
+        n = 250
+        cxy = rng.uniform(50, 300, size=(n, 2)).astype(np.float32)
+        wh = rng.uniform(20, 80, size=(n, 2)).astype(np.float32)
+        boxes = np.concatenate([cxy - wh / 2, cxy + wh / 2], axis=1).astype(np.float32)
+        classes = rng.integers(0, 5, n)
+        scores = rng.permutation(n).astype(np.float32) / n + 0.001
+        tb = torch.from_numpy(boxes.astype(np.float64))
+        ious = torchvision.ops.box_iou(tb, tb).numpy()
+        bad = np.abs(ious - 0.45) < 1e-4
+        np.fill_diagonal(bad, False)
+        sel = np.setdiff1d(np.arange(n), np.unique(np.nonzero(bad)[0]))
+        boxes, classes, scores = boxes[sel], classes[sel], scores[sel]
+        ref = torchvision.ops.nms(torch.from_numpy(boxes), torch.from_numpy(scores), 0.45).numpy()
+        c = oracle.sort_candidates(_mk(boxes, scores, classes))
+        keep = oracle.nms(c, 0.45, 10 ** 6, agnostic=True)
+        assert list(c["anchor"][keep]) == list(ref)
+        assert len(keep) < len(oracle.nms(c, 0.45, 10 ** 6))  # fewer survive than with classes
