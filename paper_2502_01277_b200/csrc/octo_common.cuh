@@ -38,10 +38,6 @@ struct QRecord {
 };
 static_assert(sizeof(QRecord) == 48, "QRecord layout");
 
-struct BranchDesc {
-    int32_t out_w, out_h;
-    uint32_t class_mask[4];
-};
 
 // Device counters of a stage (one allocation, zeroed at creation).
 struct StageCounters {
@@ -73,37 +69,6 @@ __device__ __forceinline__ void src_coord(int d, int src, int dst, float inv_den
     else if (r >= den) { q += 1; r -= den; }
     if (q >= src - 1) { i0 = src - 1; rem = 0; return; }
     i0 = q; rem = r;
-}
-
-// Six consecutive bytes (two BGR pixels) starting at byte offset `o` of a 4-byte aligned
-// row of 32-bit words; `last_word` bounds the word index so nothing past the row is read.
-__device__ __forceinline__ void load6(const uint32_t* __restrict__ row, int o, int last_word,
-                                      uint32_t& lo, uint32_t& hi) {
-    const int wi = o >> 2;
-    const int sh = (o & 3) * 8;
-    const uint32_t a = row[wi];
-    const uint32_t b = row[min(wi + 1, last_word)];
-    const uint32_t c = row[min(wi + 2, last_word)];
-    lo = __funnelshift_r(a, b, sh);  // bytes o .. o+3
-    hi = __funnelshift_r(b, c, sh);  // bytes o+4 .. o+7
-}
-
-__device__ __forceinline__ float byte_f(uint32_t w, int i) {
-    return __uint2float_rn((w >> (8 * i)) & 0xffu);
-}
-
-// Horizontal lerp of one row's two taps for the three channels; fx == 0 skips the second tap.
-__device__ __forceinline__ void row_taps(uint32_t lo, uint32_t hi, float fx, bool lerp_x,
-                                         float& c0, float& c1, float& c2) {
-    c0 = byte_f(lo, 0);
-    c1 = byte_f(lo, 1);
-    c2 = byte_f(lo, 2);
-    if (lerp_x) {
-        const float d0 = byte_f(lo, 3), d1 = byte_f(hi, 0), d2 = byte_f(hi, 1);
-        c0 = fmaf(fx, d0 - c0, c0);
-        c1 = fmaf(fx, d1 - c1, c1);
-        c2 = fmaf(fx, d2 - c2, c2);
-    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -301,7 +266,7 @@ __device__ __forceinline__ float4 box_corners(float cx, float cy, float bw, floa
     return make_float4(__fsub_rn(cx, hw), __fsub_rn(cy, hh), __fadd_rn(cx, hw), __fadd_rn(cy, hh));
 }
 
-// IoU, operation by operation: inter / ((area_a + area_b) - inter), 0 if the union is empty.
+// The two terms of IoU = inter / uni, operation by operation: uni = (area_a + area_b) - inter.
 __device__ __forceinline__ void iou_terms(const float4 a, const float4 b, float& inter, float& uni) {
     float iw = __fsub_rn(fminf(a.z, b.z), fmaxf(a.x, b.x));
     float ih = __fsub_rn(fminf(a.w, b.w), fmaxf(a.y, b.y));
@@ -311,11 +276,6 @@ __device__ __forceinline__ void iou_terms(const float4 a, const float4 b, float&
     const float area_a = __fmul_rn(__fsub_rn(a.z, a.x), __fsub_rn(a.w, a.y));
     const float area_b = __fmul_rn(__fsub_rn(b.z, b.x), __fsub_rn(b.w, b.y));
     uni = __fsub_rn(__fadd_rn(area_a, area_b), inter);
-}
-__device__ __forceinline__ float iou_fixed(const float4 a, const float4 b) {
-    float inter, uni;
-    iou_terms(a, b, inter, uni);
-    return uni > 0.0f ? __fdiv_rn(inter, uni) : 0.0f;
 }
 
 // The test fl(inter / uni) > thr without the division.  The binary32 quotient rounds to a
