@@ -47,6 +47,7 @@ struct StageCounters {
     int max_cand;
     int packed;
     int total_items;
+    int sched[2];  // crop kernel: tiles handed out beyond each CTA's first, CTAs finished (both zero between launches)
 };
 
 constexpr int kKeyAnchorBits = 25;  // anchor index field of a candidate key
@@ -99,6 +100,11 @@ __device__ __forceinline__ void lds32x3(uint32_t addr, uint32_t& a, uint32_t& b,
                  : "=r"(a), "=r"(b), "=r"(c)
                  : "r"(addr));
 }
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -108,38 +114,43 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 // Integer horizontal lerp of the three channels of one destination pixel.  `addr` is the
 // shared-space address of the 4-byte aligned word that holds the left tap's first byte (the
 // staged rows keep at least 12 readable bytes past any tap); only the low five bits of `sh`
-// = 8 * byte offset matter (the funnel shift wraps).
-__device__ __forceinline__ void hsample(uint32_t addr, uint32_t sh, uint32_t wts, uint32_t& c0, uint32_t& c1,
-                                        uint32_t& c2) {
+// = 8 * byte offset matter (the funnel shift wraps).  The sums start from kF32Int, the bit
+// pattern of 2^23: a sum v < 2^23 (255 * den with den <= 8192) then IS the binary32 number
+// 2^23 + v, so no integer-to-float conversion is needed afterwards.
+constexpr uint32_t kF32Int = 0x4B000000u;
+constexpr float kF32IntValue = 8388608.0f;
+__device__ __forceinline__ void hsample(uint32_t addr, uint32_t sh, uint32_t wts, float& c0, float& c1, float& c2) {
     uint32_t a, b, c;
     lds32x3(addr, a, b, c);
     const uint32_t lo = __funnelshift_r(a, b, sh);  // B0 G0 R0 B1
     const uint32_t hi = __funnelshift_r(b, c, sh);  // G1 R1 .. ..
     const uint32_t p01 = __byte_perm(lo, hi, 0x4130);  // B0 B1 G0 G1
     const uint32_t p2 = __byte_perm(lo, hi, 0x5252);   // R0 R1 R0 R1
-    c0 = __dp2a_lo(wts, p01, 0u);
-    c1 = __dp2a_hi(wts, p01, 0u);
-    c2 = __dp2a_lo(wts, p2, 0u);
+    c0 = __uint_as_float(__dp2a_lo(wts, p01, kF32Int));
+    c1 = __uint_as_float(__dp2a_hi(wts, p01, kF32Int));
+    c2 = __uint_as_float(__dp2a_lo(wts, p2, kF32Int));
 }
 
 // One destination pixel: horizontal integer lerp on one or two staged rows (shared-space
 // addresses row0, row0 + row_step), then the vertical lerp and all scaling in fp32 (wx / wy
-// carry 1 / (255 * den_x * den_y)).
+// carry 1 / (255 * den_x * den_y); nwx = -2^23 * wx).  With h = 2^23 + v from hsample,
+// fma(h, wx, nwx) rounds the exact product v * wx once, and h - 2^23 is exact, so the result
+// is fl(fl(v0 * wx) + v1 * wy) bit for bit.
 template <bool LERP_Y>
 __device__ __forceinline__ void sample_px(uint32_t row0, uint32_t row_step, const uint32_t off, const uint32_t wts,
-                                          float wx, float wy, float& f0, float& f1, float& f2) {
+                                          float wx, float nwx, float wy, float& f0, float& f1, float& f2) {
     const uint32_t addr = row0 + (off & ~3u), sh = off << 3;
-    uint32_t a0, a1, a2;
+    float a0, a1, a2;
     hsample(addr, sh, wts, a0, a1, a2);
-    f0 = __uint2float_rn(a0) * wx;
-    f1 = __uint2float_rn(a1) * wx;
-    f2 = __uint2float_rn(a2) * wx;
+    f0 = __fmaf_rn(a0, wx, nwx);
+    f1 = __fmaf_rn(a1, wx, nwx);
+    f2 = __fmaf_rn(a2, wx, nwx);
     if (LERP_Y) {
-        uint32_t b0, b1, b2;
+        float b0, b1, b2;
         hsample(addr + row_step, sh, wts, b0, b1, b2);
-        f0 = fmaf(__uint2float_rn(b0), wy, f0);
-        f1 = fmaf(__uint2float_rn(b1), wy, f1);
-        f2 = fmaf(__uint2float_rn(b2), wy, f2);
+        f0 = __fmaf_rn(__fsub_rn(b0, kF32IntValue), wy, f0);
+        f1 = __fmaf_rn(__fsub_rn(b1, kF32IntValue), wy, f1);
+        f2 = __fmaf_rn(__fsub_rn(b2, kF32IntValue), wy, f2);
     }
 }
 
@@ -158,11 +169,12 @@ template <bool LERP_Y, bool FILL>
 __device__ __forceinline__ void sample_row(uint32_t row0, uint32_t row_step, float wx, float wy, uint32_t xt,
                                            int pairs, int lane, __half* __restrict__ o0, __half* __restrict__ o1,
                                            __half* __restrict__ o2, float fill_f) {
+    const float nwx = -kF32IntValue * wx;
     for (int pair = lane; pair < pairs; pair += 32) {
         const uint4 ee = lds128(xt + 16u * (uint32_t)pair);  // two XEntry: {off, wts} x 2
         float a0, a1, a2, b0, b1, b2;
-        sample_px<LERP_Y>(row0, row_step, ee.x, ee.y, wx, wy, a0, a1, a2);
-        sample_px<LERP_Y>(row0, row_step, ee.z, ee.w, wx, wy, b0, b1, b2);
+        sample_px<LERP_Y>(row0, row_step, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
+        sample_px<LERP_Y>(row0, row_step, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
         if (FILL) {
             if (ee.y == 0u) { a0 = fill_f; a1 = fill_f; a2 = fill_f; }
             if (ee.w == 0u) { b0 = fill_f; b1 = fill_f; b2 = fill_f; }
@@ -221,6 +233,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, ui
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, int limit = 1 << 20) {
     for (int i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// The same for a warp that expects to wait long (a producer waiting for its consumers): plain
+// phase tests with a sleep in between, so that the waiting warp takes almost no issue slots
+// from the working warps of its scheduler.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_sleeping(uint64_t* bar, uint32_t parity, unsigned sleep_ns,
+                                                   int limit = 1 << 20) {
+    for (int i = 0; i < limit; ++i) {
+        if (mbar_test_wait(bar, parity)) return true;
+        __nanosleep(sleep_ns);
+    }
     return false;
 }
 // Global -> shared bulk copy; both addresses 16-byte aligned, bytes a multiple of 16.

@@ -29,13 +29,15 @@ namespace octo {
 // segment longer than kCropMaxStride - 16 bytes (a rectangle wider than about 5300 pixels)
 // is split into column tiles, so one row pair always fits.  Two buffers form a ring between
 // the producer warp and the consumer warps.
-constexpr int kCropStages = 2;         // ring depth (row buffers and tap tables)
+constexpr int kCropStages = 2;         // ring depth (row buffers)
+constexpr int kCropTables = kCropStages + 1;  // tap tables, one more than ring slots
 constexpr int kCropRowBudget = 32768;  // bytes per ring buffer
 constexpr int kCropMaxStride = kCropRowBudget / 2;
 constexpr int kCropTilePx = 5300;
 constexpr int kCropMaxPassRows = 32;
 constexpr int kCropCtasPerSm = 3;
 constexpr int kCropConsumerWarps = 8;
+constexpr unsigned kCropProducerSleepNs = 200;  // between the producer's polls of an "empty" barrier
 constexpr int kCropKernelThreads = 32 * (kCropConsumerWarps + 1);  // + one producer warp
 
 // One pass of a CTA: output rows [r0, r0 + nr) x columns [c0, c0 + ncols) of one item.  The
@@ -56,7 +58,8 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             const int* __restrict__ bcount, const int* __restrict__ bidx, const octo_det_t* __restrict__ dets,
             int* __restrict__ offsets, int* __restrict__ n_items, octo_item_t* __restrict__ items,
             __half* __restrict__ out, int ow, int oh, int band_rows, int swap_rb, StageCounters* __restrict__ ctr,
-            const QRecord* __restrict__ qrec, const int* __restrict__ qpacked, unsigned int* __restrict__ qstatus) {
+            const QRecord* __restrict__ qrec, const int* __restrict__ qpacked, unsigned int* __restrict__ qstatus,
+            int* __restrict__ sched) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t full[kCropStages], empty[kCropStages];
     __shared__ CropPass s_pass[kCropStages];
@@ -64,7 +67,7 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
     __shared__ int s_off[CAP + 1];                                // exclusive scan of the frame counts
 
     unsigned char* const s_rows0 = smem;
-    XEntry* const s_xtab0 = reinterpret_cast<XEntry*>(smem + kCropStages * kCropRowBudget);  // kCropStages tables of ow entries
+    XEntry* const s_xtab0 = reinterpret_cast<XEntry*>(smem + kCropStages * kCropRowBudget);  // kCropTables tables of ow entries
     unsigned int* const status = QUEUE ? qstatus : &ctr->status;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -116,12 +119,12 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         const float inv_dx = 1.0f / (float)(2 * ow), inv_dy = 1.0f / (float)(2 * oh);
         // every scale factor folded into the vertical weights: 1 / (255 * den_x * den_y)
         const float inv_all = 1.0f / (255.0f * (float)(2 * ow) * (float)(2 * oh));
-        // Tiles of this CTA: index blockIdx.x + t * gridDim.x = slot * bands + band, t = 0, 1, ...
-        // Items are resolved 32 tiles at a time, one per lane (q_* registers), so the dependent
-        // loads slot -> detection index -> detection cost one round trip per 32 tiles.
+        // Tiles (index = slot * bands + band) are handed out dynamically: the first tile of a CTA
+        // is blockIdx.x, every further one comes from an atomic counter, so CTAs that drew cheap
+        // crops (small source rectangles) take more of them and the grid finishes together.  The
+        // round trips of a tile's resolution (counter -> detection index -> detection) are hidden
+        // behind the passes that are already staged in the ring.
         int w_tiles = 0;  // tiles opened so far
-        int q_slot = 0, q_band = 0, q_pitch = 0, q_rx0 = 0, q_ry0 = 0, q_rx1 = 1, q_ry1 = 1;
-        const uint8_t* q_data = nullptr;
         int w_slot = 0, w_band = 0;
         int w_pitch = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
         const uint8_t* w_data = nullptr;
@@ -148,61 +151,51 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             w_stride = w_seg + 16;
             w_pass_rows = max(1, min(min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows), band_rows));
         };
-        // lane l resolves the item of tile w_tiles + l
-        auto resolve_batch = [&]() {
-            const long long tile = (long long)blockIdx.x + (long long)(w_tiles + lane) * (long long)gridDim.x;
-            q_slot = (int)min(tile / bands, (long long)packed);  // >= packed: no such tile
-            q_band = (int)(tile % bands);
-            if (q_slot >= packed) return;
-            if (QUEUE) {
-                const QRecord rec = qrec[q_slot];
-                q_data = rec.data; q_pitch = rec.pitch;
-                q_rx0 = rec.rx0; q_ry0 = rec.ry0; q_rx1 = rec.rx1; q_ry1 = rec.ry1;
-                return;
-            }
-            const int item = first_item + q_slot;
-            int lo = 0, hi = n;  // largest f with s_off[f] <= item (frames without items are skipped)
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (s_off[mid] <= item) lo = mid; else hi = mid;
-            }
-            const int f = lo;
-            const int det = bidx[(size_t)f * max_det + (item - s_off[f])];
-            const octo_det_t d = dets[(size_t)f * max_det + det];
-            const FrameDesc& fd = tab.f[f];
-            // outward-rounded rectangle, clamped so that it is never empty
-            int rx0 = (int)floorf(d.x1), ry0 = (int)floorf(d.y1);
-            int rx1 = (int)ceilf(d.x2), ry1 = (int)ceilf(d.y2);
-            rx0 = min(max(rx0, 0), fd.w - 1);
-            ry0 = min(max(ry0, 0), fd.h - 1);
-            rx1 = min(max(rx1, rx0 + 1), fd.w);
-            ry1 = min(max(ry1, ry0 + 1), fd.h);
-            if (q_band == 0) {  // the tile of a slot's first band records the item
-                octo_item_t it;
-                it.frame = f; it.det = det;
-                it.rx0 = rx0; it.ry0 = ry0; it.rx1 = rx1; it.ry1 = ry1;
-                it._pad[0] = 0; it._pad[1] = 0;
-                items[q_slot] = it;
-            }
-            q_data = fd.data; q_pitch = fd.pitch;
-            q_rx0 = rx0; q_ry0 = ry0; q_rx1 = rx1; q_ry1 = ry1;
-        };
-        // first pass of the next tile, if there is one
+        // first pass of the next tile, if there is one; every lane resolves the same item
         auto open_tile = [&]() {
-            const int src = w_tiles & 31;
-            if (src == 0) resolve_batch();
-            __syncwarp();
+            long long tile = blockIdx.x;
+            if (w_tiles > 0) {
+                int t = 0;
+                if (lane == 0) t = atomicAdd(sched, 1);
+                tile = (long long)gridDim.x + (long long)__shfl_sync(0xffffffffu, t, 0);
+            }
             w_tiles += 1;
-            w_slot = __shfl_sync(0xffffffffu, q_slot, src);
-            w_band = __shfl_sync(0xffffffffu, q_band, src);
-            const unsigned long long dptr = __shfl_sync(0xffffffffu, (unsigned long long)q_data, src);
-            const int pitch = __shfl_sync(0xffffffffu, q_pitch, src);
-            const int rx0 = __shfl_sync(0xffffffffu, q_rx0, src), ry0 = __shfl_sync(0xffffffffu, q_ry0, src);
-            const int rx1 = __shfl_sync(0xffffffffu, q_rx1, src), ry1 = __shfl_sync(0xffffffffu, q_ry1, src);
-            w_valid = w_slot < packed;
+            w_valid = tile < (long long)packed * bands;
             if (!w_valid) return;
-            w_data = reinterpret_cast<const uint8_t*>(dptr);
-            w_pitch = pitch;
+            w_slot = (int)(tile / bands);
+            w_band = (int)(tile - (long long)w_slot * bands);
+            int rx0, ry0, rx1, ry1;
+            if (QUEUE) {
+                const QRecord rec = qrec[w_slot];
+                w_data = rec.data; w_pitch = rec.pitch;
+                rx0 = rec.rx0; ry0 = rec.ry0; rx1 = rec.rx1; ry1 = rec.ry1;
+            } else {
+                const int item = first_item + w_slot;
+                int lo = 0, hi = n;  // largest f with s_off[f] <= item (frames without items are skipped)
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (s_off[mid] <= item) lo = mid; else hi = mid;
+                }
+                const int f = lo;
+                const int det = bidx[(size_t)f * max_det + (item - s_off[f])];
+                const octo_det_t d = dets[(size_t)f * max_det + det];
+                const FrameDesc& fd = tab.f[f];
+                // outward-rounded rectangle, clamped so that it is never empty
+                rx0 = (int)floorf(d.x1); ry0 = (int)floorf(d.y1);
+                rx1 = (int)ceilf(d.x2); ry1 = (int)ceilf(d.y2);
+                rx0 = min(max(rx0, 0), fd.w - 1);
+                ry0 = min(max(ry0, 0), fd.h - 1);
+                rx1 = min(max(rx1, rx0 + 1), fd.w);
+                ry1 = min(max(ry1, ry0 + 1), fd.h);
+                if (w_band == 0 && lane == 0) {  // the tile of a slot's first band records the item
+                    octo_item_t it;
+                    it.frame = f; it.det = det;
+                    it.rx0 = rx0; it.ry0 = ry0; it.rx1 = rx1; it.ry1 = ry1;
+                    it._pad[0] = 0; it._pad[1] = 0;
+                    items[w_slot] = it;
+                }
+                w_data = fd.data; w_pitch = fd.pitch;
+            }
             w_rx0 = rx0; w_ry0 = ry0; w_cw = rx1 - rx0; w_ch = ry1 - ry0;
             const int full_seg = ((3 * rx1 + 15) & ~15) - ((3 * rx0) & ~15);
             w_tile_cols =
@@ -232,61 +225,64 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
 
         open_tile();
         uint32_t ephase = 0u;  // bit b: parity of empty[b] to wait for
-        int tb = kCropStages - 1;
+        int tb = kCropTables - 1;
         for (int k = 0;; ++k) {
             const int b = k % kCropStages;
+            // ---- prepare the pass in registers; nothing of ring slot b is touched yet ----
+            if (w_valid && w_new) {
+                // taps of every output column: byte offset inside a frame row + integer weights.
+                // Tables rotate with the tiles.  There is one more table than ring slots: the
+                // passes still in flight (k - kCropStages .. k - 1) belong to at most kCropStages
+                // tiles, so the table of the tile before those is free before this pass's wait.
+                tb = (tb + 1) % kCropTables;
+                XEntry* const xt = s_xtab0 + (size_t)tb * ow;
+                for (int dx = lane; dx < ow; dx += 32) xt[dx] = make_xentry(dx, w_cw, ow, inv_dx, 3 * w_rx0);
+            }
+            CropPass p;
+            p.valid = w_valid ? 1 : 0;
+            p.table = tb;
+            p.slot = w_slot; p.r0 = w_r0; p.nr = w_nr; p.c0 = w_c0; p.ncols = w_ncols;
+            p._pad = 0;
+            // lane r owns output row w_r0 + r of the pass
+            int ry = 0;
+            uint32_t bytes = 0;
+            RowInfo ri;
+            ri.row0 = 0; ri.step = 0; ri.wx = 0.0f; ri.wy = 0.0f;
+            const uint8_t* src = nullptr;
+            const bool has_row = w_valid && lane < w_nr;
+            if (has_row) {
+                int y0;
+                src_coord(w_r0 + lane, w_ch, oh, inv_dy, y0, ry);
+                bytes = (uint32_t)w_seg * (ry != 0 ? 2u : 1u);
+                ri.row0 = 2 * lane * w_stride - w_seg_lo;  // table offsets are relative to the frame row
+                ri.step = w_stride;
+                ri.wx = (float)(2 * oh - ry) * inv_all;
+                ri.wy = (float)ry * inv_all;
+                src = w_data + (size_t)(w_ry0 + y0) * (size_t)w_pitch + w_seg_lo;
+            }
+            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+            // ---- ring slot b: wait until the consumers have finished the pass that used it ----
             if (k >= kCropStages) {
                 const uint32_t par = (ephase >> b) & 1u;
-                // the consumers have finished the pass that used ring slot b
-                if (!mbar_wait_bounded(&empty[b], par) && !mbar_wait_bounded(&empty[b], par)) {
+                if (!mbar_wait_sleeping(&empty[b], par, kCropProducerSleepNs) && !mbar_wait_sleeping(&empty[b], par, kCropProducerSleepNs)) {
                     if (lane == 0) atomicOr(status, 0x4u);
                     break;
                 }
                 ephase ^= 1u << b;
             }
-            if (w_valid && w_new) {
-                // taps of every output column: byte offset inside a frame row + integer weights.
-                // Tables rotate with the tiles: this one belonged to the tile kCropStages tiles
-                // back, all of whose passes the wait above has seen finished (every tile in
-                // between has at least one pass).
-                tb = (tb + 1) % kCropStages;
-                XEntry* const xt = s_xtab0 + (size_t)tb * ow;
-                for (int dx = lane; dx < ow; dx += 32) xt[dx] = make_xentry(dx, w_cw, ow, inv_dx, 3 * w_rx0);
-            }
-            if (lane == 0) {
-                CropPass p;
-                p.valid = w_valid ? 1 : 0;
-                p.table = tb;
-                p.slot = w_slot; p.r0 = w_r0; p.nr = w_nr; p.c0 = w_c0; p.ncols = w_ncols;
-                p._pad = 0;
-                s_pass[b] = p;
-            }
+            if (lane == 0) s_pass[b] = p;
             if (!w_valid) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&full[b]);  // the end-of-work record
                 break;
             }
-            // lane r owns output row w_r0 + r of the pass
-            int y0 = 0, ry = 0;
-            uint32_t bytes = 0;
-            if (lane < w_nr) {
-                src_coord(w_r0 + lane, w_ch, oh, inv_dy, y0, ry);
-                bytes = (uint32_t)w_seg * (ry != 0 ? 2u : 1u);
-                RowInfo ri;
-                ri.row0 = 2 * lane * w_stride - w_seg_lo;  // table offsets are relative to the frame row
-                ri.step = w_stride;
-                ri.wx = (float)(2 * oh - ry) * inv_all;
-                ri.wy = (float)ry * inv_all;
-                s_row[b][lane] = ri;
-            }
-            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+            if (has_row) s_row[b][lane] = ri;
             fence_proxy_async();
             __syncwarp();  // table, pass record and row data are written before the barrier is armed
             if (lane == 0) mbar_expect_tx(&full[b], total);
             __syncwarp();
-            if (lane < w_nr) {
+            if (has_row) {
                 unsigned char* dst = s_rows0 + (size_t)b * kCropRowBudget + (size_t)(2 * lane) * w_stride;
-                const uint8_t* src = w_data + (size_t)(w_ry0 + y0) * (size_t)w_pitch + w_seg_lo;
                 bulk_g2s(dst, src, (uint32_t)w_seg, &full[b]);
                 if (ry != 0) bulk_g2s(dst + w_stride, src + w_pitch, (uint32_t)w_seg, &full[b]);
             }
@@ -318,30 +314,43 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             __half* const t2 = out2 + tile_off;
             const int pairs = cur.ncols >> 1;
             const int npairs = cur.nr * pairs;
-            const float inv_pairs = 1.0f / (float)pairs;
-            for (int idx = threadIdx.x; idx < npairs; idx += 32 * kCropConsumerWarps) {
-                int r = __float2int_rz(__int2float_rn(idx) * inv_pairs);
-                int pair = idx - r * pairs;
-                if (pair >= pairs) { pair -= pairs; ++r; }
-                else if (pair < 0) { pair += pairs; --r; }
+            // (row, pair) of this thread's first element, then advanced by the stride in place
+            constexpr int kStride = 32 * kCropConsumerWarps;
+            const int dr = kStride / pairs, dp = kStride - dr * pairs;
+            int r = (int)threadIdx.x / pairs, pair = (int)threadIdx.x - r * pairs;
+            for (int idx = threadIdx.x; idx < npairs; idx += kStride) {
                 const uint4 rw = lds128(rinfo + 16u * (uint32_t)r);
                 const uint4 ee = lds128(xt + 16u * (uint32_t)pair);
                 const float wx = __uint_as_float(rw.z), wy = __uint_as_float(rw.w);
+                const float nwx = -kF32IntValue * wx;
                 float a0, a1, a2, b0, b1, b2;
                 if (wy != 0.0f) {
-                    sample_px<true>(rows + rw.x, rw.y, ee.x, ee.y, wx, wy, a0, a1, a2);
-                    sample_px<true>(rows + rw.x, rw.y, ee.z, ee.w, wx, wy, b0, b1, b2);
+                    sample_px<true>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
+                    sample_px<true>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
                 } else {
-                    sample_px<false>(rows + rw.x, rw.y, ee.x, ee.y, wx, wy, a0, a1, a2);
-                    sample_px<false>(rows + rw.x, rw.y, ee.z, ee.w, wx, wy, b0, b1, b2);
+                    sample_px<false>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
+                    sample_px<false>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
                 }
                 const uint32_t o = (uint32_t)(r * ow + 2 * pair);
                 *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(a0, b0);
                 *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(a1, b1);
                 *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(a2, b2);
+                r += dr;
+                pair += dp;
+                if (pair >= pairs) { pair -= pairs; ++r; }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[b]);  // this warp is done with ring slot b
+        }
+    }
+    // The last CTA to finish puts the tile counter back to zero for the next launch.
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(sched + 1, 1) == (int)gridDim.x - 1) {
+            sched[0] = 0;
+            sched[1] = 0;
+            __threadfence();
         }
     }
 }
@@ -364,16 +373,16 @@ static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     long long work = (long long)a.max_items * bands;
     int grid = (int)(work < cap ? work : cap);
     if (grid < 1) grid = 1;  // a zero-slot window still gets its offsets and totals
-    const size_t smem = (size_t)kCropStages * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)a.out_w);
+    const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)a.out_w;
     crop_kernel<CAP, false><<<grid, kCropKernelThreads, smem, stream>>>(
         tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
         a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, band_rows, a.swap_rb, a.d_ctr, nullptr,
-        nullptr, nullptr);
+        nullptr, nullptr, a.d_ctr->sched);
     return cudaGetLastError();
 }
 
 cudaError_t prepare_crop() {
-    const int smem = kCropStages * (kCropRowBudget + (int)sizeof(XEntry) * 2048);
+    const int smem = kCropStages * kCropRowBudget + kCropTables * (int)sizeof(XEntry) * 2048;
     cudaError_t e;
     e = cudaFuncSetAttribute(crop_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -393,7 +402,7 @@ cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream) {
 
 // Crop the records staged by a queue pop (at most bz of them) into the downstream batch.
 cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int bz, void* d_out, int out_w,
-                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, cudaStream_t stream) {
+                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, int* d_sched, cudaStream_t stream) {
     static FrameTable<8> tab;  // unused in queue mode
     const long long cap = (long long)sm_count * kCropCtasPerSm;
     long long bands_want = (8 * cap + bz - 1) / bz;
@@ -404,10 +413,10 @@ cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int
     const int bands = (out_h + band_rows - 1) / band_rows;
     const long long work = (long long)bz * bands;
     const int grid = (int)(work < cap ? work : cap);
-    const size_t smem = (size_t)kCropStages * ((size_t)kCropRowBudget + sizeof(XEntry) * (size_t)out_w);
+    const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)out_w;
     crop_kernel<8, true><<<grid, kCropKernelThreads, smem, stream>>>(
         tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
-        out_w, out_h, band_rows, swap_rb, nullptr, d_staged, d_qpacked, d_status);
+        out_w, out_h, band_rows, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched);
     return cudaGetLastError();
 }
 

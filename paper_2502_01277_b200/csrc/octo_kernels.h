@@ -64,7 +64,7 @@ cudaError_t launch_decode(const float* d_head, int n, int A, int C, int logits, 
 cudaError_t launch_nms(const NmsArgs& a, cudaStream_t stream);
 cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream);  // batch assembler + crop-resize
 cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int bz, void* d_out, int out_w,
-                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, cudaStream_t stream);
+                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, int* d_sched, cudaStream_t stream);
 
 constexpr int kLetterboxMaxWidth = 8192;  // widest frame the row staging supports
 

@@ -21,6 +21,7 @@ struct QueueState {
     long long dropped;
     int seq;               // pushes so far
     unsigned int status;
+    int sched[2];          // tile scheduler words of the crop kernel (zero between launches)
 };
 
 constexpr int kQueueThreads = 1024;
@@ -206,6 +207,6 @@ extern "C" int octo_queue_pop(octo_queue_t* q, int32_t bz, void* d_out_f16, octo
                                            reinterpret_cast<QRecord*>(d_items_out), d_info, q->d_qpacked);
     if (cudaGetLastError() != cudaSuccess) return OCTO_E_CUDA;
     cudaError_t e = launch_crop_queue(q->d_staged, q->d_qpacked, bz, d_out_f16, q->out_w, q->out_h, q->swap_rb,
-                                      q->sm_count, &q->d_state->status, stream);
+                                      q->sm_count, &q->d_state->status, q->d_state->sched, stream);
     return e == cudaSuccess ? OCTO_OK : OCTO_E_CUDA;
 }
