@@ -37,6 +37,7 @@ constexpr int kCropTilePx = 5300;
 constexpr int kCropMaxPassRows = 32;
 constexpr int kCropCtasPerSm = 3;
 constexpr int kCropConsumerWarps = 8;
+constexpr int kCropTilesPerCta = 4;  // measured: 4 > 8 > 16 > 1 for small batches; a tile switch costs about 1 us
 constexpr unsigned kCropProducerSleepNs = 200;  // between the producer's polls of an "empty" barrier
 constexpr int kCropKernelThreads = 32 * (kCropConsumerWarps + 1);  // + one producer warp
 
@@ -57,7 +58,7 @@ __global__ void __launch_bounds__(kCropKernelThreads, kCropCtasPerSm)
 crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int first_item, int max_items,
             const int* __restrict__ bcount, const int* __restrict__ bidx, const octo_det_t* __restrict__ dets,
             int* __restrict__ offsets, int* __restrict__ n_items, octo_item_t* __restrict__ items,
-            __half* __restrict__ out, int ow, int oh, int band_rows, int swap_rb, StageCounters* __restrict__ ctr,
+            __half* __restrict__ out, int ow, int oh, int swap_rb, StageCounters* __restrict__ ctr,
             const QRecord* __restrict__ qrec, const int* __restrict__ qpacked, unsigned int* __restrict__ qstatus,
             int* __restrict__ sched) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -111,6 +112,12 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         }
     }
 
+    // Tiles are (slot, row band).  One band per crop amortises the per-tile work (item lookup, tap
+    // table) best; crops are cut into bands (multiples of 8 rows) only as far as needed to give
+    // every CTA about kCropTilesPerCta tiles, which keeps the end of the grid short.
+    const int bands_want = packed > 0 ? (kCropTilesPerCta * (int)gridDim.x + packed - 1) / packed : 1;
+    const int bands_req = min(max(bands_want, 1), (oh + 7) >> 3);
+    const int band_rows = min(((oh + bands_req - 1) / bands_req + 7) & ~7, oh);
     const int bands = (oh + band_rows - 1) / band_rows;
     const size_t plane = (size_t)ow * (size_t)oh;
 
@@ -359,24 +366,16 @@ template <int CAP>
 static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     static FrameTable<CAP> tab;
     for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
-    // Tiles are (slot, row band).  One band per crop amortises the per-tile work (item lookup,
-    // tap table) best; crops are only cut into bands when there are too few of them to fill
-    // the grid about eight times over (the slots are usually provisioned generously).  Bands are multiples of the consumer warp count.
+    // The kernel cuts crops into row bands itself once it knows how many items there are; the
+    // grid only has to be large enough for the finest cut.
     const long long cap = (long long)a.sm_count * kCropCtasPerSm;
-    const long long slots = a.max_items > 0 ? a.max_items : 1;
-    long long bands_want = (8 * cap + slots - 1) / slots;
-    const int max_bands = (a.out_h + 7) / 8;
-    const int bands_req = (int)(bands_want < 1 ? 1 : (bands_want > max_bands ? max_bands : bands_want));
-    int band_rows = ((a.out_h + bands_req - 1) / bands_req + 7) & ~7;
-    band_rows = band_rows > a.out_h ? a.out_h : band_rows;
-    const int bands = (a.out_h + band_rows - 1) / band_rows;
-    long long work = (long long)a.max_items * bands;
+    const long long work = (long long)a.max_items * ((a.out_h + 7) / 8);
     int grid = (int)(work < cap ? work : cap);
     if (grid < 1) grid = 1;  // a zero-slot window still gets its offsets and totals
     const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)a.out_w;
     crop_kernel<CAP, false><<<grid, kCropKernelThreads, smem, stream>>>(
         tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
-        a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, band_rows, a.swap_rb, a.d_ctr, nullptr,
+        a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, a.swap_rb, a.d_ctr, nullptr,
         nullptr, nullptr, a.d_ctr->sched);
     return cudaGetLastError();
 }
@@ -405,18 +404,12 @@ cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int
                               int out_h, int swap_rb, int sm_count, unsigned int* d_status, int* d_sched, cudaStream_t stream) {
     static FrameTable<8> tab;  // unused in queue mode
     const long long cap = (long long)sm_count * kCropCtasPerSm;
-    long long bands_want = (8 * cap + bz - 1) / bz;
-    const int max_bands = (out_h + 7) / 8;
-    const int bands_req = (int)(bands_want < 1 ? 1 : (bands_want > max_bands ? max_bands : bands_want));
-    int band_rows = ((out_h + bands_req - 1) / bands_req + 7) & ~7;
-    band_rows = band_rows > out_h ? out_h : band_rows;
-    const int bands = (out_h + band_rows - 1) / band_rows;
-    const long long work = (long long)bz * bands;
+    const long long work = (long long)bz * ((out_h + 7) / 8);
     const int grid = (int)(work < cap ? work : cap);
     const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)out_w;
     crop_kernel<8, true><<<grid, kCropKernelThreads, smem, stream>>>(
         tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
-        out_w, out_h, band_rows, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched);
+        out_w, out_h, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched);
     return cudaGetLastError();
 }
 
