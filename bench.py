@@ -98,9 +98,13 @@ def crop_bytes(items: np.ndarray, ow: int, oh: int) -> int:
     return int(len(items) * 3 * ow * oh * 2 + int((cw * ch * 3).sum()))
 
 
-def decode_bytes(n: int, a: int, c: int, candidates: int, logits: bool) -> int:
-    """One 32-byte sector per head row for the obj scan (logit heads) or the whole row
-    (probability heads), plus the full row and the 8-byte key of each candidate."""
+def decode_bytes(n: int, a: int, c: int, candidates: int, logits: bool, layout: str = "rows") -> int:
+    """Rows layout: one 32-byte sector per head row for the obj scan (logit heads) or the whole
+    row (probability heads), plus the full row and the 8-byte key of each candidate.  Planes
+    layout: every class plane (the maximum over classes needs all of them), plus four box
+    values and the key of each candidate."""
+    if layout == "planes":
+        return int(4 * c * a * n + candidates * (4 * 32 + 8))
     row = 4 * (5 + c)
     scan = 32 * a * n if logits else row * a * n
     return int(scan + candidates * (row + 8))
@@ -186,7 +190,7 @@ def oracle_pass(batch, frames_used: int, threads: int) -> float:
     t0 = time.perf_counter()
     oracle.run_stage(batch.frames[:frames_used], batch.sizes[:frames_used], batch.head[:frames_used],
                      wl.net_size, wl.branches, logits=wl.logits, conf=wl.conf_thresh, iou_thr=wl.iou_thresh,
-                     max_det=wl.max_det, threads=threads)
+                     max_det=wl.max_det, threads=threads, layout=wl.head_layout, multi_label=wl.multi_label)
     return time.perf_counter() - t0
 
 
@@ -262,7 +266,8 @@ def run_octo(args):
 
     stage = octo.Stage(device=local_rank, net_size=s, max_batch=n, num_anchors=wl.num_anchors,
                        num_classes=wl.num_classes, head_is_logits=wl.logits, conf_thresh=wl.conf_thresh,
-                       iou_thresh=wl.iou_thresh, max_det=wl.max_det, branches=wl.branches)
+                       iou_thresh=wl.iou_thresh, max_det=wl.max_det, branches=wl.branches,
+                       head_layout=wl.head_layout, multi_label=wl.multi_label)
     stream = torch.cuda.Stream(dev)
     cap = n * wl.items_per_frame
 
@@ -359,7 +364,7 @@ def run_octo(args):
     kern = {}
     alg = {
         "letterbox": letterbox_bytes(batch.sizes, s),
-        "decode": decode_bytes(n, wl.num_anchors, wl.num_classes, int(cand_per_step), wl.logits),
+        "decode": decode_bytes(n, wl.num_anchors, wl.num_classes, int(cand_per_step), wl.logits, wl.head_layout),
         "crop": sum(crop_bytes(items[b], *wl.branches[b]) for b in range(len(wl.branches))) / len(wl.branches),
     }
     names = octo.binding.KERNEL_NAMES
@@ -406,7 +411,7 @@ def run_octo(args):
             ln.stage = octo.Stage(device=local_rank, net_size=s, max_batch=c, num_anchors=wl.num_anchors,
                                   num_classes=wl.num_classes, head_is_logits=wl.logits,
                                   conf_thresh=wl.conf_thresh, iou_thresh=wl.iou_thresh, max_det=wl.max_det,
-                                  branches=wl.branches)
+                                  branches=wl.branches, head_layout=wl.head_layout, multi_label=wl.multi_label)
             ln.stream = torch.cuda.Stream(dev)
             ln.small = torch.cuda.Event()
             ln.head = torch.empty((c,) + tuple(h_head.shape[1:]), dtype=torch.float32, device=dev)
@@ -502,7 +507,7 @@ def run_octo(args):
             "config": {
                 "workload": f"{name} B={n}" + (" per GPU" if world > 1 else ""),
                 "frames": "x".join(str(v) for v in batch.sizes[0]) + (" (mixed)" if len(set(batch.sizes)) > 1 else ""),
-                "net_size": s, "head": [n, wl.num_anchors, 5 + wl.num_classes],
+                "net_size": s, "head": list(batch.head.shape),
                 "crops": [list(b) for b in wl.branches], "items_per_step": [t[1] for t in totals],
                 "candidates_per_step": cand_per_step, "parallelism": f"replicas x{world}",
                 "l2": (f"{n_sets} rotating input/output sets, {n_sets * (in_bytes + out_bytes) / 2**20:.0f} MiB working set"

@@ -66,14 +66,26 @@ typedef enum {
 #define OCTO_STATUS_COPY_TIMEOUT 0x4u   /* a bulk-copy wait ran out; that tile was skipped    */
 #define OCTO_STATUS_BIG_NMS 0x8u        /* an image had more candidates than fit on chip and   */
                                         /* took the slower global-memory path (informational)  */
+#define OCTO_STATUS_CAND_OVERFLOW 0x10u /* multi-label decode found more candidates in an image */
+                                        /* than the workspace holds; the excess was dropped    */
+
+/* Head layouts (octo_stage_config_t.head_layout). */
+#define OCTO_HEAD_ROWS 0   /* [n, A, 5 + C]: rows (cx, cy, w, h, obj, class_0 ..)              */
+#define OCTO_HEAD_PLANES 1 /* [n, 4 + C, A]: planes cx, cy, w, h, class_0 ..; no objectness    */
 
 typedef struct octo_stage octo_stage_t; /* opaque; owned by the library */
 
 /* One downstream branch (e.g. vehicle classifier 224x224, plate detector 256x256).
- * class_mask: bit k (word k/32, bit k%32) set => detections of class k feed this branch. */
+ * class_mask: bit k (word k/32, bit k%32) set => detections of class k feed this branch.
+ * The last four fields select what the downstream model expects of its input; all zero gives
+ * the plain form (stretch, value / 255). */
 typedef struct {
     int32_t out_w, out_h;   /* crop size; out_w must be a multiple of 8 */
     uint32_t class_mask[4];
+    int32_t keep_aspect;    /* 1: fit the rectangle into out_w x out_h without distortion     */
+                            /* (centred, rest of the slot = the stage's pad_value)            */
+    int32_t normalize;      /* 1: output = (value / 255 - mean[p]) / std[p] for output plane p */
+    float mean[3], std[3];  /* per OUTPUT plane (after swap_rb); std > 0; used if normalize   */
 } octo_branch_cfg_t;
 
 typedef struct {
@@ -90,6 +102,8 @@ typedef struct {
     int32_t swap_rb;        /* 1: output plane 0 = input channel 2 (BGR -> RGB)             */
     int32_t num_branches;   /* 1..OCTO_MAX_BRANCHES                                         */
     int32_t class_agnostic; /* 1: NMS suppresses across classes (one class for NMS only)    */
+    int32_t head_layout;    /* OCTO_HEAD_ROWS (0) or OCTO_HEAD_PLANES; see octo_postprocess_batch */
+    int32_t multi_label;    /* 1: every class above the threshold is a candidate of its own  */
     octo_branch_cfg_t branch[OCTO_MAX_BRANCHES];
 } octo_stage_config_t;
 
@@ -194,6 +208,16 @@ OCTO_API int octo_adopt_regions(octo_stage_t* st, const octo_region_t* regions, 
  * binary32 as inter / (area_a + area_b - inter) on letterbox-pixel corners
  * x1 = cx - w/2 ...; at most max_det are kept.  Kept boxes are mapped to frame pixels,
  * X = (x - pad_left) * fl(w / nw), clamped to [0, w] x [0, h].
+ * Variants (stage configuration; the paper's pipelines mix detector families, Section V-A).
+ *   head_layout = OCTO_HEAD_PLANES: d_head is [n, 4 + C, A] (anchor-free heads; value e of
+ *     anchor a at e * A + a, 16-byte alignment lets the scan use vector loads).  There is no
+ *     objectness: score = sigma(c_k*) for logits, c_k* for probabilities; everything else as
+ *     above.
+ *   multi_label = 1: every class k whose own score (sigma(obj) * sigma(c_k), or the planes
+ *     form) exceeds conf_thresh is a candidate of class k; candidates of one anchor share its
+ *     box.  Order: score descending, then anchor, then class.  The workspace holds 2 * P
+ *     candidates per image (P = A rounded up to a power of two); an image that yields more
+ *     sets OCTO_STATUS_CAND_OVERFLOW and loses the excess.  Not combinable with class_agnostic.
  * Errors: OCTO_E_INVALID_ARG, OCTO_E_NO_PREPROCESS, OCTO_E_CUDA.
  */
 OCTO_API int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int32_t n,
@@ -215,6 +239,11 @@ OCTO_API int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int32
  * rectangle is rx0 = clamp(floor(x1), 0, w-1), rx1 = clamp(ceil(x2), rx0 + 1, w), likewise
  * in y; the rectangle is stretched to out_w x out_h with the same bilinear rule as the
  * letterbox (taps clamped inside the rectangle), same plane order, /255, binary16.
+ * Branch options.  keep_aspect: the cw x ch rectangle is resized to nw x nh, where the side
+ * with the larger ratio fills the slot (nw = out_w if out_w * ch <= out_h * cw, else nh =
+ * out_h) and the other is round-half-up of the exact quotient (at least 1), centred with the
+ * odd pixel right / bottom as in the letterbox; the rest of the slot holds pad_value / 255.
+ * normalize: every output value v (pixels and padding alike) becomes (v - mean[p]) / std[p].
  * Uses the detections written by the last octo_postprocess_batch (d_dets must still be
  * valid) and the frames of the last octo_preprocess_batch.
  * Errors: OCTO_E_INVALID_ARG, OCTO_E_NO_PREPROCESS, OCTO_E_NO_POSTPROCESS, OCTO_E_CUDA.

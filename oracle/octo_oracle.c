@@ -211,13 +211,72 @@ int32_t orc_decode(const float* head, int32_t A, int32_t C, int32_t logits, floa
     return n;
 }
 
-/* R4: total order -- score descending, then anchor ascending. */
+/* R3 variants: other head layouts and multi-label candidates.
+ *   layout 0  rows   [A][5 + C]: (cx, cy, w, h, obj, class_0 ..), the form above.
+ *   layout 1  planes [4 + C][A]: element e of anchor a at head[e * A + a]; anchor-free heads
+ *             carry no objectness, the score is the class value alone: sigma(c_k) for logits,
+ *             c_k for probabilities.
+ *   multi_label 0: one candidate per anchor, k* = first maximal class value.
+ *   multi_label 1: every class k whose own score fl(sigma(obj) * sigma(c_k)) (rows) or
+ *             sigma(c_k) (planes) exceeds conf is a candidate of that class; an anchor can
+ *             yield several candidates that share its box.
+ * The row filter is the same: every value of the anchor finite, w > 0, h > 0.  Output in
+ * (anchor, class) order; returns the count (at most `cap` are written). */
+int32_t orc_decode_ex(const float* head, int32_t A, int32_t C, int32_t logits, float conf,
+                      int32_t layout, int32_t multi_label, orc_det_t* out, int32_t cap) {
+    int32_t n = 0;
+    const int nbox = layout == 0 ? 5 : 4; /* values before the class values */
+    const int row = nbox + C;
+    float* v = (float*)malloc(sizeof(float) * (size_t)row);
+    for (int32_t a = 0; a < A; ++a) {
+        for (int e = 0; e < row; ++e)
+            v[e] = layout == 0 ? head[(size_t)a * (size_t)row + (size_t)e] : head[(size_t)e * (size_t)A + (size_t)a];
+        int ok = 1;
+        for (int e = 0; e < row; ++e) ok &= finite_f(v[e]);
+        if (!ok) continue;
+        if (!(v[2] > 0.0f) || !(v[3] > 0.0f)) continue;
+        const float* cv = v + nbox;
+        float so = 1.0f; /* objectness factor; absent in the planes layout */
+        if (layout == 0) so = logits ? orc_sigmoid(v[4]) : v[4];
+        float hw = 0.5f * v[2], hh = 0.5f * v[3];
+        orc_det_t d;
+        d.x1 = v[0] - hw; d.y1 = v[1] - hh; d.x2 = v[0] + hw; d.y2 = v[1] + hh;
+        d.anchor = a; d._pad = 0;
+        if (!multi_label) {
+            int best = 0;
+            float bv = cv[0];
+            for (int k = 1; k < C; ++k)
+                if (cv[k] > bv) { bv = cv[k]; best = k; }
+            float sc = logits ? orc_sigmoid(bv) : bv;
+            float score = layout == 0 ? so * sc : sc;
+            if (!(score > conf)) continue;
+            d.score = score; d.cls = best;
+            if (n < cap) out[n] = d;
+            n++;
+        } else {
+            for (int k = 0; k < C; ++k) {
+                float sc = logits ? orc_sigmoid(cv[k]) : cv[k];
+                float score = layout == 0 ? so * sc : sc;
+                if (!(score > conf)) continue;
+                d.score = score; d.cls = k;
+                if (n < cap) out[n] = d;
+                n++;
+            }
+        }
+    }
+    free(v);
+    return n;
+}
+
+/* R4: total order -- score descending, then anchor ascending; candidates of one anchor
+ * (multi-label decode) that tie in score go by ascending class. */
 static int cand_cmp(const void* pa, const void* pb) {
     const orc_det_t* a = (const orc_det_t*)pa;
     const orc_det_t* b = (const orc_det_t*)pb;
     if (a->score > b->score) return -1;
     if (a->score < b->score) return 1;
-    return (a->anchor > b->anchor) - (a->anchor < b->anchor);
+    if (a->anchor != b->anchor) return (a->anchor > b->anchor) - (a->anchor < b->anchor);
+    return (a->cls > b->cls) - (a->cls < b->cls);
 }
 void orc_sort(orc_det_t* c, int32_t n) { qsort(c, (size_t)n, sizeof(orc_det_t), cand_cmp); }
 
@@ -298,6 +357,27 @@ int32_t orc_postprocess_image_ex(const float* head, int32_t A, int32_t C, int32_
     orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * (size_t)(A > 0 ? A : 1));
     int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
     int32_t n = orc_decode(head, A, C, logits, conf, cand);
+    orc_sort(cand, n);
+    int32_t k = orc_nms_ex(cand, n, iou_thr, max_det, agnostic, keep);
+    for (int32_t t = 0; t < k; ++t) {
+        dets[t] = cand[keep[t]];
+        orc_scale_back(&dets[t], w, h, S);
+    }
+    if (n_cand) *n_cand = n;
+    free(cand);
+    free(keep);
+    return k;
+}
+
+/* R3..R6 for one image with the decode variants of orc_decode_ex. */
+int32_t orc_postprocess_image_v2(const float* head, int32_t A, int32_t C, int32_t logits, float conf,
+                                 float iou_thr, int32_t max_det, int32_t w, int32_t h, int32_t S,
+                                 int32_t agnostic, int32_t layout, int32_t multi_label, orc_det_t* dets,
+                                 int32_t* n_cand) {
+    const size_t cap = (size_t)(A > 0 ? A : 1) * (size_t)(multi_label ? (C > 0 ? C : 1) : 1);
+    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * cap);
+    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
+    int32_t n = orc_decode_ex(head, A, C, logits, conf, layout, multi_label, cand, (int32_t)cap);
     orc_sort(cand, n);
     int32_t k = orc_nms_ex(cand, n, iou_thr, max_det, agnostic, keep);
     for (int32_t t = 0; t < k; ++t) {

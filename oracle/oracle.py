@@ -50,6 +50,10 @@ def _load():
     lib.orc_sigmoid.restype = f32
     lib.orc_decode.argtypes = [vp, i32, i32, i32, f32, vp]
     lib.orc_decode.restype = i32
+    lib.orc_decode_ex.argtypes = [vp, i32, i32, i32, f32, i32, i32, vp, i32]
+    lib.orc_decode_ex.restype = i32
+    lib.orc_postprocess_image_v2.argtypes = [vp, i32, i32, i32, f32, f32, i32, i32, i32, i32, i32, i32, i32, vp, vp]
+    lib.orc_postprocess_image_v2.restype = i32
     lib.orc_sort.argtypes = [vp, i32]
     lib.orc_sort.restype = None
     lib.orc_iou.argtypes = [vp, vp]
@@ -132,12 +136,31 @@ def sigmoid(x) -> np.ndarray:
     return out.reshape(arr.shape)
 
 
-def decode(head: np.ndarray, logits: bool = True, conf: float = 0.25) -> np.ndarray:
-    """head float32 [A, 5 + C] -> candidates (DET_DTYPE) in anchor order, letterbox pixels."""
+LAYOUTS = {"rows": 0, "planes": 1}
+
+
+def _head_dims(h: np.ndarray, layout: str) -> Tuple[int, int]:
+    """(A, C) of one image's head: rows [A, 5 + C] or planes [4 + C, A]."""
+    if layout == "rows":
+        return h.shape[0], h.shape[1] - 5
+    return h.shape[1], h.shape[0] - 4
+
+
+def decode(head: np.ndarray, logits: bool = True, conf: float = 0.25, layout: str = "rows",
+           multi_label: bool = False) -> np.ndarray:
+    """One image's head (rows [A, 5 + C] or planes [4 + C, A], float32) -> candidates (DET_DTYPE)
+    in (anchor, class) order, letterbox pixels."""
     h = np.ascontiguousarray(head, dtype=np.float32)
-    a, row = h.shape
-    out = np.zeros(max(a, 1), dtype=DET_DTYPE)
-    n = _load().orc_decode(_ptr(h), a, row - 5, 1 if logits else 0, np.float32(conf), _ptr(out))
+    if layout == "rows" and not multi_label:
+        a, row = h.shape
+        out = np.zeros(max(a, 1), dtype=DET_DTYPE)
+        n = _load().orc_decode(_ptr(h), a, row - 5, 1 if logits else 0, np.float32(conf), _ptr(out))
+        return out[:n].copy()
+    a, c = _head_dims(h, layout)
+    cap = max(a * (c if multi_label else 1), 1)
+    out = np.zeros(cap, dtype=DET_DTYPE)
+    n = _load().orc_decode_ex(_ptr(h), a, c, 1 if logits else 0, np.float32(conf), LAYOUTS[layout],
+                              1 if multi_label else 0, _ptr(out), cap)
     return out[:n].copy()
 
 
@@ -171,15 +194,23 @@ def scale_back(dets: np.ndarray, w: int, h: int, s: int) -> np.ndarray:
 
 
 def postprocess_image(head: np.ndarray, w: int, h: int, s: int, logits: bool = True,
-                      conf: float = 0.25, iou_thr: float = 0.45, max_det: int = 300, agnostic: bool = False):
-    """head [A, 5+C] -> (dets in frame pixels [kept], candidate count)."""
+                      conf: float = 0.25, iou_thr: float = 0.45, max_det: int = 300, agnostic: bool = False,
+                      layout: str = "rows", multi_label: bool = False):
+    """One image's head (rows [A, 5+C] or planes [4+C, A]) -> (dets in frame pixels [kept],
+    candidate count)."""
     hd = np.ascontiguousarray(head, dtype=np.float32)
-    a, row = hd.shape
     dets = np.zeros(max(max_det, 1), dtype=DET_DTYPE)
     ncand = np.zeros(1, dtype=np.int32)
-    k = _load().orc_postprocess_image_ex(_ptr(hd), a, row - 5, 1 if logits else 0, np.float32(conf),
-                                         np.float32(iou_thr), max_det, w, h, s, 1 if agnostic else 0,
-                                         _ptr(dets), _ptr(ncand))
+    if layout == "rows" and not multi_label:
+        a, row = hd.shape
+        k = _load().orc_postprocess_image_ex(_ptr(hd), a, row - 5, 1 if logits else 0, np.float32(conf),
+                                             np.float32(iou_thr), max_det, w, h, s, 1 if agnostic else 0,
+                                             _ptr(dets), _ptr(ncand))
+    else:
+        a, c = _head_dims(hd, layout)
+        k = _load().orc_postprocess_image_v2(_ptr(hd), a, c, 1 if logits else 0, np.float32(conf),
+                                             np.float32(iou_thr), max_det, w, h, s, 1 if agnostic else 0,
+                                             LAYOUTS[layout], 1 if multi_label else 0, _ptr(dets), _ptr(ncand))
     return dets[:k].copy(), int(ncand[0])
 
 
@@ -251,7 +282,8 @@ def run_stage(frames: Sequence[np.ndarray], sizes: Sequence[Tuple[int, int]], he
               conf: float = 0.25, iou_thr: float = 0.45, max_det: int = 300, pad_value: int = 114,
               swap_rb: bool = True, class_masks: Optional[Sequence[Sequence[int]]] = None,
               do_letterbox: bool = True, do_crops: bool = True, max_crops: Optional[int] = None,
-              threads: int = 1, agnostic: bool = False) -> StageResult:
+              threads: int = 1, agnostic: bool = False, layout: str = "rows",
+              multi_label: bool = False) -> StageResult:
     """Whole stage over one batch, frame by frame (optionally a thread per frame; the C
     routines release the GIL).  max_crops bounds the crops rendered per branch."""
     n = len(frames)
@@ -265,7 +297,7 @@ def run_stage(frames: Sequence[np.ndarray], sizes: Sequence[Tuple[int, int]], he
         w, h = sizes[i]
         if do_letterbox:
             det_in[i] = letterbox(frames[i], w, h, s, pad_value, swap_rb)
-        d, nc = postprocess_image(head[i], w, h, s, logits, conf, iou_thr, max_det, agnostic)
+        d, nc = postprocess_image(head[i], w, h, s, logits, conf, iou_thr, max_det, agnostic, layout, multi_label)
         dets[i, : len(d)] = d
         counts[i] = len(d)
         ncand[i] = nc

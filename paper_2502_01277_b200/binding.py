@@ -34,6 +34,11 @@ OCTO_STATUS_NONFINITE = 0x1
 OCTO_STATUS_TRUNCATED = 0x2
 OCTO_STATUS_COPY_TIMEOUT = 0x4
 OCTO_STATUS_BIG_NMS = 0x8
+OCTO_STATUS_CAND_OVERFLOW = 0x10
+
+OCTO_HEAD_ROWS = 0
+OCTO_HEAD_PLANES = 1
+HEAD_LAYOUTS = {"rows": OCTO_HEAD_ROWS, "planes": OCTO_HEAD_PLANES}
 
 EXPORTS = (
     "octo_stage_create", "octo_stage_destroy", "octo_preprocess_batch", "octo_postprocess_batch",
@@ -46,7 +51,9 @@ EXPORTS = (
 
 
 class BranchCfg(ctypes.Structure):
-    _fields_ = [("out_w", ctypes.c_int32), ("out_h", ctypes.c_int32), ("class_mask", ctypes.c_uint32 * 4)]
+    _fields_ = [("out_w", ctypes.c_int32), ("out_h", ctypes.c_int32), ("class_mask", ctypes.c_uint32 * 4),
+                ("keep_aspect", ctypes.c_int32), ("normalize", ctypes.c_int32),
+                ("mean", ctypes.c_float * 3), ("std", ctypes.c_float * 3)]
 
 
 class StageConfig(ctypes.Structure):
@@ -56,6 +63,7 @@ class StageConfig(ctypes.Structure):
         ("head_is_logits", ctypes.c_int32), ("conf_thresh", ctypes.c_float),
         ("iou_thresh", ctypes.c_float), ("max_det", ctypes.c_int32), ("pad_value", ctypes.c_int32),
         ("swap_rb", ctypes.c_int32), ("num_branches", ctypes.c_int32), ("class_agnostic", ctypes.c_int32),
+        ("head_layout", ctypes.c_int32), ("multi_label", ctypes.c_int32),
         ("branch", BranchCfg * OCTO_MAX_BRANCHES),
     ]
 
@@ -169,7 +177,10 @@ def make_config(*, device: int = 0, net_size: int = 640, max_batch: int = 8, num
                 iou_thresh: float = 0.45, max_det: int = 300, pad_value: int = 114, swap_rb: bool = True,
                 branches: Sequence[Tuple[int, int]] = ((224, 224),),
                 class_masks: Optional[Sequence[Sequence[int]]] = None,
-                class_agnostic: bool = False) -> StageConfig:
+                class_agnostic: bool = False, head_layout: str = "rows",
+                multi_label: bool = False, crop_options: Optional[Sequence[Optional[dict]]] = None) -> StageConfig:
+    """crop_options: per branch None or a dict with any of keep_aspect (bool), mean and std
+    (three floats each, per output plane; giving them turns normalisation on)."""
     cfg = StageConfig()
     cfg.device, cfg.net_size, cfg.max_batch = device, net_size, max_batch
     cfg.num_anchors, cfg.num_classes = num_anchors, num_classes
@@ -178,11 +189,20 @@ def make_config(*, device: int = 0, net_size: int = 640, max_batch: int = 8, num
     cfg.max_det, cfg.pad_value, cfg.swap_rb = max_det, pad_value, 1 if swap_rb else 0
     cfg.num_branches = len(branches)
     cfg.class_agnostic = 1 if class_agnostic else 0
+    cfg.head_layout = HEAD_LAYOUTS[head_layout]
+    cfg.multi_label = 1 if multi_label else 0
     for b, (ow, oh) in enumerate(branches[:OCTO_MAX_BRANCHES]):
         cfg.branch[b].out_w, cfg.branch[b].out_h = ow, oh
         mask = class_masks[b] if class_masks is not None else (0xFFFFFFFF,) * 4
         for k in range(4):
             cfg.branch[b].class_mask[k] = int(mask[k]) & 0xFFFFFFFF
+        opt = (crop_options[b] if crop_options is not None else None) or {}
+        cfg.branch[b].keep_aspect = 1 if opt.get("keep_aspect") else 0
+        if "mean" in opt or "std" in opt:
+            cfg.branch[b].normalize = 1
+            for k in range(3):
+                cfg.branch[b].mean[k] = float(opt.get("mean", (0.0, 0.0, 0.0))[k])
+                cfg.branch[b].std[k] = float(opt.get("std", (1.0, 1.0, 1.0))[k])
     return cfg
 
 

@@ -8,7 +8,15 @@
 // sequence and appended to the image's key list with one atomic; the key carries class,
 // inverted score bits and anchor, so later steps need nothing else from this kernel and the
 // nondeterministic append order is erased by the sort.
+//
+// Variants.  Multi-label: a passing row yields one key per class whose own score exceeds the
+// threshold.  Planes layout [n, 4 + C, A] (anchor-free heads without objectness): consecutive
+// anchors are contiguous in every plane, so the scan is a dense, coalesced read of the C class
+// planes (the whole head must be read: the maximum over classes needs every value); the four
+// box planes are read only for anchors whose score passes.
 #include "octo_common.cuh"
+#include <cmath>
+
 #include "octo_kernels.h"
 
 namespace octo {
@@ -24,6 +32,13 @@ __device__ __forceinline__ float ld_obj(const float* p) {
     return v;
 }
 
+// Candidate key: class | inverted score bits | anchor (ascending key = descending score, then
+// ascending anchor inside a class).
+__device__ __forceinline__ unsigned long long make_key(int cls, float score, int anchor) {
+    return ((unsigned long long)(unsigned)cls << 57) | ((unsigned long long)(~__float_as_uint(score)) << kKeyAnchorBits) |
+           (unsigned long long)(unsigned)anchor;
+}
+
 // kDecPerThread anchors per thread: 4 for large batches, 1 when the grid would otherwise be
 // too small to cover the SMs.
 template <int kDecPerThread>
@@ -31,9 +46,11 @@ __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf, int key_stride,
               unsigned long long* __restrict__ keys, int* __restrict__ cand_count,
               unsigned int* __restrict__ status) {
-    // mode bit 0: obj / class values are logits; bit 1: class-agnostic NMS (key class field 0)
+    // mode bit 0: obj / class values are logits; bit 1: class-agnostic NMS (key class field 0);
+    // bit 2: multi-label candidates
     const int logits = mode & 1;
     const bool agnostic = (mode & 2) != 0;
+    const bool multi = (mode & 4) != 0;
     const int img = blockIdx.y;
     const int row_len = 5 + C;
     const float* __restrict__ hbase = head + (size_t)img * (size_t)A * (size_t)row_len;
@@ -65,12 +82,13 @@ decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf
             const int ra = a_warp + u * 32 + src;
             const float* __restrict__ row = hbase + (size_t)ra * row_len;
             // the warp reads the row; lane l holds elements l, l+32, l+64, ...
+            constexpr int kRowRegs = (5 + 128 + 31) / 32;
             bool fin = true;
             float best = -INFINITY;
             int best_k = 0x7fffffff;
             float e0 = 0.0f;
 #pragma unroll
-            for (int j = 0; j < (5 + 128 + 31) / 32; ++j) {
+            for (int j = 0; j < kRowRegs; ++j) {
                 const int e = lane + 32 * j;
                 if (e < row_len) {
                     const float v = __ldg(row + e);
@@ -80,28 +98,53 @@ decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf
                 }
             }
             fin = __all_sync(0xffffffffu, fin);
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, best, off);
-                const int ok = __shfl_xor_sync(0xffffffffu, best_k, off);
-                if (ov > best || (ov == best && ok < best_k)) { best = ov; best_k = ok; }
-            }
-            const float cx = __shfl_sync(0xffffffffu, e0, 0);
-            const float cy = __shfl_sync(0xffffffffu, e0, 1);
             const float bw = __shfl_sync(0xffffffffu, e0, 2);
             const float bh = __shfl_sync(0xffffffffu, e0, 3);
             const float ob = __shfl_sync(0xffffffffu, e0, 4);
-            (void)cx; (void)cy;
             if (!fin) { nonfinite_seen = true; continue; }
-            if (lane == 0 && bw > 0.0f && bh > 0.0f) {
-                const float score = logits ? __fmul_rn(sigmoid_fixed(ob), sigmoid_fixed(best))
-                                           : __fmul_rn(ob, best);
-                if (score > conf) {
-                    const int slot = atomicAdd(cand_count + img, 1);
-                    const unsigned long long key = ((unsigned long long)(unsigned)(agnostic ? 0 : best_k) << 57) |
-                                                   ((unsigned long long)(~__float_as_uint(score)) << kKeyAnchorBits) |
-                                                   (unsigned long long)(unsigned)ra;
-                    if (slot < key_stride) keys[(size_t)img * key_stride + slot] = key;
+            if (!(bw > 0.0f && bh > 0.0f)) continue;
+            if (!multi) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) {
+                    const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+                    const int ok = __shfl_xor_sync(0xffffffffu, best_k, off);
+                    if (ov > best || (ov == best && ok < best_k)) { best = ov; best_k = ok; }
+                }
+                if (lane == 0) {
+                    const float score = logits ? __fmul_rn(sigmoid_fixed(ob), sigmoid_fixed(best))
+                                               : __fmul_rn(ob, best);
+                    if (score > conf) {
+                        const int slot = atomicAdd(cand_count + img, 1);
+                        if (slot < key_stride)
+                            keys[(size_t)img * key_stride + slot] = make_key(agnostic ? 0 : best_k, score, ra);
+                        else
+                            atomicOr(status, 0x10u);
+                    }
+                }
+            } else {
+                // one candidate per class whose own score passes; the keys of a row go out in
+                // groups of up to 32 with one counter update per group
+                const float so = logits ? sigmoid_fixed(ob) : ob;
+#pragma unroll
+                for (int j = 0; j < kRowRegs; ++j) {
+                    const int e = lane + 32 * j;
+                    float score = 0.0f;
+                    bool hit = false;
+                    if (e >= 5 && e < row_len) {
+                        const float v = __ldg(row + e);  // second pass over the row: an L1 hit
+                        score = __fmul_rn(so, logits ? sigmoid_fixed(v) : v);
+                        hit = score > conf;
+                    }
+                    const unsigned hits = __ballot_sync(0xffffffffu, hit);
+                    if (hits == 0u) continue;
+                    int base = 0;
+                    if (lane == 0) base = atomicAdd(cand_count + img, __popc(hits));
+                    base = __shfl_sync(0xffffffffu, base, 0);
+                    if (hit) {
+                        const int slot = base + __popc(hits & ((1u << lane) - 1u));
+                        if (slot < key_stride) keys[(size_t)img * key_stride + slot] = make_key(e - 5, score, ra);
+                        else atomicOr(status, 0x10u);
+                    }
                 }
             }
         }
@@ -109,19 +152,147 @@ decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf
     if (__any_sync(0xffffffffu, nonfinite_seen) && lane == 0) atomicOr(status, 0x1u);
 }
 
-cudaError_t launch_decode(const float* d_head, int n, int A, int C, int logits, float conf, int key_stride,
-                          unsigned long long* d_keys, int* d_cand_count, unsigned int* d_status,
-                          cudaStream_t stream) {
-    // d_cand_count is zero on entry: zeroed at stage creation and re-zeroed by the NMS kernel.
-    const int per_cta4 = kDecThreads * 4;
-    if ((long long)n * ((A + per_cta4 - 1) / per_cta4) >= 296) {
-        dim3 grid((A + per_cta4 - 1) / per_cta4, n);
-        decode_kernel<4><<<grid, kDecThreads, 0, stream>>>(d_head, A, C, logits, conf, key_stride, d_keys,
-                                                          d_cand_count, d_status);
+// Planes layout [n, 4 + C, A].  A CTA owns 32 * VEC consecutive anchors (VEC = 4 with 16-byte
+// loads when A is a multiple of 4, else 1).  Lane l of every warp reads anchors (32 * cta + l) *
+// VEC .., so a warp load covers consecutive addresses of one plane; the eight warps split the C
+// class planes between them (warp w takes classes w, w + 8, ...), which puts all loads of a
+// thread in flight at once, and leave their running first maxima in shared memory, where one
+// thread per anchor merges them.  For multi-label heads in logit form a value is only run
+// through the fixed logistic sequence when it lies above `pre`, a bound placed safely below
+// the threshold's logit, so that the common case costs one comparison per value.
+constexpr int kPlaneWarps = kDecThreads / 32;
+
+template <int VEC>
+__global__ void __launch_bounds__(kDecThreads)
+decode_planes_kernel(const float* __restrict__ head, int A, int C, int mode, float conf, float pre, int key_stride,
+                     unsigned long long* __restrict__ keys, int* __restrict__ cand_count,
+                     unsigned int* __restrict__ status) {
+    __shared__ float s_best[kPlaneWarps][32 * VEC];
+    __shared__ int s_k[kPlaneWarps][32 * VEC];
+    __shared__ unsigned s_flags[kPlaneWarps][32];  // bits 0..3: non-finite seen, 4..7: above `pre`
+    const int logits = mode & 1;
+    const bool agnostic = (mode & 2) != 0;
+    const bool multi = (mode & 4) != 0;
+    const int img = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float* __restrict__ hbase = head + (size_t)img * (size_t)(4 + C) * (size_t)A;
+    const int a0 = (blockIdx.x * 32 + lane) * VEC;
+
+    float best[VEC];
+    int best_k[VEC];
+    unsigned flags = 0u;
+#pragma unroll
+    for (int u = 0; u < VEC; ++u) { best[u] = -INFINITY; best_k[u] = 0x7fffffff; }
+    if (a0 < A) {
+        const float* __restrict__ cls0 = hbase + (size_t)4 * A + a0;
+#pragma unroll 4
+        for (int k = warp; k < C; k += kPlaneWarps) {
+            float v[VEC];
+            if (VEC == 4) {
+                const float4 q = __ldg(reinterpret_cast<const float4*>(cls0 + (size_t)k * A));
+                v[0] = q.x; v[1 % VEC] = q.y; v[2 % VEC] = q.z; v[3 % VEC] = q.w;
+            } else {
+                v[0] = __ldg(cls0 + (size_t)k * A);
+            }
+#pragma unroll
+            for (int u = 0; u < VEC; ++u) {
+                if (!finite_f(v[u])) flags |= 1u << u;
+                if (v[u] > best[u]) { best[u] = v[u]; best_k[u] = k; }
+                if (multi && v[u] > pre) flags |= 16u << u;
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < VEC; ++u) {
+        s_best[warp][lane * VEC + u] = best[u];
+        s_k[warp][lane * VEC + u] = best_k[u];
+    }
+    s_flags[warp][lane] = flags;
+    __syncthreads();
+
+    // one thread per anchor of the CTA
+    if (threadIdx.x >= 32 * VEC) return;
+    const int t = threadIdx.x, u = t % VEC;
+    const int anchor = blockIdx.x * 32 * VEC + t;
+    if (anchor >= A) return;
+    float bv = -INFINITY;
+    int bk = 0x7fffffff;
+    unsigned fl = 0u;
+#pragma unroll
+    for (int w = 0; w < kPlaneWarps; ++w) {
+        const float v = s_best[w][t];
+        const int k = s_k[w][t];
+        if (v > bv || (v == bv && k < bk)) { bv = v; bk = k; }  // first maximum over all classes
+        fl |= s_flags[w][t / VEC];
+    }
+    const bool bad = (fl >> u) & 1u;
+    if (bad) atomicOr(status, 0x1u);
+    const float* __restrict__ bx = hbase + anchor;
+    auto box_ok = [&]() {  // finite box with w, h > 0
+        const float cx = __ldg(bx), cy = __ldg(bx + A), bw = __ldg(bx + 2 * (size_t)A), bh = __ldg(bx + 3 * (size_t)A);
+        if (!(finite_f(cx) && finite_f(cy) && finite_f(bw) && finite_f(bh))) { atomicOr(status, 0x1u); return false; }
+        return bw > 0.0f && bh > 0.0f;
+    };
+    auto emit = [&](int cls, float score) {
+        const int slot = atomicAdd(cand_count + img, 1);
+        if (slot < key_stride) keys[(size_t)img * key_stride + slot] = make_key(cls, score, anchor);
+        else atomicOr(status, 0x10u);
+    };
+    if (!multi) {
+        if (bad || bk == 0x7fffffff) return;
+        const float score = logits ? sigmoid_fixed(bv) : bv;
+        if (!(score > conf)) return;
+        if (!box_ok()) return;
+        emit(agnostic ? 0 : bk, score);
     } else {
-        dim3 grid((A + kDecThreads - 1) / kDecThreads, n);
-        decode_kernel<1><<<grid, kDecThreads, 0, stream>>>(d_head, A, C, logits, conf, key_stride, d_keys,
-                                                          d_cand_count, d_status);
+        // rare: walk the anchor's classes again (the values are in L1 / L2 by now)
+        if (bad || !((fl >> (4 + u)) & 1u)) return;
+        if (!box_ok()) return;
+        const float* __restrict__ cv = hbase + (size_t)4 * A + anchor;
+        for (int k = 0; k < C; ++k) {
+            const float v = __ldg(cv + (size_t)k * A);
+            if (!(v > pre)) continue;
+            const float score = logits ? sigmoid_fixed(v) : v;
+            if (score > conf) emit(k, score);
+        }
+    }
+}
+
+cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
+    // d_cand_count is zero on entry: zeroed at stage creation and re-zeroed by the NMS kernel.
+    const int mode = (a.logits ? 1 : 0) | (a.class_agnostic ? 2 : 0) | (a.multi_label ? 4 : 0);
+    if (a.layout == OCTO_HEAD_PLANES) {
+        // Multi-label prefilter in the head's own units: for probabilities the threshold itself;
+        // for logits the threshold's logit lowered by a margin that dwarfs the few-ulp error of
+        // the fixed logistic sequence (no prefilter where the logistic curve is too flat for that).
+        float pre = a.conf;
+        if (a.logits) {
+            pre = -INFINITY;
+            if (a.conf > 0.0f && a.conf <= 0.99f) {
+                const double t = log((double)a.conf / (1.0 - (double)a.conf));
+                pre = (float)(t - 1e-3 * (1.0 + fabs(t)));
+            }
+        }
+        if ((a.A & 3) == 0 && (reinterpret_cast<uintptr_t>(a.d_head) & 15) == 0) {
+            dim3 grid((a.A / 4 + 31) / 32, a.n);
+            decode_planes_kernel<4><<<grid, kDecThreads, 0, stream>>>(a.d_head, a.A, a.C, mode, a.conf, pre,
+                                                                     a.key_stride, a.d_keys, a.d_cand_count, a.d_status);
+        } else {
+            dim3 grid((a.A + 31) / 32, a.n);
+            decode_planes_kernel<1><<<grid, kDecThreads, 0, stream>>>(a.d_head, a.A, a.C, mode, a.conf, pre,
+                                                                     a.key_stride, a.d_keys, a.d_cand_count, a.d_status);
+        }
+        return cudaGetLastError();
+    }
+    const int per_cta4 = kDecThreads * 4;
+    if ((long long)a.n * ((a.A + per_cta4 - 1) / per_cta4) >= 296) {
+        dim3 grid((a.A + per_cta4 - 1) / per_cta4, a.n);
+        decode_kernel<4><<<grid, kDecThreads, 0, stream>>>(a.d_head, a.A, a.C, mode, a.conf, a.key_stride, a.d_keys,
+                                                          a.d_cand_count, a.d_status);
+    } else {
+        dim3 grid((a.A + kDecThreads - 1) / kDecThreads, a.n);
+        decode_kernel<1><<<grid, kDecThreads, 0, stream>>>(a.d_head, a.A, a.C, mode, a.conf, a.key_stride, a.d_keys,
+                                                          a.d_cand_count, a.d_status);
     }
     return cudaGetLastError();
 }

@@ -15,11 +15,24 @@ struct BranchMasks {
     uint32_t m[OCTO_MAX_BRANCHES][4];
 };
 
+struct DecodeArgs {
+    const float* d_head;
+    int n, A, C;
+    int layout;  // OCTO_HEAD_ROWS / OCTO_HEAD_PLANES
+    int logits, class_agnostic, multi_label;
+    float conf;
+    int key_stride;
+    unsigned long long* d_keys;
+    int* d_cand_count;
+    unsigned int* d_status;
+};
+
 struct NmsArgs {
     const FrameDesc* frames;  // host
     int n;
     const float* d_head;
     int A, C;
+    int layout;  // OCTO_HEAD_ROWS / OCTO_HEAD_PLANES
     float iou_thr;
     int max_det, key_stride;
     unsigned long long* d_keys;
@@ -58,9 +71,7 @@ cudaError_t prepare_crop();
 
 cudaError_t launch_letterbox(const FrameDesc* frames, int n, void* d_out, int S, int max_w, int pad_value,
                              int swap_rb, unsigned int* d_status, cudaStream_t stream);
-cudaError_t launch_decode(const float* d_head, int n, int A, int C, int logits, float conf, int key_stride,
-                          unsigned long long* d_keys, int* d_cand_count, unsigned int* d_status,
-                          cudaStream_t stream);
+cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
 cudaError_t launch_nms(const NmsArgs& a, cudaStream_t stream);
 cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream);  // batch assembler + crop-resize
 cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int bz, void* d_out, int out_w,

@@ -65,13 +65,15 @@ __device__ __forceinline__ void bitonic_range(unsigned long long* __restrict__ k
     if (BLOCK) __syncthreads(); else __syncwarp();
 }
 
-__device__ __forceinline__ float4 gather_box(const float* __restrict__ hrow) {
-    return box_corners(__ldg(hrow), __ldg(hrow + 1), __ldg(hrow + 2), __ldg(hrow + 3));
+// Box of one anchor; es = distance between consecutive values of an anchor (1 in the rows
+// layout, A in the planes layout).
+__device__ __forceinline__ float4 gather_box(const float* __restrict__ p, size_t es) {
+    return box_corners(__ldg(p), __ldg(p + es), __ldg(p + 2 * es), __ldg(p + 3 * es));
 }
 
 template <int CAP>
 __global__ void __launch_bounds__(kNmsThreads, 1)
-nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict__ head, int A, int C,
+nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict__ head, int A, int C, int layout,
            const IouTest iou_test, int max_det, int key_stride, unsigned long long* __restrict__ gkeys,
            float4* __restrict__ gboxes, int* __restrict__ cand_count, octo_det_rec* __restrict__ dets,
            int* __restrict__ counts, int num_branches, int class_agnostic,
@@ -84,11 +86,14 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
 
     const int img = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int row_len = 5 + C;
-    const float* __restrict__ hbase = head + (size_t)img * (size_t)A * (size_t)row_len;
+    // rows layout [A][5 + C] or planes layout [4 + C][A]
+    const int nbox = layout == OCTO_HEAD_PLANES ? 4 : 5;
+    const size_t es = layout == OCTO_HEAD_PLANES ? (size_t)A : 1;          // value to value
+    const size_t as = layout == OCTO_HEAD_PLANES ? 1 : (size_t)(nbox + C);  // anchor to anchor
+    const float* __restrict__ hbase = head + (size_t)img * (size_t)A * (size_t)(nbox + C);
 
     int cnt = cand_count[img];
-    cnt = min(cnt, min(A, key_stride));
+    cnt = min(cnt, key_stride);
     if (threadIdx.x < 128) { seg_cnt[threadIdx.x] = 0; nkept[threadIdx.x] = 0; }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -189,7 +194,7 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
         }
         for (int p = s + lane; p < e; p += 32) {
             const int anchor = (int)(keys[p] & ((1ull << kKeyAnchorBits) - 1));
-            boxes[p] = gather_box(hbase + (size_t)anchor * row_len);
+            boxes[p] = gather_box(hbase + (size_t)anchor * as, es);
         }
         __syncwarp();
         int nk = 0;  // survivors of this class, compacted at [s, s + nk)
@@ -318,14 +323,14 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
         int cls = (int)(g & 127u);
         const int anchor = (int)((g >> 7) & ((1ull << kKeyAnchorBits) - 1));
         const float score = __uint_as_float(~(unsigned)(g >> 32));
-        const float4 b = gather_box(hbase + (size_t)anchor * row_len);
+        const float4 b = gather_box(hbase + (size_t)anchor * as, es);
         if (class_agnostic) {
             // NMS ran with every candidate in class 0: recover the real class (first maximum)
-            const float* __restrict__ cv = hbase + (size_t)anchor * row_len + 5;
+            const float* __restrict__ cv = hbase + (size_t)anchor * as + (size_t)nbox * es;
             float best = __ldg(cv);
             cls = 0;
             for (int k = 1; k < C; ++k) {
-                const float v = __ldg(cv + k);
+                const float v = __ldg(cv + (size_t)k * es);
                 if (v > best) { best = v; cls = k; }
             }
         }
@@ -389,7 +394,7 @@ static cudaError_t launch_cap(const NmsArgs& a, cudaStream_t stream) {
     unsigned int up_bits;
     memcpy(&up_bits, &up, sizeof(up_bits));
     iou_test.tie_up = (up_bits & 1u) == 0u ? 1 : 0;
-    nms_kernel<CAP><<<a.n, kNmsThreads, smem, stream>>>(tab, a.d_head, a.A, a.C, iou_test, a.max_det, a.key_stride,
+    nms_kernel<CAP><<<a.n, kNmsThreads, smem, stream>>>(tab, a.d_head, a.A, a.C, a.layout, iou_test, a.max_det, a.key_stride,
                                                        a.d_keys, a.d_boxes, a.d_cand_count,
                                                        reinterpret_cast<octo_det_rec*>(a.d_dets), a.d_counts,
                                                        a.num_branches, a.class_agnostic, a.masks, a.d_bcount, a.d_bidx, a.max_batch,

@@ -136,8 +136,15 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
     int key_stride = 2;
     while (key_stride < num_anchors) key_stride <<= 1;  // <= kStaticMaxAnchors
 
-    e = launch_decode(d_head, 1, num_anchors, num_classes, head_is_logits, conf_thresh, key_stride, d_keys, d_cand,
-                      &d_ctr->status, stream);
+    DecodeArgs da;
+    da.d_head = d_head;
+    da.n = 1; da.A = num_anchors; da.C = num_classes;
+    da.layout = OCTO_HEAD_ROWS;
+    da.logits = head_is_logits; da.class_agnostic = 0; da.multi_label = 0;
+    da.conf = conf_thresh;
+    da.key_stride = key_stride;
+    da.d_keys = d_keys; da.d_cand_count = d_cand; da.d_status = &d_ctr->status;
+    e = launch_decode(da, stream);
     if (e != cudaSuccess) return OCTO_E_CUDA;
 
     FrameDesc fd;
@@ -148,6 +155,7 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
     a.d_head = d_head;
     a.A = num_anchors;
     a.C = num_classes;
+    a.layout = OCTO_HEAD_ROWS;
     a.iou_thr = iou_thresh;
     a.max_det = max_det;
     a.key_stride = key_stride;

@@ -1,6 +1,7 @@
 // Stage object and the extern "C" boundary (see include/octo.h for the contract).
 #include <cstdio>
 #include <cstdlib>
+#include <cmath>
 #include <cstring>
 #include <new>
 
@@ -54,10 +55,21 @@ static int validate_config(const octo_stage_config_t* c) {
     if (c->swap_rb != 0 && c->swap_rb != 1) return OCTO_E_INVALID_ARG;
     if (c->num_branches < 1 || c->num_branches > OCTO_MAX_BRANCHES) return OCTO_E_INVALID_ARG;
     if (c->class_agnostic != 0 && c->class_agnostic != 1) return OCTO_E_INVALID_ARG;
+    if (c->head_layout != OCTO_HEAD_ROWS && c->head_layout != OCTO_HEAD_PLANES) return OCTO_E_INVALID_ARG;
+    if (c->multi_label != 0 && c->multi_label != 1) return OCTO_E_INVALID_ARG;
+    if (c->multi_label && c->class_agnostic) return OCTO_E_INVALID_ARG;
     for (int b = 0; b < c->num_branches; ++b) {
         const octo_branch_cfg_t& br = c->branch[b];
         if (br.out_w < 8 || br.out_w > 2048 || (br.out_w & 7)) return OCTO_E_INVALID_ARG;
         if (br.out_h < 1 || br.out_h > 2048) return OCTO_E_INVALID_ARG;
+        if (br.keep_aspect != 0 && br.keep_aspect != 1) return OCTO_E_INVALID_ARG;
+        if (br.normalize != 0 && br.normalize != 1) return OCTO_E_INVALID_ARG;
+        if (br.normalize) {
+            for (int k = 0; k < 3; ++k) {
+                if (!(fabsf(br.mean[k]) <= 1e6f)) return OCTO_E_INVALID_ARG;          // finite, sane
+                if (!(br.std[k] >= 1e-6f) || !(br.std[k] <= 1e6f)) return OCTO_E_INVALID_ARG;
+            }
+        }
     }
     return OCTO_OK;
 }
@@ -103,6 +115,7 @@ extern "C" int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** 
     OCTO_CUDA(cudaDeviceGetAttribute(&st->sm_count, cudaDevAttrMultiProcessorCount, cfg->device));
     int ks = 2;
     while (ks < cfg->num_anchors) ks <<= 1;
+    if (cfg->multi_label) ks <<= 1;  // an anchor can yield several candidates
     st->key_stride = ks;
 
     const size_t mb = (size_t)cfg->max_batch;
@@ -251,8 +264,15 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     OCTO_CUDA(cudaSetDevice(c.device));
     {
         ScopedKernelTimer t(st, OCTO_K_DECODE, stream);
-        OCTO_CUDA(launch_decode(d_head, n, c.num_anchors, c.num_classes, c.head_is_logits | (c.class_agnostic << 1), c.conf_thresh,
-                                st->key_stride, st->d_keys, st->d_cand_count, &st->d_ctr->status, stream));
+        DecodeArgs da;
+        da.d_head = d_head;
+        da.n = n; da.A = c.num_anchors; da.C = c.num_classes;
+        da.layout = c.head_layout;
+        da.logits = c.head_is_logits; da.class_agnostic = c.class_agnostic; da.multi_label = c.multi_label;
+        da.conf = c.conf_thresh;
+        da.key_stride = st->key_stride;
+        da.d_keys = st->d_keys; da.d_cand_count = st->d_cand_count; da.d_status = &st->d_ctr->status;
+        OCTO_CUDA(launch_decode(da, stream));
     }
     st->launches += 1;
     NmsArgs a;
@@ -261,6 +281,7 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     a.d_head = d_head;
     a.A = c.num_anchors;
     a.C = c.num_classes;
+    a.layout = c.head_layout;
     a.iou_thr = c.iou_thresh;
     a.max_det = c.max_det;
     a.key_stride = st->key_stride;

@@ -31,7 +31,8 @@ def upload_frames(frames: Sequence[np.ndarray], device="cuda:0") -> List[torch.T
 def make_stage(wl, max_batch: int, **over) -> "octo.Stage":
     kw = dict(net_size=wl.net_size, max_batch=max_batch, num_anchors=wl.num_anchors,
               num_classes=wl.num_classes, head_is_logits=wl.logits, conf_thresh=wl.conf_thresh,
-              iou_thresh=wl.iou_thresh, max_det=wl.max_det, branches=wl.branches)
+              iou_thresh=wl.iou_thresh, max_det=wl.max_det, branches=wl.branches,
+              head_layout=wl.head_layout, multi_label=wl.multi_label)
     kw.update(over)
     return octo.Stage(**kw)
 

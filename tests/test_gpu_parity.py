@@ -51,7 +51,8 @@ def _check_branch(res, ref, b, first_item=0, max_items=None, crops_checked=None)
 
 def _oracle(b, **kw):
     wl = b.workload
-    args = dict(logits=wl.logits, conf=wl.conf_thresh, iou_thr=wl.iou_thresh, max_det=wl.max_det, threads=THREADS)
+    args = dict(logits=wl.logits, conf=wl.conf_thresh, iou_thr=wl.iou_thresh, max_det=wl.max_det, threads=THREADS,
+                layout=wl.head_layout, multi_label=wl.multi_label)
     args.update(kw)
     return oracle.run_stage(b.frames, b.sizes, b.head, wl.net_size, wl.branches, **args)
 

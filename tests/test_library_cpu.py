@@ -40,8 +40,8 @@ def test_version_and_strerror():
 
 
 def test_struct_layouts_match_header():
-    assert ctypes.sizeof(binding.BranchCfg) == 24
-    assert ctypes.sizeof(binding.StageConfig) == 13 * 4 + 4 * 24
+    assert ctypes.sizeof(binding.BranchCfg) == 56
+    assert ctypes.sizeof(binding.StageConfig) == 15 * 4 + 4 * 56
     assert ctypes.sizeof(binding.Frame) == 24
     assert binding.DET_DTYPE.itemsize == 32 and binding.ITEM_DTYPE.itemsize == 32
     assert ctypes.sizeof(binding.StageStats) == 40
@@ -52,7 +52,7 @@ def test_struct_layouts_match_header():
     ("num_anchors", 0), ("num_anchors", (1 << 24) + 1), ("num_classes", 0), ("num_classes", 129),
     ("head_is_logits", 2), ("conf_thresh", -0.1), ("conf_thresh", float("nan")), ("iou_thresh", 1.5),
     ("max_det", 0), ("pad_value", 256), ("pad_value", -1), ("swap_rb", 3), ("num_branches", 0),
-    ("num_branches", 5), ("device", -1),
+    ("num_branches", 5), ("device", -1), ("head_layout", 2), ("multi_label", 2), ("class_agnostic", 2),
 ])
 def test_create_rejects_bad_config_before_any_cuda_call(field, value):
     cfg = octo.make_config()

@@ -81,10 +81,15 @@ class Workload:
     # canvas rows [lo, hi) in which raised boxes are placed so that crops land on image
     # content (rows 140..500 hold a 16:9 frame on a 640 canvas); a recipe constant
     box_rows: Tuple[float, float] = (140.0, 500.0)
+    # "rows": head [N, A, 5 + C] with an objectness column; "planes": anchor-free head
+    # [N, 4 + C, A] (one prediction per grid cell, no objectness column)
+    head_layout: str = "rows"
+    multi_label: bool = False
+    bg_mean: float = -4.0  # mean of the background obj / class logits
 
     @property
     def num_anchors(self) -> int:
-        return num_anchors(self.net_size)
+        return num_anchors(self.net_size) // (3 if self.head_layout == "planes" else 1)
 
 
 WORKLOADS = {
@@ -99,6 +104,11 @@ WORKLOADS = {
                           items_per_frame=1000),
     "sweep": Workload("sweep", 4, 640, ((1920, 1080),), 64, "smooth", 200, 25, (40.0, 200.0),
                       0.15, (0.8, 1.25), 300, ((224, 224),)),
+    # decode variant: the sweep recipe with an anchor-free head in planes layout.  Without an
+    # objectness factor the score is the class value alone, so the background class logits sit
+    # lower (-7) to keep background candidates as rare as in the other recipes.
+    "anchor_free": Workload("anchor_free", 5, 640, ((1920, 1080),), 64, "smooth", 200, 25, (40.0, 200.0),
+                            0.15, (0.8, 1.25), 300, ((224, 224),), head_layout="planes", bg_mean=-7.0),
 }
 
 
@@ -107,7 +117,7 @@ class Batch:
     workload: Workload
     frames: List[np.ndarray]  # each uint8 [h, pitch]; pixel (y, x) = row[3x : 3x+3] in B, G, R
     sizes: List[Tuple[int, int]]  # (w, h) per frame
-    head: np.ndarray  # float32 [N, A, 5 + C]
+    head: np.ndarray  # float32 [N, A, 5 + C] (rows layout) or [N, 4 + C, A] (planes layout)
     first_frame: int = 0
     meta: dict = field(default_factory=dict)
 
@@ -139,7 +149,8 @@ def make_batch(name_or_workload, batch: Optional[int] = None, first_frame: int =
         else:
             sizes.append(wl.frame_sizes[lib.wl_coin(wl.seed, gi) % len(wl.frame_sizes)])
     frames = [np.empty((h, _pitch(w)), dtype=np.uint8) for (w, h) in sizes]
-    head = np.empty((n, a, 5 + c), dtype=np.float32)
+    planes = wl.head_layout == "planes"
+    head = np.empty((n, 4 + c, a) if planes else (n, a, 5 + c), dtype=np.float32)
     u8p = ctypes.POINTER(ctypes.c_uint8)
     f32p = ctypes.POINTER(ctypes.c_float)
     fgen = lib.wl_frame_uniform if wl.frame_kind == "uniform" else lib.wl_frame_smooth
@@ -149,10 +160,13 @@ def make_batch(name_or_workload, batch: Optional[int] = None, first_frame: int =
         w, h = sizes[i]
         fgen(wl.seed, gi, w, h, frames[i].shape[1], frames[i].ctypes.data_as(u8p))
         y_lo, y_hi = wl.box_rows
+        rows = np.empty((a, 5 + c), dtype=np.float32) if planes else head[i]
         lib.wl_head(wl.seed, gi, s, a, c, wl.n_raised, wl.n_groups, y_lo, y_hi,
                     wl.size_range[0], wl.size_range[1], wl.jitter, wl.scale_range[0],
-                    wl.scale_range[1], -4.0, 2.0, 0.5, 1 if wl.logits else 0,
-                    head[i].ctypes.data_as(f32p))
+                    wl.scale_range[1], wl.bg_mean, 2.0, 0.5, 1 if wl.logits else 0,
+                    rows.ctypes.data_as(f32p))
+        if planes:
+            head[i] = rows_to_planes(rows)
 
     nthreads = threads or min(n, os.cpu_count() or 1)
     if nthreads <= 1 or n == 1:
@@ -162,6 +176,11 @@ def make_batch(name_or_workload, batch: Optional[int] = None, first_frame: int =
         with ThreadPoolExecutor(max_workers=nthreads) as ex:
             list(ex.map(one, range(n)))
     return Batch(wl, frames, sizes, head, first_frame)
+
+
+def rows_to_planes(rows: np.ndarray) -> np.ndarray:
+    """Layout change only: rows [A, 5 + C] -> planes [4 + C, A] with the objectness column dropped."""
+    return np.ascontiguousarray(np.concatenate([rows[:, :4], rows[:, 5:]], axis=1).T)
 
 
 def make_heads(seed: int, n: int, net_size: int, num_classes: int = 80, n_raised: int = 10, n_groups: int = 4,
