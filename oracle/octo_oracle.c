@@ -444,6 +444,59 @@ void orc_crop(const uint8_t* img, int32_t w, int32_t h, int32_t pitch, const orc
     free(tmp);
 }
 
+/* R7 variants (branch options).
+ *   keep_aspect: the cw x ch rectangle keeps its shape inside the ow x oh slot.  The side with
+ *     the larger ratio fills the slot: if ow*ch <= oh*cw then nw = ow and nh = ch*ow/cw rounded
+ *     half-up in exact integer arithmetic (at least 1), else nh = oh and nw likewise; the image
+ *     is centred, an odd remainder puts the extra canvas pixel right / bottom (the letterbox
+ *     rule of R1 on a rectangular canvas); the canvas holds pad_value.
+ *   normalize: every output value v (= raw / 255, pixels and canvas alike) becomes
+ *     (v - mean[p]) / std[p] for output plane p, in double, before the single rounding to half.
+ * geom receives {nw, nh, pad_l, pad_t}. */
+void orc_fit_geometry(int32_t cw, int32_t ch, int32_t ow, int32_t oh, int32_t* geom) {
+    int64_t CW = cw, CH = ch, OW = ow, OH = oh, nw, nh;
+    if (OW * CH <= OH * CW) {
+        nw = OW;
+        nh = (2 * CH * OW + CW) / (2 * CW);
+        if (nh < 1) nh = 1;
+    } else {
+        nh = OH;
+        nw = (2 * CW * OH + CH) / (2 * CH);
+        if (nw < 1) nw = 1;
+    }
+    geom[0] = (int32_t)nw;
+    geom[1] = (int32_t)nh;
+    geom[2] = (int32_t)((OW - nw) / 2);
+    geom[3] = (int32_t)((OH - nh) / 2);
+}
+
+void orc_crop_ex(const uint8_t* img, int32_t w, int32_t h, int32_t pitch, const orc_det_t* d,
+                 int32_t ow, int32_t oh, int32_t swap_rb, int32_t keep_aspect, int32_t pad_value,
+                 int32_t normalize, const float* mean, const float* std, uint16_t* out) {
+    int32_t r[4], g[4];
+    orc_crop_rect(d, w, h, r);
+    const int32_t cw = r[2] - r[0], ch = r[3] - r[1];
+    g[0] = ow; g[1] = oh; g[2] = 0; g[3] = 0;
+    if (keep_aspect) orc_fit_geometry(cw, ch, ow, oh, g);
+    const int32_t nw = g[0], nh = g[1], pl = g[2], pt = g[3];
+    double* tmp = (double*)malloc(sizeof(double) * 3 * (size_t)nw * (size_t)nh);
+    orc_resize_f64(img, pitch, r[0], r[1], cw, ch, nw, nh, tmp);
+    size_t plane = (size_t)ow * (size_t)oh;
+    for (int p = 0; p < 3; ++p) {
+        int c = swap_rb ? 2 - p : p;
+        double m = normalize ? (double)mean[p] : 0.0, sd = normalize ? (double)std[p] : 1.0;
+        uint16_t fill = orc_f64_to_half(((double)pad_value / 255.0 - m) / sd);
+        for (size_t i = 0; i < plane; ++i) out[(size_t)p * plane + i] = fill;
+        for (int y = 0; y < nh; ++y)
+            for (int x = 0; x < nw; ++x) {
+                double v = tmp[((size_t)c * (size_t)nh + (size_t)y) * (size_t)nw + (size_t)x] / 255.0;
+                out[(size_t)p * plane + (size_t)(pt + y) * (size_t)ow + (size_t)(pl + x)] =
+                    orc_f64_to_half((v - m) / sd);
+            }
+    }
+    free(tmp);
+}
+
 /* R8: batch assembler for one branch.  m_n = number of frame n's kept detections whose
  * class bit is set in class_mask (128 bits, bit k of word k/32); offsets = exclusive prefix
  * sum, offsets[N] = total.  Item offsets[n]+j is the j-th such detection of frame n in NMS

@@ -74,6 +74,10 @@ def _load():
     lib.orc_crop_rect.restype = None
     lib.orc_crop.argtypes = [vp, i32, i32, i32, vp, i32, i32, i32, vp]
     lib.orc_crop.restype = None
+    lib.orc_fit_geometry.argtypes = [i32, i32, i32, i32, vp]
+    lib.orc_fit_geometry.restype = None
+    lib.orc_crop_ex.argtypes = [vp, i32, i32, i32, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]
+    lib.orc_crop_ex.restype = None
     lib.orc_assemble.argtypes = [vp, vp, i32, i32, vp, i32, i32, vp, vp, vp]
     lib.orc_assemble.restype = None
     _lib = lib
@@ -237,13 +241,29 @@ def crop_rect(det: np.ndarray, w: int, h: int) -> Tuple[int, int, int, int]:
     return tuple(int(v) for v in r)
 
 
+def fit_geometry(cw: int, ch: int, ow: int, oh: int) -> Tuple[int, int, int, int]:
+    """(nw, nh, pad_left, pad_top) of a cw x ch rectangle fitted into an ow x oh slot."""
+    g = np.zeros(4, dtype=np.int32)
+    _load().orc_fit_geometry(cw, ch, ow, oh, _ptr(g))
+    return tuple(int(v) for v in g)
+
+
 def crop(img: np.ndarray, w: int, h: int, det: np.ndarray, ow: int, oh: int,
-         swap_rb: bool = True) -> np.ndarray:
-    """One detection -> uint16 [3, oh, ow] binary16 bit patterns."""
+         swap_rb: bool = True, keep_aspect: bool = False, pad_value: int = 114,
+         mean: Optional[Sequence[float]] = None, std: Optional[Sequence[float]] = None) -> np.ndarray:
+    """One detection -> uint16 [3, oh, ow] binary16 bit patterns.  keep_aspect fits the rectangle
+    into the slot without distortion; mean / std (per output plane) turn normalisation on."""
     a = _frame2d(img)
     d = np.ascontiguousarray(np.atleast_1d(det), dtype=DET_DTYPE)
     out = np.empty((3, oh, ow), dtype=np.uint16)
-    _load().orc_crop(_ptr(a), w, h, a.shape[1], _ptr(d), ow, oh, 1 if swap_rb else 0, _ptr(out))
+    norm = mean is not None or std is not None
+    if not keep_aspect and not norm:
+        _load().orc_crop(_ptr(a), w, h, a.shape[1], _ptr(d), ow, oh, 1 if swap_rb else 0, _ptr(out))
+        return out
+    m = np.asarray(mean if mean is not None else (0.0, 0.0, 0.0), dtype=np.float32)
+    sd = np.asarray(std if std is not None else (1.0, 1.0, 1.0), dtype=np.float32)
+    _load().orc_crop_ex(_ptr(a), w, h, a.shape[1], _ptr(d), ow, oh, 1 if swap_rb else 0,
+                        1 if keep_aspect else 0, pad_value, 1 if norm else 0, _ptr(m), _ptr(sd), _ptr(out))
     return out
 
 
@@ -283,7 +303,7 @@ def run_stage(frames: Sequence[np.ndarray], sizes: Sequence[Tuple[int, int]], he
               swap_rb: bool = True, class_masks: Optional[Sequence[Sequence[int]]] = None,
               do_letterbox: bool = True, do_crops: bool = True, max_crops: Optional[int] = None,
               threads: int = 1, agnostic: bool = False, layout: str = "rows",
-              multi_label: bool = False) -> StageResult:
+              multi_label: bool = False, crop_options: Optional[Sequence[Optional[dict]]] = None) -> StageResult:
     """Whole stage over one batch, frame by frame (optionally a thread per frame; the C
     routines release the GIL).  max_crops bounds the crops rendered per branch."""
     n = len(frames)
@@ -323,10 +343,12 @@ def run_stage(frames: Sequence[np.ndarray], sizes: Sequence[Tuple[int, int]], he
             m = len(items) if max_crops is None else min(len(items), max_crops)
             crops = np.empty((m, 3, oh, ow), dtype=np.uint16)
 
-            def per_item(k: int, _crops=crops, _items=items, _ow=ow, _oh=oh) -> None:
+            opt = dict((crop_options[b] if crop_options is not None else None) or {})
+
+            def per_item(k: int, _crops=crops, _items=items, _ow=ow, _oh=oh, _opt=opt) -> None:
                 f, j = _items[k]
                 w, h = sizes[f]
-                _crops[k] = crop(frames[f], w, h, dets[f, j], _ow, _oh, swap_rb)
+                _crops[k] = crop(frames[f], w, h, dets[f, j], _ow, _oh, swap_rb, pad_value=pad_value, **_opt)
 
             pmap(per_item, m)
         res.offsets.append(offsets)

@@ -21,6 +21,8 @@
 // downstream slot.  Measured: large passes matter more than occupancy (2 x 32 KB buffers at
 // 3 CTAs/SM beat 2 x 24 KB at 4, 3 x 22 KB at 3 and 4 x 12 KB at 4).
 #include "octo_common.cuh"
+#include <cstring>
+
 #include "octo_kernels.h"
 
 namespace octo {
@@ -53,14 +55,19 @@ struct __align__(16) CropPass {
 // QUEUE = false: items come from the stage's current batch through the assembler above.
 // QUEUE = true: items are self-contained records popped from a device queue (qrec[0, *qpacked));
 // the assembler is skipped and nothing but the crops is written.
-template <int CAP, bool QUEUE>
+//
+// GENERAL = true adds the branch options: aspect-preserving fit (per item: fitted size nw x nh and
+// offsets inside the slot, canvas columns marked by zero weights in the tap table, canvas rows by a
+// negative row step) and per-plane normalisation (one fused multiply-add per value).  The plain
+// form carries none of that code.
+template <int CAP, bool QUEUE, bool GENERAL>
 __global__ void __launch_bounds__(kCropKernelThreads, kCropCtasPerSm)
 crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int first_item, int max_items,
             const int* __restrict__ bcount, const int* __restrict__ bidx, const octo_det_t* __restrict__ dets,
             int* __restrict__ offsets, int* __restrict__ n_items, octo_item_t* __restrict__ items,
             __half* __restrict__ out, int ow, int oh, int swap_rb, StageCounters* __restrict__ ctr,
             const QRecord* __restrict__ qrec, const int* __restrict__ qpacked, unsigned int* __restrict__ qstatus,
-            int* __restrict__ sched) {
+            int* __restrict__ sched, const CropOpts opts) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t full[kCropStages], empty[kCropStages];
     __shared__ CropPass s_pass[kCropStages];
@@ -139,6 +146,10 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         int w_c0 = 0, w_ncols = 0, w_r0 = 0, w_nr = 0;
         int w_seg_lo = 0, w_seg = 0, w_stride = 16, w_pass_rows = 1;
         bool w_valid = false, w_new = false;
+        // size and offset of the resized rectangle inside the slot: the whole slot unless the
+        // branch keeps the aspect ratio
+        int w_nw = ow, w_nh = oh, w_pl = 0, w_pt = 0;
+        float w_inv_dx = inv_dx, w_inv_dy = inv_dy, w_inv_all = inv_all;
 
         // geometry of the column tile starting at w_c0
         auto set_tile = [&]() {
@@ -148,8 +159,11 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             int lo = full_lo, hi = full_hi;
             if (w_tile_cols != ow) {
                 int xa, xb, rem;
-                src_coord(w_c0, w_cw, ow, inv_dx, xa, rem);
-                src_coord(w_c0 + w_ncols - 1, w_cw, ow, inv_dx, xb, rem);
+                // canvas columns count as the nearest image column
+                const int ia = min(max(w_c0 - w_pl, 0), w_nw - 1);
+                const int ib = min(max(w_c0 + w_ncols - 1 - w_pl, 0), w_nw - 1);
+                src_coord(ia, w_cw, w_nw, w_inv_dx, xa, rem);
+                src_coord(ib, w_cw, w_nw, w_inv_dx, xb, rem);
                 lo = (3 * (w_rx0 + xa)) & ~15;
                 hi = min((3 * (w_rx0 + xb) + 6 + 15) & ~15, full_hi);
             }
@@ -204,9 +218,25 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 w_data = fd.data; w_pitch = fd.pitch;
             }
             w_rx0 = rx0; w_ry0 = ry0; w_cw = rx1 - rx0; w_ch = ry1 - ry0;
+            if (GENERAL && opts.keep_aspect) {
+                // the side with the larger ratio fills the slot, the other is the exact quotient
+                // rounded half-up (at least 1); centred, odd remainder right / bottom
+                if ((long long)ow * w_ch <= (long long)oh * w_cw) {
+                    w_nw = ow;
+                    w_nh = max(1, (int)((2ll * w_ch * ow + w_cw) / (2ll * w_cw)));
+                } else {
+                    w_nh = oh;
+                    w_nw = max(1, (int)((2ll * w_cw * oh + w_ch) / (2ll * w_ch)));
+                }
+                w_pl = (ow - w_nw) >> 1;
+                w_pt = (oh - w_nh) >> 1;
+                w_inv_dx = 1.0f / (float)(2 * w_nw);
+                w_inv_dy = 1.0f / (float)(2 * w_nh);
+                w_inv_all = 1.0f / (255.0f * (float)(2 * w_nw) * (float)(2 * w_nh));
+            }
             const int full_seg = ((3 * rx1 + 15) & ~15) - ((3 * rx0) & ~15);
             w_tile_cols =
-                (full_seg + 16 > kCropMaxStride) ? max(2, (int)((long long)kCropTilePx * ow / w_cw) & ~1) : ow;
+                (full_seg + 16 > kCropMaxStride) ? max(2, (int)((long long)kCropTilePx * w_nw / w_cw) & ~1) : ow;
             w_c0 = 0;
             set_tile();
             w_row_lo = w_band * band_rows;
@@ -243,7 +273,18 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 // tiles, so the table of the tile before those is free before this pass's wait.
                 tb = (tb + 1) % kCropTables;
                 XEntry* const xt = s_xtab0 + (size_t)tb * ow;
-                for (int dx = lane; dx < ow; dx += 32) xt[dx] = make_xentry(dx, w_cw, ow, inv_dx, 3 * w_rx0);
+                for (int dx = lane; dx < ow; dx += 32) {
+                    if (GENERAL) {
+                        // a canvas column keeps the (valid) offset of the nearest image column
+                        // and gets zero weights, which mark it for the consumers
+                        const int ix = dx - w_pl, ixc = min(max(ix, 0), w_nw - 1);
+                        XEntry e = make_xentry(ixc, w_cw, w_nw, w_inv_dx, 3 * w_rx0);
+                        if (ix != ixc) e.wts = 0u;
+                        xt[dx] = e;
+                    } else {
+                        xt[dx] = make_xentry(dx, w_cw, ow, inv_dx, 3 * w_rx0);
+                    }
+                }
             }
             CropPass p;
             p.valid = w_valid ? 1 : 0;
@@ -256,16 +297,20 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             RowInfo ri;
             ri.row0 = 0; ri.step = 0; ri.wx = 0.0f; ri.wy = 0.0f;
             const uint8_t* src = nullptr;
-            const bool has_row = w_valid && lane < w_nr;
+            const bool in_pass = w_valid && lane < w_nr;
+            const int iy = w_r0 + lane - w_pt;  // row inside the resized rectangle
+            const bool has_row = in_pass && (!GENERAL || (iy >= 0 && iy < w_nh));
             if (has_row) {
                 int y0;
-                src_coord(w_r0 + lane, w_ch, oh, inv_dy, y0, ry);
+                src_coord(iy, w_ch, w_nh, w_inv_dy, y0, ry);
                 bytes = (uint32_t)w_seg * (ry != 0 ? 2u : 1u);
                 ri.row0 = 2 * lane * w_stride - w_seg_lo;  // table offsets are relative to the frame row
                 ri.step = w_stride;
-                ri.wx = (float)(2 * oh - ry) * inv_all;
-                ri.wy = (float)ry * inv_all;
+                ri.wx = (float)(2 * w_nh - ry) * w_inv_all;
+                ri.wy = (float)ry * w_inv_all;
                 src = w_data + (size_t)(w_ry0 + y0) * (size_t)w_pitch + w_seg_lo;
+            } else if (GENERAL) {
+                ri.step = -1;  // canvas row: nothing is staged for it
             }
             const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
             // ---- ring slot b: wait until the consumers have finished the pass that used it ----
@@ -283,7 +328,7 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 if (lane == 0) mbar_arrive(&full[b]);  // the end-of-work record
                 break;
             }
-            if (has_row) s_row[b][lane] = ri;
+            if (in_pass) s_row[b][lane] = ri;
             fence_proxy_async();
             __syncwarp();  // table, pass record and row data are written before the barrier is armed
             if (lane == 0) mbar_expect_tx(&full[b], total);
@@ -331,12 +376,24 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 const float wx = __uint_as_float(rw.z), wy = __uint_as_float(rw.w);
                 const float nwx = -kF32IntValue * wx;
                 float a0, a1, a2, b0, b1, b2;
-                if (wy != 0.0f) {
-                    sample_px<true>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
-                    sample_px<true>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+                if (GENERAL && (int)rw.y < 0) {  // canvas row
+                    a0 = b0 = opts.fill[0]; a1 = b1 = opts.fill[1]; a2 = b2 = opts.fill[2];
                 } else {
-                    sample_px<false>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
-                    sample_px<false>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+                    if (wy != 0.0f) {
+                        sample_px<true>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
+                        sample_px<true>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+                    } else {
+                        sample_px<false>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
+                        sample_px<false>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+                    }
+                    if (GENERAL) {
+                        a0 = ee.y ? fmaf(a0, opts.sc[0], opts.of[0]) : opts.fill[0];
+                        a1 = ee.y ? fmaf(a1, opts.sc[1], opts.of[1]) : opts.fill[1];
+                        a2 = ee.y ? fmaf(a2, opts.sc[2], opts.of[2]) : opts.fill[2];
+                        b0 = ee.w ? fmaf(b0, opts.sc[0], opts.of[0]) : opts.fill[0];
+                        b1 = ee.w ? fmaf(b1, opts.sc[1], opts.of[1]) : opts.fill[1];
+                        b2 = ee.w ? fmaf(b2, opts.sc[2], opts.of[2]) : opts.fill[2];
+                    }
                 }
                 const uint32_t o = (uint32_t)(r * ow + 2 * pair);
                 *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(a0, b0);
@@ -373,23 +430,33 @@ static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
     int grid = (int)(work < cap ? work : cap);
     if (grid < 1) grid = 1;  // a zero-slot window still gets its offsets and totals
     const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)a.out_w;
-    crop_kernel<CAP, false><<<grid, kCropKernelThreads, smem, stream>>>(
-        tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
-        a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, a.swap_rb, a.d_ctr, nullptr,
-        nullptr, nullptr, a.d_ctr->sched);
+    if (a.general)
+        crop_kernel<CAP, false, true><<<grid, kCropKernelThreads, smem, stream>>>(
+            tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
+            a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, a.swap_rb, a.d_ctr, nullptr, nullptr,
+            nullptr, a.d_ctr->sched, a.opts);
+    else
+        crop_kernel<CAP, false, false><<<grid, kCropKernelThreads, smem, stream>>>(
+            tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
+            a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, a.swap_rb, a.d_ctr, nullptr, nullptr,
+            nullptr, a.d_ctr->sched, a.opts);
     return cudaGetLastError();
 }
 
 cudaError_t prepare_crop() {
     const int smem = kCropStages * kCropRowBudget + kCropTables * (int)sizeof(XEntry) * 2048;
     cudaError_t e;
-    e = cudaFuncSetAttribute(crop_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(crop_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(crop_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(crop_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    const void* kernels[] = {
+        (const void*)crop_kernel<8, false, false>,   (const void*)crop_kernel<8, false, true>,
+        (const void*)crop_kernel<64, false, false>,  (const void*)crop_kernel<64, false, true>,
+        (const void*)crop_kernel<512, false, false>, (const void*)crop_kernel<512, false, true>,
+        (const void*)crop_kernel<8, true, false>,
+    };
+    for (const void* k : kernels) {
+        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 // Assembler + crop-resize of one branch window (a.max_items may be 0).
@@ -407,9 +474,11 @@ cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int
     const long long work = (long long)bz * ((out_h + 7) / 8);
     const int grid = (int)(work < cap ? work : cap);
     const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)out_w;
-    crop_kernel<8, true><<<grid, kCropKernelThreads, smem, stream>>>(
+    CropOpts opts;
+    memset(&opts, 0, sizeof(opts));
+    crop_kernel<8, true, false><<<grid, kCropKernelThreads, smem, stream>>>(
         tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
-        out_w, out_h, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched);
+        out_w, out_h, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched, opts);
     return cudaGetLastError();
 }
 

@@ -49,6 +49,13 @@ struct NmsArgs {
     StageCounters* d_ctr;
 };
 
+// Branch options of the crop kernel, per INPUT channel c (output plane swap_rb ? 2 - c : c):
+// value' = value * sc[c] + of[c]; fill[c] is the canvas value after the same mapping.
+struct CropOpts {
+    int keep_aspect;
+    float sc[3], of[3], fill[3];
+};
+
 struct CropArgs {
     const FrameDesc* frames;  // host
     int n;
@@ -62,6 +69,8 @@ struct CropArgs {
     void* d_out;
     int out_w, out_h, swap_rb, sm_count;
     StageCounters* d_ctr;
+    bool general;   // keep_aspect or normalize set for the branch
+    CropOpts opts;
 };
 
 // Opt the kernels of every table capacity into the shared memory they need (current device).

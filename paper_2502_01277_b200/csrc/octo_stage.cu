@@ -346,6 +346,19 @@ extern "C" int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_i
     a.swap_rb = c.swap_rb;
     a.sm_count = st->sm_count;
     a.d_ctr = st->d_ctr;
+    {
+        // branch options, expressed per input channel c (it lands in output plane swap ? 2 - c : c)
+        const octo_branch_cfg_t& br = c.branch[branch];
+        a.general = br.keep_aspect != 0 || br.normalize != 0;
+        a.opts.keep_aspect = br.keep_aspect;
+        for (int ch = 0; ch < 3; ++ch) {
+            const int p = c.swap_rb ? 2 - ch : ch;
+            const double m = br.normalize ? (double)br.mean[p] : 0.0, sd = br.normalize ? (double)br.std[p] : 1.0;
+            a.opts.sc[ch] = (float)(1.0 / sd);
+            a.opts.of[ch] = (float)(-m / sd);
+            a.opts.fill[ch] = (float)(((double)c.pad_value / 255.0 - m) / sd);
+        }
+    }
     OCTO_CUDA(cudaSetDevice(c.device));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     {
