@@ -40,13 +40,16 @@ UNIT = "frames/s"
 # reported as null.
 NCU_TRAFFIC = {
     # kernel: (source files, sha256[:16] of their concatenation at capture time, bytes per unit, unit)
-    # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md)
+    # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md); decode_planes on the
+    # anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "871dcab23b897b84", 493693.0, "crop"),
+             "30c103e879ad76e5", 487372.0, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                  "bc1f87af93a7ce97", 3705012.0, "frame"),
+                  "e8dcf55213e0dc25", 3701808.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "933edd2128942e38", 1696520.0, "frame"),
+               "75e75da9f5c5fef2", 1701316.0, "frame"),
+    "decode_planes": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
+                      "75e75da9f5c5fef2", 2812624.0, "frame"),
 }
 
 
@@ -61,6 +64,8 @@ def parse_args():
     p.add_argument("--e2e-steps", type=int, default=None)
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
+    p.add_argument("--graph", action="store_true",
+                   help="replay each step from a captured CUDA graph (small batches are launch-bound)")
     return p.parse_args()
 
 
@@ -335,8 +340,31 @@ def run_octo(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    ms_total = timed(args.steps, lambda i: step(sets[i % n_sets]))
-    gpu_launches = stage.launch_count - launches0
+    launches_per_step = (stage.launch_count - launches0) // max(warm, 1) if warm else 0
+    launches0 = stage.launch_count
+    if args.graph:
+        # one graph per input/output set: the stage calls only enqueue kernels, so a step can be
+        # captured once and replayed; the frame table travels in the kernel parameters
+        graphs = []
+        for z in sets:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                step(z)
+            graphs.append(g)
+        torch.cuda.synchronize(dev)
+
+        def replay(i):
+            with torch.cuda.stream(stream):
+                graphs[i % n_sets].replay()
+
+        for i in range(3):
+            replay(i)
+        launches0 = stage.launch_count
+        ms_total = timed(args.steps, replay)
+        gpu_launches = launches_per_step * args.steps  # kernels run from the graph, not counted by the stage
+    else:
+        ms_total = timed(args.steps, lambda i: step(sets[i % n_sets]))
+        gpu_launches = stage.launch_count - launches0
     ms_per_step = ms_total / args.steps
     value = world * n / (ms_per_step * 1e-3)
 
@@ -388,7 +416,8 @@ def run_octo(args):
         "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})", "unit": "GB/s",
         "frac": kern[dominant]["gbs"] / hbm_peak, "frac_of_nominal_8TBs": kern[dominant]["gbs"] / 8000.0,
         "alg_bytes_per_launch": alg[dominant], "ms_per_launch": kern[dominant]["ms_per_launch"],
-        "traffic": traffic_for(dominant, units),
+        "traffic": traffic_for("decode_planes" if dominant == "decode" and wl.head_layout == "planes" else dominant,
+                               units),
     }
 
     # ---- end to end from pinned host buffers ----
@@ -510,6 +539,7 @@ def run_octo(args):
                 "net_size": s, "head": list(batch.head.shape),
                 "crops": [list(b) for b in wl.branches], "items_per_step": [t[1] for t in totals],
                 "candidates_per_step": cand_per_step, "parallelism": f"replicas x{world}",
+                "launch": "CUDA graph replay" if args.graph else "stream launches",
                 "l2": (f"{n_sets} rotating input/output sets, {n_sets * (in_bytes + out_bytes) / 2**20:.0f} MiB working set"
                        if n_sets > 1 else f"one set of {(in_bytes + out_bytes) / 2**20:.0f} MiB per step, larger than L2"),
             },
