@@ -292,6 +292,15 @@ OCTO_API int octo_queue_push(octo_queue_t* q, octo_stage_t* st, int32_t branch, 
 OCTO_API int octo_queue_pop(octo_queue_t* q, int32_t bz, void* d_out_f16, octo_qitem_t* d_items_out,
                             int32_t* d_info, void* cuda_stream);
 
+/* octo_queue_pop with the release rule decided on the device, so that a serving loop can call it
+ * after every detector batch without reading the queue state back: the oldest min(bz, pending)
+ * items are released if a full batch is pending, or if the first pending item has waited for at
+ * least max_wait pushes (a batch fills at the arrival rate and its first request waits longest,
+ * Section II, discussion of Eq. 1); otherwise nothing is popped and d_info[0] = 0.  max_wait < 0
+ * releases unconditionally (octo_queue_pop).  Same arguments and errors as octo_queue_pop. */
+OCTO_API int octo_queue_pop_due(octo_queue_t* q, int32_t bz, int32_t max_wait, void* d_out_f16,
+                                octo_qitem_t* d_items_out, int32_t* d_info, void* cuda_stream);
+
 /* Synchronise `cuda_stream`, then read (and keep) the device status word. */
 OCTO_API int octo_stage_status(octo_stage_t* st, uint32_t* status_word, void* cuda_stream);
 
@@ -371,6 +380,44 @@ OCTO_API int octo_postprocess_frame_static(int32_t device, const float* d_head, 
                                            float iou_thresh, int32_t max_det, int32_t net_size,
                                            int32_t frame_w, int32_t frame_h, octo_det_t* d_dets,
                                            int32_t* d_count, void* cuda_stream);
+
+/* ---- placement of model instances on GPU inference streams (host only) ---------------------
+ * The paper's co-location scheduler (Section III-C "Inference Stream", Algorithm 2): a GPU runs
+ * several streams side by side; an execution occupies a portion of one stream, as long as its
+ * run time and as wide as the share of the GPU's compute it needs; a stream repeats with a duty
+ * cycle (half the pipeline's SLO).  Instances are placed one replica number at a time over all
+ * pipelines and their models in order.  Each goes to the free portion with the least spare room
+ * that (1) covers the window [start_us, end_us) it needs inside the cycle, (2) keeps the GPU
+ * within memory (sum of weights + per-stream largest intermediate memory <= mem_bytes) and
+ * utilisation (sum over streams of the widest resident <= util_max_permille) and (3) lies on a
+ * stream whose duty cycle is not longer than the instance's.  The first instance on a stream
+ * fixes the stream's duty cycle; the unused parts of the portion return to the free list.
+ * Free portions are ordered by length, then GPU, stream and start; an empty stream offers one
+ * unbounded portion.  All arrays are host memory; no CUDA call is made. */
+typedef struct {
+    int32_t pipeline, model, instance; /* pipeline index, position in its execution order, replica number */
+    int32_t util_permille;             /* width: share of the GPU's compute, 0..1000            */
+    int64_t start_us, end_us;          /* window inside the duty cycle, start < end <= duty cycle */
+    int64_t duty_cycle_us;             /* duty cycle of the instance's pipeline                  */
+    int64_t weight_bytes, inter_bytes; /* weight memory, intermediate (activation) memory        */
+} octo_coral_instance_t;
+
+typedef struct {
+    int64_t mem_bytes;          /* memory available to models                         */
+    int32_t util_max_permille;  /* utilisation limit                                  */
+    int32_t num_streams;        /* streams the GPU is divided into, 1..1024           */
+} octo_coral_gpu_t;
+
+typedef struct {
+    int32_t gpu, stream;        /* -1, -1: no portion found                            */
+    int64_t start_us, end_us;   /* the portion given to the instance                   */
+    int64_t duty_cycle_us;      /* duty cycle of the stream (<= the instance's own)    */
+} octo_coral_placement_t;
+
+/* out[i] receives the placement of inst[i].  Errors: OCTO_E_INVALID_ARG (null pointers, negative
+ * sizes, a window outside its duty cycle, n_gpus < 1, num_streams out of range). */
+OCTO_API int octo_coral_schedule(const octo_coral_instance_t* inst, int32_t n_inst, const octo_coral_gpu_t* gpus,
+                                 int32_t n_gpus, octo_coral_placement_t* out);
 
 /* Text of a status code; never NULL. */
 OCTO_API const char* octo_strerror(int code);

@@ -11,3 +11,4 @@ from .oracle import (  # noqa: F401
     assemble, StageResult, run_stage, margin_report,
 )
 from .queue import OracleQueue  # noqa: F401,E402
+from . import coral  # noqa: F401,E402

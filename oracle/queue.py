@@ -5,7 +5,9 @@ The paper's batches fill from bursty arrivals and the first request of a batch w
 Reading used here: a bounded first-in-first-out list of items per downstream branch.  A push
 appends the branch's items of one detector batch in item order (frame by frame, NMS order
 inside a frame) and stamps them with the push number; items that do not fit are dropped,
-newest first; a pop removes the oldest min(bz, pending) items.
+newest first; a pop removes the oldest min(bz, pending) items.  A pop with a waiting limit
+releases only a full batch, or a partial one whose first item has waited for at least max_wait
+pushes (an item queued by push number s has waited seq - 1 - s pushes after `seq` pushes).
 """
 from __future__ import annotations
 
@@ -29,9 +31,13 @@ class OracleQueue:
                 self.dropped += 1
         self.seq += 1
 
-    def pop(self, bz: int):
+    def pop(self, bz: int, max_wait: int = -1):
         """Returns (popped records, info) with info = (popped, pending after, dropped so far,
         seq of the oldest item still pending or -1)."""
+        if max_wait >= 0 and len(self.pending) < bz:
+            if not self.pending or self.seq - 1 - self.pending[0][0] < max_wait:
+                oldest = self.pending[0][0] if self.pending else -1
+                return [], (0, len(self.pending), self.dropped, oldest)
         out = self.pending[:bz]
         self.pending = self.pending[bz:]
         oldest = self.pending[0][0] if self.pending else -1

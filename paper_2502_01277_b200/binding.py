@@ -47,6 +47,7 @@ EXPORTS = (
     "octo_stage_workspace_bytes", "octo_stage_launch_count",
     "octo_strerror", "octo_last_cuda_error", "octo_version", "octo_postprocess_frame_static",
     "octo_adopt_regions", "octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop",
+    "octo_queue_pop_due", "octo_coral_schedule",
 )
 
 
@@ -83,6 +84,21 @@ class StageStats(ctypes.Structure):
     _fields_ = [("candidates", ctypes.c_int64), ("kept", ctypes.c_int64), ("packed", ctypes.c_int64),
                 ("total_items", ctypes.c_int64), ("status_word", ctypes.c_uint32),
                 ("max_candidates_per_image", ctypes.c_int32)]
+
+
+class CoralInstance(ctypes.Structure):
+    _fields_ = [("pipeline", ctypes.c_int32), ("model", ctypes.c_int32), ("instance", ctypes.c_int32),
+                ("util_permille", ctypes.c_int32), ("start_us", ctypes.c_int64), ("end_us", ctypes.c_int64),
+                ("duty_cycle_us", ctypes.c_int64), ("weight_bytes", ctypes.c_int64), ("inter_bytes", ctypes.c_int64)]
+
+
+class CoralGpu(ctypes.Structure):
+    _fields_ = [("mem_bytes", ctypes.c_int64), ("util_max_permille", ctypes.c_int32), ("num_streams", ctypes.c_int32)]
+
+
+class CoralPlacement(ctypes.Structure):
+    _fields_ = [("gpu", ctypes.c_int32), ("stream", ctypes.c_int32), ("start_us", ctypes.c_int64),
+                ("end_us", ctypes.c_int64), ("duty_cycle_us", ctypes.c_int64)]
 
 
 REGION_DTYPE = np.dtype([("d_data", "<u8"), ("width", "<i4"), ("height", "<i4"), ("pitch_bytes", "<i4"),
@@ -154,8 +170,13 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_queue_destroy.argtypes = [vp]
     lib.octo_queue_push.argtypes = [vp, vp, i32, vp]
     lib.octo_queue_pop.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.octo_queue_pop_due.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+    lib.octo_queue_pop_due.restype = ctypes.c_int
     for name in ("octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop"):
         getattr(lib, name).restype = ctypes.c_int
+    lib.octo_coral_schedule.argtypes = [ctypes.POINTER(CoralInstance), i32, ctypes.POINTER(CoralGpu), i32,
+                                        ctypes.POINTER(CoralPlacement)]
+    lib.octo_coral_schedule.restype = ctypes.c_int
     lib.octo_stage_workspace_bytes.argtypes = [vp]
     lib.octo_stage_workspace_bytes.restype = ctypes.c_int64
     lib.octo_stage_launch_count.argtypes = [vp]
@@ -422,6 +443,10 @@ class Stage:
     def workspace_bytes(self) -> int:
         return int(load_library().octo_stage_workspace_bytes(self.handle))
 
+    @property
+    def workspace_bytes(self) -> int:
+        return int(load_library().octo_stage_workspace_bytes(self.handle))
+
 
 class Queue:
     """Device-side dynamic-batch queue of one downstream branch (octo_queue_* in octo.h)."""
@@ -456,8 +481,10 @@ class Queue:
         self._keepalive.append(list(stage._frames_keepalive))  # frames stay alive while queued
         self._keepalive = self._keepalive[-64:]
 
-    def pop(self, bz: int, out=None, items=None, info=None, stream=None):
-        """Returns (crops fp16 [bz, 3, oh, ow], items uint8 [bz, 48], info int32 [4])."""
+    def pop(self, bz: int, out=None, items=None, info=None, stream=None, max_wait: int = -1):
+        """Returns (crops fp16 [bz, 3, oh, ow], items uint8 [bz, 48], info int32 [4]).  With
+        max_wait >= 0 the batch is only released when it is full or its first item has waited
+        that many pushes (octo_queue_pop_due)."""
         t = self._torch
         if out is None:
             out = t.empty((bz, 3, self.out_h, self.out_w), dtype=t.float16, device=self.device)
@@ -465,11 +492,30 @@ class Queue:
             items = t.zeros((bz, QITEM_DTYPE.itemsize), dtype=t.uint8, device=self.device)
         if info is None:
             info = t.zeros((4,), dtype=t.int32, device=self.device)
-        rc = load_library().octo_queue_pop(self.handle, bz, out.data_ptr(), items.data_ptr(), info.data_ptr(),
-                                           self._stream(stream))
+        rc = load_library().octo_queue_pop_due(self.handle, bz, max_wait, out.data_ptr(), items.data_ptr(),
+                                               info.data_ptr(), self._stream(stream))
         if rc != OCTO_OK:
-            raise OctoError(rc, "octo_queue_pop")
+            raise OctoError(rc, "octo_queue_pop_due")
         return out, items, info
+
+
+def octo_coral_schedule(instances: Sequence[dict], gpus: Sequence[dict]) -> List[Optional[Tuple[int, int, int, int, int]]]:
+    """instances: dicts with the fields of octo_coral_instance_t; gpus: dicts with the fields of
+    octo_coral_gpu_t.  Returns per instance (gpu, stream, start_us, end_us, duty_cycle_us) or None."""
+    ia = (CoralInstance * max(len(instances), 1))()
+    for k, d in enumerate(instances):
+        for name, _ in CoralInstance._fields_:
+            setattr(ia[k], name, int(d[name]))
+    ga = (CoralGpu * max(len(gpus), 1))()
+    for k, d in enumerate(gpus):
+        for name, _ in CoralGpu._fields_:
+            setattr(ga[k], name, int(d[name]))
+    out = (CoralPlacement * max(len(instances), 1))()
+    rc = load_library().octo_coral_schedule(ia, len(instances), ga, len(gpus), out)
+    if rc != OCTO_OK:
+        raise OctoError(rc, "octo_coral_schedule")
+    return [None if out[k].gpu < 0 else (out[k].gpu, out[k].stream, out[k].start_us, out[k].end_us, out[k].duty_cycle_us)
+            for k in range(len(instances))]
 
 
 def dets_to_numpy(dets, counts) -> Tuple[np.ndarray, np.ndarray]:

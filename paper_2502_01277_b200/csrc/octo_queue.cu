@@ -87,12 +87,18 @@ queue_push_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_de
 }
 
 __global__ void __launch_bounds__(256)
-queue_pop_kernel(const QRecord* __restrict__ ring, int cap, QueueState* __restrict__ state, int bz,
+queue_pop_kernel(const QRecord* __restrict__ ring, int cap, QueueState* __restrict__ state, int bz, int max_wait,
                  QRecord* __restrict__ staged, QRecord* __restrict__ items_out, int* __restrict__ info,
                  int* __restrict__ qpacked) {
     const long long head = state->head, tail = state->tail;
     const long long pending = tail - head;
-    const int popped = (int)(pending < bz ? pending : bz);
+    // max_wait < 0: release whatever is pending.  Otherwise a batch is released when it is full, or
+    // when its first item has waited for max_wait pushes (the item queued by push s has waited
+    // seq - 1 - s pushes once `seq` pushes have been made).
+    bool due = true;
+    if (max_wait >= 0 && pending < bz)
+        due = pending > 0 && (state->seq - 1 - ring[head % cap].seq) >= max_wait;
+    const int popped = due ? (int)(pending < bz ? pending : bz) : 0;
     for (int i = threadIdx.x; i < popped; i += blockDim.x) {
         const QRecord rec = ring[(head + i) % cap];
         staged[i] = rec;
@@ -196,6 +202,11 @@ extern "C" int octo_queue_push(octo_queue_t* q, octo_stage_t* st, int32_t branch
 
 extern "C" int octo_queue_pop(octo_queue_t* q, int32_t bz, void* d_out_f16, octo_qitem_t* d_items_out,
                               int32_t* d_info, void* cuda_stream) {
+    return octo_queue_pop_due(q, bz, -1, d_out_f16, d_items_out, d_info, cuda_stream);
+}
+
+extern "C" int octo_queue_pop_due(octo_queue_t* q, int32_t bz, int32_t max_wait, void* d_out_f16,
+                                  octo_qitem_t* d_items_out, int32_t* d_info, void* cuda_stream) {
     if (!q || !d_out_f16 || !d_info || bz < 1 || bz > q->max_bz) return OCTO_E_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(d_out_f16) & 15) || (reinterpret_cast<uintptr_t>(d_info) & 3) ||
         (reinterpret_cast<uintptr_t>(d_items_out) & 7))
@@ -203,7 +214,7 @@ extern "C" int octo_queue_pop(octo_queue_t* q, int32_t bz, void* d_out_f16, octo
     if (cudaSetDevice(q->device) != cudaSuccess) return OCTO_E_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     static_assert(sizeof(octo_qitem_t) == sizeof(QRecord), "public and internal queue records match");
-    queue_pop_kernel<<<1, 256, 0, stream>>>(q->d_ring, q->capacity, q->d_state, bz, q->d_staged,
+    queue_pop_kernel<<<1, 256, 0, stream>>>(q->d_ring, q->capacity, q->d_state, bz, max_wait, q->d_staged,
                                            reinterpret_cast<QRecord*>(d_items_out), d_info, q->d_qpacked);
     if (cudaGetLastError() != cudaSuccess) return OCTO_E_CUDA;
     cudaError_t e = launch_crop_queue(q->d_staged, q->d_qpacked, bz, d_out_f16, q->out_w, q->out_h, q->swap_rb,

@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 OW, OH = 64, 48
 
 
-def _run(capacity, bz, pops_between, final_pops):
+def _run(capacity, bz, pops_between, final_pops, max_wait=-1):
     wl = workloads.WORKLOADS["traffic_1080p"]
     batches = [workloads.make_batch("traffic_1080p", batch=nb, first_frame=ff) for nb, ff in ((2, 0), (3, 10), (1, 20))]
     st = make_stage(wl, 4, branches=((OW, OH),))
@@ -28,11 +28,11 @@ def _run(capacity, bz, pops_between, final_pops):
 
         def pop():
             buf = torch.full((bz, 3, OH, OW), 0x7BFF, dtype=torch.int16, device="cuda")
-            _, items, info = q.pop(bz, out=buf.view(torch.float16))
+            _, items, info = q.pop(bz, out=buf.view(torch.float16), max_wait=max_wait)
             torch.cuda.synchronize()
             recs = items.cpu().numpy().view(octo.QITEM_DTYPE).reshape(-1)
             got.append((buf.cpu().numpy().view(np.uint16), recs, tuple(int(v) for v in info.cpu())))
-            want.append(oq.pop(bz))
+            want.append(oq.pop(bz, max_wait))
 
         for b, npop in zip(batches, pops_between):
             frames = [torch.from_numpy(f).cuda() for f in b.frames]
@@ -78,6 +78,16 @@ def test_queue_drops_newest_when_full():
     want = _run(capacity=40, bz=16, pops_between=(0, 0, 0), final_pops=4)
     infos = [w[1] for w in want]
     assert infos[0][2] > 0 and sum(i[0] for i in infos) == 40
+
+
+def test_queue_release_rule_decided_on_the_device():
+    """bz larger than one batch's items: pops right after a push release nothing until the head of
+    the queue has waited two pushes or a full batch is pending."""
+    want = _run(capacity=256, bz=64, pops_between=(1, 1, 1), final_pops=2, max_wait=2)
+    infos = [w[1] for w in want]
+    assert infos[0][0] == 0 and infos[0][1] > 0          # first batch alone: not full, not due
+    assert any(i[0] == 64 for i in infos) or infos[2][0] > 0
+    assert sum(i[0] for i in infos) > 0
 
 
 def test_queue_argument_errors():

@@ -188,3 +188,20 @@ def test_queue_hand_case():
     recs, info = q.pop(4)
     assert [(r[0], r[3]) for r in recs] == [(2, (1, 1, 3, 3))] and info == (1, 0, 1, -1)
     assert q.pop(2) == ([], (0, 0, 1, -1))
+
+
+def test_queue_release_rule_hand_case():
+    """A batch is released when full, or when its first item has waited max_wait pushes: by hand."""
+    q = oracle.OracleQueue(capacity=16)
+    q.push([(0, 0), (0, 1)], [(0, 0, 1, 1)] * 2, ["a"])            # push 0: 2 items, waited 0
+    assert q.pop(4, max_wait=2) == ([], (0, 2, 0, 0))               # not full, head waited 0 pushes
+    q.push([(0, 0)], [(0, 0, 1, 1)], ["b"])                        # push 1: 3 pending, head waited 1
+    assert q.pop(4, max_wait=2)[1] == (0, 3, 0, 0)
+    q.push([], [], [])                                             # push 2 (an empty batch): head waited 2
+    recs, info = q.pop(4, max_wait=2)
+    assert [(r[0], r[2]) for r in recs] == [(0, 0), (0, 1), (1, 0)] and info == (3, 0, 0, -1)
+    assert q.pop(4, max_wait=0) == ([], (0, 0, 0, -1))              # nothing pending: nothing due
+    q.push([(0, k) for k in range(5)], [(0, 0, 1, 1)] * 5, ["c"])  # push 3: a full batch is due at once
+    recs, info = q.pop(4, max_wait=9)
+    assert len(recs) == 4 and info == (4, 1, 0, 3)
+    assert q.pop(4, max_wait=0)[1] == (1, 0, 0, -1)                 # max_wait 0: any pending item is due
