@@ -29,6 +29,8 @@ constexpr int kNmsThreads = 1024;
 constexpr int kNmsSmemCap = 8192;   // candidates handled on chip: 8 B key + 16 B box each
 constexpr int kWarpSortMax = 2048;  // largest class segment a single warp sorts
 constexpr int kRankSortMax = 512;   // up to here the warp sorts by counting instead of a network
+constexpr int kSmallMax = 256;      // images with at most this many candidates take the short path
+constexpr int kSmallWords = kSmallMax / 32;
 
 __device__ __forceinline__ void cmp_swap(unsigned long long* __restrict__ k, int i, int j) {
     const unsigned long long a = k[i], b = k[j];
@@ -118,200 +120,324 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
         if (threadIdx.x == 0) atomicOr(&ctr->status, 0x8u);
     }
 
-    // ---- bucket the keys by class: histogram, scan, scatter ----
-    for (int i = threadIdx.x; i < cnt; i += kNmsThreads) atomicAdd(&seg_cnt[(int)(gk[i] >> 57)], 1);
-    __syncthreads();
-    if (warp == 0) {
-        int run = 0;
-#pragma unroll
-        for (int base = 0; base < 128; base += 32) {
-            const int v = seg_cnt[base + lane];
-            int inc = v;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, inc, off);
-                if (lane >= off) inc += t;
-            }
-            seg_start[base + lane] = run + inc - v;
-            cursor[base + lane] = run + inc - v;
-            run += __shfl_sync(0xffffffffu, inc, 31);
-            if (__any_sync(0xffffffffu, v > kWarpSortMax) && lane == 0) s_big = 1;
-        }
-    }
-    __syncthreads();
-    {
-        // off chip the scatter goes through the box workspace and back into the key array
-        unsigned long long* const dst = on_chip ? keys : reinterpret_cast<unsigned long long*>(boxes);
-        for (int i = threadIdx.x; i < cnt; i += kNmsThreads) {
-            const unsigned long long k = gk[i];
-            dst[atomicAdd(&cursor[(int)(k >> 57)], 1)] = k;
+    // boxes are dead once NMS is done: their memory holds the ordered survivors (and the ranks)
+    unsigned long long* const ordered = reinterpret_cast<unsigned long long*>(boxes);
+    int nout;
+    if (cnt <= kSmallMax) {
+        // ---- short path for images with few candidates (the common case in serving): one
+        // thread per candidate and short phases between barriers.  Candidates are bucketed by
+        // class, ordered inside their class by counting, tested against the earlier candidates of
+        // the class in parallel (one bit each, relative to the class's first position); one
+        // thread per class then walks the class in order with the survivor set in a register (a
+        // candidate survives iff none of its suppressors did), and the survivors find their place
+        // in the global order (score, anchor, class) by counting among themselves. ----
+        __shared__ int s_m;
+        unsigned long long* const ukey = keys;                   // bucketed by class, unordered inside
+        unsigned long long* const skey = keys + kSmallMax;       // ordered inside each class
+        unsigned long long* const surv = keys + 2 * kSmallMax;   // global-order keys of the survivors
+        float4* const ubox = reinterpret_cast<float4*>(keys + 3 * kSmallMax);
+        float4* const sbox = ubox + kSmallMax;
+        unsigned int* const sup = reinterpret_cast<unsigned int*>(sbox + kSmallMax);  // [kSmallMax][kSmallWords]
+        unsigned char* const alive = reinterpret_cast<unsigned char*>(sup + kSmallMax * kSmallWords);
+        const int t = threadIdx.x;
+        unsigned long long k = kKeySentinel;
+        float4 box = make_float4(0.f, 0.f, 0.f, 0.f);
+        int cls = 0;
+        if (t == 0) s_m = 0;
+        if (t < cnt) {
+            k = gk[t];
+            cls = (int)(k >> 57);
+            atomicAdd(&seg_cnt[cls], 1);
+            box = gather_box(hbase + (size_t)(k & ((1ull << kKeyAnchorBits) - 1)) * as, es);
         }
         __syncthreads();
-        if (!on_chip) {
-            for (int i = threadIdx.x; i < cnt; i += kNmsThreads) keys[i] = dst[i];
-            __syncthreads();
-        }
-    }
-
-    // ---- very large classes are sorted by the whole CTA ----
-    if (s_big) {
-        for (int cls = 0; cls < 128; ++cls) {
-            const int m = seg_cnt[cls];
-            if (m > kWarpSortMax) bitonic_range<true>(keys + seg_start[cls], m, threadIdx.x, kNmsThreads);
-        }
-    }
-
-    // ---- one warp per class: sort, gather boxes, greedy NMS ----
-    for (int cls = warp; cls < 128; cls += kNmsThreads / 32) {
-        const int m = seg_cnt[cls];
-        if (m == 0) continue;
-        const int s = seg_start[cls], e = s + m;
-        if (m > 1 && m <= kRankSortMax) {
-            // small class: every key counts the keys below it and moves to that position, staged
-            // in the (not yet used) box slots of the segment
-            unsigned long long* const tmp = reinterpret_cast<unsigned long long*>(boxes + s);
-            for (int i0 = lane; i0 < m; i0 += 128) {
-                // up to four keys per lane share one pass over the segment
-                const unsigned long long k0 = keys[s + i0];
-                const unsigned long long k1 = i0 + 32 < m ? keys[s + i0 + 32] : kKeySentinel;
-                const unsigned long long k2 = i0 + 64 < m ? keys[s + i0 + 64] : kKeySentinel;
-                const unsigned long long k3 = i0 + 96 < m ? keys[s + i0 + 96] : kKeySentinel;
-                int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
-                for (int j = 0; j < m; ++j) {
-                    const unsigned long long kj = keys[s + j];
-                    r0 += kj < k0; r1 += kj < k1; r2 += kj < k2; r3 += kj < k3;
-                }
-                tmp[r0] = k0;
-                if (i0 + 32 < m) tmp[r1] = k1;
-                if (i0 + 64 < m) tmp[r2] = k2;
-                if (i0 + 96 < m) tmp[r3] = k3;
-            }
-            __syncwarp();
-            for (int p = lane; p < m; p += 32) keys[s + p] = tmp[p];
-            __syncwarp();
-        } else if (m > 1 && m <= kWarpSortMax) {
-            bitonic_range<false>(keys + s, m, lane, 32);
-        }
-        for (int p = s + lane; p < e; p += 32) {
-            const int anchor = (int)(keys[p] & ((1ull << kKeyAnchorBits) - 1));
-            boxes[p] = gather_box(hbase + (size_t)anchor * as, es);
-        }
-        __syncwarp();
-        int nk = 0;  // survivors of this class, compacted at [s, s + nk)
-        for (int c0 = s; c0 < e && nk < max_det; c0 += 32) {
-            const int p = c0 + lane;
-            const bool valid = p < e;
-            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            unsigned long long k = kKeySentinel;
-            if (valid) { b = boxes[p]; k = keys[p]; }
-            bool alive = valid;
-            for (int t = 0; t < nk; ++t) {
-                if (!__any_sync(0xffffffffu, alive)) break;
-                const float4 kb = boxes[s + t];
-                if (alive && iou_above(kb, b, iou_test)) alive = false;
-            }
-            unsigned rem = __ballot_sync(0xffffffffu, alive);
-            unsigned keptmask = 0;
-            while (rem) {
-                const int l = __ffs(rem) - 1;
-                keptmask |= 1u << l;
-                float4 lb;
-                lb.x = __shfl_sync(0xffffffffu, b.x, l);
-                lb.y = __shfl_sync(0xffffffffu, b.y, l);
-                lb.z = __shfl_sync(0xffffffffu, b.z, l);
-                lb.w = __shfl_sync(0xffffffffu, b.w, l);
-                if (alive && lane > l && iou_above(lb, b, iou_test)) alive = false;
-                rem = __ballot_sync(0xffffffffu, alive) & ~((2u << l) - 1u);
-            }
-            __syncwarp();
-            const int allowed = min(__popc(keptmask), max_det - nk);
-            if ((keptmask >> lane) & 1u) {
-                const int r = __popc(keptmask & ((1u << lane) - 1u));
-                if (r < allowed) {
-                    boxes[s + nk + r] = b;
-                    // re-key for the global order: inverted score | anchor | class
-                    keys[s + nk + r] = ((k & ((1ull << 57) - 1)) << 7) | (k >> 57);
-                }
-            }
-            __syncwarp();
-            nk += allowed;
-        }
-        for (int p = s + nk + lane; p < e; p += 32) keys[p] = kKeySentinel;
-        if (lane == 0 && nk > 0) {
-            nkept[cls] = nk;
-            atomicAdd(&s_total, nk);
-            live[atomicAdd(&s_live, 1)] = cls;
-        }
-    }
-    __syncthreads();
-
-    // ---- global score order: merge of the per-class survivor lists by rank ----
-    const int nout = min(s_total, max_det);
-    const int nlive = s_live;
-    if (warp == 0) {
-        // exclusive scan of the survivor counts over the live classes -> cursor[q]
-        int run = 0;
-        for (int base = 0; base < nlive; base += 32) {
-            const int q = base + lane;
-            const int v = q < nlive ? nkept[live[q]] : 0;
-            int inc = v;
+        if (warp == 0) {
+            int run = 0;
 #pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, inc, off);
-                if (lane >= off) inc += t;
+            for (int base = 0; base < 128; base += 32) {
+                const int v = seg_cnt[base + lane];
+                int inc = v;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int u = __shfl_up_sync(0xffffffffu, inc, off);
+                    if (lane >= off) inc += u;
+                }
+                seg_start[base + lane] = run + inc - v;
+                cursor[base + lane] = run + inc - v;
+                run += __shfl_sync(0xffffffffu, inc, 31);
             }
-            if (q < nlive) cursor[q] = run + inc - v;
-            run += __shfl_sync(0xffffffffu, inc, 31);
         }
+        __syncthreads();
+        if (t < cnt) {
+            const int pos = atomicAdd(&cursor[cls], 1);
+            ukey[pos] = k;
+            ubox[pos] = box;
+        }
+        __syncthreads();
+        int start = 0;
+        if (t < cnt) {  // from here on thread t owns bucket position t
+            k = ukey[t];
+            box = ubox[t];
+            cls = (int)(k >> 57);
+            start = seg_start[cls];
+            const int m = seg_cnt[cls];
+            int r = 0;
+            for (int j = start; j < start + m; ++j) r += ukey[j] < k;
+            skey[start + r] = k;
+            sbox[start + r] = box;
+        }
+        __syncthreads();
+        if (t < cnt) {  // ... and ordered position t (same class, hence the same start)
+            const float4 bi = sbox[t];
+            const int words = (t - start + 31) >> 5;  // words that hold predecessors
+            for (int w = 0; w < words; ++w) {
+                unsigned bits = 0u;
+                const int j0 = start + (w << 5), j1 = min(j0 + 32, t);
+                for (int j = j0; j < j1; ++j)
+                    if (iou_above(sbox[j], bi, iou_test)) bits |= 1u << (j - j0);
+                sup[t * kSmallWords + w] = bits;
+            }
+        }
+        __syncthreads();
+        if (t < cnt && t == start) {  // first position of a class: walk the class in order
+            const int m = seg_cnt[cls];
+            if (m <= 32) {
+                unsigned kept = 0u;
+                alive[t] = 1;
+                kept = 1u;
+                for (int i = 1; i < m; ++i) {
+                    const bool ok = (sup[(t + i) * kSmallWords] & kept) == 0u;
+                    alive[t + i] = ok ? 1 : 0;
+                    if (ok) kept |= 1u << i;
+                }
+            } else {
+                unsigned kept[kSmallWords];
+#pragma unroll
+                for (int w = 0; w < kSmallWords; ++w) kept[w] = 0u;
+                for (int i = 0; i < m; ++i) {
+                    bool ok = true;
+#pragma unroll
+                    for (int w = 0; w < kSmallWords; ++w)
+                        if (w < ((i + 31) >> 5) && (sup[(t + i) * kSmallWords + w] & kept[w]) != 0u) ok = false;
+                    alive[t + i] = ok ? 1 : 0;
+#pragma unroll
+                    for (int w = 0; w < kSmallWords; ++w)
+                        if (ok && w == (i >> 5)) kept[w] |= 1u << (i & 31);
+                }
+            }
+        }
+        __syncthreads();
+        unsigned long long g = kKeySentinel;
+        const bool mine = t < cnt && alive[t] != 0;
+        if (mine) {
+            const unsigned long long ks = skey[t];
+            g = ((ks & ((1ull << 57) - 1)) << 7) | (ks >> 57);  // inverted score | anchor | class
+            surv[atomicAdd(&s_m, 1)] = g;
+        }
+        __syncthreads();
+        const int m_all = s_m;
+        if (mine) {
+            int r = 0;
+            for (int j = 0; j < m_all; ++j) r += surv[j] < g;
+            if (r < max_det) ordered[r] = g;
+        }
+        nout = min(m_all, max_det);
+        __syncthreads();
+    } else {
+        // ---- bucket the keys by class: histogram, scan, scatter ----
+        for (int i = threadIdx.x; i < cnt; i += kNmsThreads) atomicAdd(&seg_cnt[(int)(gk[i] >> 57)], 1);
+        __syncthreads();
+        if (warp == 0) {
+            int run = 0;
+    #pragma unroll
+            for (int base = 0; base < 128; base += 32) {
+                const int v = seg_cnt[base + lane];
+                int inc = v;
+    #pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, inc, off);
+                    if (lane >= off) inc += t;
+                }
+                seg_start[base + lane] = run + inc - v;
+                cursor[base + lane] = run + inc - v;
+                run += __shfl_sync(0xffffffffu, inc, 31);
+                if (__any_sync(0xffffffffu, v > kWarpSortMax) && lane == 0) s_big = 1;
+            }
+        }
+        __syncthreads();
+        {
+            // off chip the scatter goes through the box workspace and back into the key array
+            unsigned long long* const dst = on_chip ? keys : reinterpret_cast<unsigned long long*>(boxes);
+            for (int i = threadIdx.x; i < cnt; i += kNmsThreads) {
+                const unsigned long long k = gk[i];
+                dst[atomicAdd(&cursor[(int)(k >> 57)], 1)] = k;
+            }
+            __syncthreads();
+            if (!on_chip) {
+                for (int i = threadIdx.x; i < cnt; i += kNmsThreads) keys[i] = dst[i];
+                __syncthreads();
+            }
+        }
+
+        // ---- very large classes are sorted by the whole CTA ----
+        if (s_big) {
+            for (int cls = 0; cls < 128; ++cls) {
+                const int m = seg_cnt[cls];
+                if (m > kWarpSortMax) bitonic_range<true>(keys + seg_start[cls], m, threadIdx.x, kNmsThreads);
+            }
+        }
+
+        // ---- one warp per class: sort, gather boxes, greedy NMS ----
+        for (int cls = warp; cls < 128; cls += kNmsThreads / 32) {
+            const int m = seg_cnt[cls];
+            if (m == 0) continue;
+            const int s = seg_start[cls], e = s + m;
+            if (m > 1 && m <= kRankSortMax) {
+                // small class: every key counts the keys below it and moves to that position, staged
+                // in the (not yet used) box slots of the segment
+                unsigned long long* const tmp = reinterpret_cast<unsigned long long*>(boxes + s);
+                for (int i0 = lane; i0 < m; i0 += 128) {
+                    // up to four keys per lane share one pass over the segment
+                    const unsigned long long k0 = keys[s + i0];
+                    const unsigned long long k1 = i0 + 32 < m ? keys[s + i0 + 32] : kKeySentinel;
+                    const unsigned long long k2 = i0 + 64 < m ? keys[s + i0 + 64] : kKeySentinel;
+                    const unsigned long long k3 = i0 + 96 < m ? keys[s + i0 + 96] : kKeySentinel;
+                    int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+                    for (int j = 0; j < m; ++j) {
+                        const unsigned long long kj = keys[s + j];
+                        r0 += kj < k0; r1 += kj < k1; r2 += kj < k2; r3 += kj < k3;
+                    }
+                    tmp[r0] = k0;
+                    if (i0 + 32 < m) tmp[r1] = k1;
+                    if (i0 + 64 < m) tmp[r2] = k2;
+                    if (i0 + 96 < m) tmp[r3] = k3;
+                }
+                __syncwarp();
+                for (int p = lane; p < m; p += 32) keys[s + p] = tmp[p];
+                __syncwarp();
+            } else if (m > 1 && m <= kWarpSortMax) {
+                bitonic_range<false>(keys + s, m, lane, 32);
+            }
+            for (int p = s + lane; p < e; p += 32) {
+                const int anchor = (int)(keys[p] & ((1ull << kKeyAnchorBits) - 1));
+                boxes[p] = gather_box(hbase + (size_t)anchor * as, es);
+            }
+            __syncwarp();
+            int nk = 0;  // survivors of this class, compacted at [s, s + nk)
+            for (int c0 = s; c0 < e && nk < max_det; c0 += 32) {
+                const int p = c0 + lane;
+                const bool valid = p < e;
+                float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+                unsigned long long k = kKeySentinel;
+                if (valid) { b = boxes[p]; k = keys[p]; }
+                bool alive = valid;
+                for (int t = 0; t < nk; ++t) {
+                    if (!__any_sync(0xffffffffu, alive)) break;
+                    const float4 kb = boxes[s + t];
+                    if (alive && iou_above(kb, b, iou_test)) alive = false;
+                }
+                unsigned rem = __ballot_sync(0xffffffffu, alive);
+                unsigned keptmask = 0;
+                while (rem) {
+                    const int l = __ffs(rem) - 1;
+                    keptmask |= 1u << l;
+                    float4 lb;
+                    lb.x = __shfl_sync(0xffffffffu, b.x, l);
+                    lb.y = __shfl_sync(0xffffffffu, b.y, l);
+                    lb.z = __shfl_sync(0xffffffffu, b.z, l);
+                    lb.w = __shfl_sync(0xffffffffu, b.w, l);
+                    if (alive && lane > l && iou_above(lb, b, iou_test)) alive = false;
+                    rem = __ballot_sync(0xffffffffu, alive) & ~((2u << l) - 1u);
+                }
+                __syncwarp();
+                const int allowed = min(__popc(keptmask), max_det - nk);
+                if ((keptmask >> lane) & 1u) {
+                    const int r = __popc(keptmask & ((1u << lane) - 1u));
+                    if (r < allowed) {
+                        boxes[s + nk + r] = b;
+                        // re-key for the global order: inverted score | anchor | class
+                        keys[s + nk + r] = ((k & ((1ull << 57) - 1)) << 7) | (k >> 57);
+                    }
+                }
+                __syncwarp();
+                nk += allowed;
+            }
+            for (int p = s + nk + lane; p < e; p += 32) keys[p] = kKeySentinel;
+            if (lane == 0 && nk > 0) {
+                nkept[cls] = nk;
+                atomicAdd(&s_total, nk);
+                live[atomicAdd(&s_live, 1)] = cls;
+            }
+        }
+        __syncthreads();
+
+        // ---- global score order: merge of the per-class survivor lists by rank ----
+        const int nlive = s_live;
+        if (warp == 0) {
+            // exclusive scan of the survivor counts over the live classes -> cursor[q]
+            int run = 0;
+            for (int base = 0; base < nlive; base += 32) {
+                const int q = base + lane;
+                const int v = q < nlive ? nkept[live[q]] : 0;
+                int inc = v;
+    #pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, inc, off);
+                    if (lane >= off) inc += t;
+                }
+                if (q < nlive) cursor[q] = run + inc - v;
+                run += __shfl_sync(0xffffffffu, inc, 31);
+            }
+        }
+        __syncthreads();
+        // boxes are no longer needed: their memory holds the ordered survivors and the ranks
+        int* const rank = reinterpret_cast<int*>(ordered + min(max_det, cnt));
+        const int total = s_total;
+        // survivor e (dense numbering over the live classes): rank starts as the index in its own list
+        for (int e = threadIdx.x; e < total; e += kNmsThreads) {
+            int lo = 0, hi = nlive;  // live class q with cursor[q] <= e < cursor[q + 1]
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (cursor[mid] <= e) lo = mid; else hi = mid;
+            }
+            rank[e] = e - cursor[lo];
+        }
+        __syncthreads();
+        // every (survivor, other live class) pair adds the number of that class's survivors that
+        // precede the survivor; pairs are independent, so the searches run in parallel
+        // (neighbouring threads take neighbouring survivors against the same class, so the list reads
+        // broadcast and the rank updates hit different addresses)
+        for (int i = threadIdx.x; i < total * nlive; i += kNmsThreads) {
+            const int q = i / total, e = i - q * total;
+            int lo = 0, hi = nlive;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (cursor[mid] <= e) lo = mid; else hi = mid;
+            }
+            if (lo == q) continue;
+            const unsigned long long g = keys[seg_start[live[lo]] + (e - cursor[lo])];
+            const unsigned long long* const list = keys + seg_start[live[q]];
+            int l2 = 0, h2 = nkept[live[q]];
+            while (l2 < h2) {
+                const int mid = (l2 + h2) >> 1;
+                if (list[mid] < g) l2 = mid + 1; else h2 = mid;
+            }
+            if (l2) atomicAdd(&rank[e], l2);
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < total; e += kNmsThreads) {
+            const int r = rank[e];
+            if (r >= max_det) continue;
+            int lo = 0, hi = nlive;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (cursor[mid] <= e) lo = mid; else hi = mid;
+            }
+            ordered[r] = keys[seg_start[live[lo]] + (e - cursor[lo])];
+        }
+        __syncthreads();
+        nout = min(s_total, max_det);
     }
-    __syncthreads();
-    // boxes are no longer needed: their memory holds the ordered survivors and the ranks
-    unsigned long long* const ordered = reinterpret_cast<unsigned long long*>(boxes);
-    int* const rank = reinterpret_cast<int*>(ordered + min(max_det, cnt));
-    const int total = s_total;
-    // survivor e (dense numbering over the live classes): rank starts as the index in its own list
-    for (int e = threadIdx.x; e < total; e += kNmsThreads) {
-        int lo = 0, hi = nlive;  // live class q with cursor[q] <= e < cursor[q + 1]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (cursor[mid] <= e) lo = mid; else hi = mid;
-        }
-        rank[e] = e - cursor[lo];
-    }
-    __syncthreads();
-    // every (survivor, other live class) pair adds the number of that class's survivors that
-    // precede the survivor; pairs are independent, so the searches run in parallel
-    // (neighbouring threads take neighbouring survivors against the same class, so the list reads
-    // broadcast and the rank updates hit different addresses)
-    for (int i = threadIdx.x; i < total * nlive; i += kNmsThreads) {
-        const int q = i / total, e = i - q * total;
-        int lo = 0, hi = nlive;
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (cursor[mid] <= e) lo = mid; else hi = mid;
-        }
-        if (lo == q) continue;
-        const unsigned long long g = keys[seg_start[live[lo]] + (e - cursor[lo])];
-        const unsigned long long* const list = keys + seg_start[live[q]];
-        int l2 = 0, h2 = nkept[live[q]];
-        while (l2 < h2) {
-            const int mid = (l2 + h2) >> 1;
-            if (list[mid] < g) l2 = mid + 1; else h2 = mid;
-        }
-        if (l2) atomicAdd(&rank[e], l2);
-    }
-    __syncthreads();
-    for (int e = threadIdx.x; e < total; e += kNmsThreads) {
-        const int r = rank[e];
-        if (r >= max_det) continue;
-        int lo = 0, hi = nlive;
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (cursor[mid] <= e) lo = mid; else hi = mid;
-        }
-        ordered[r] = keys[seg_start[live[lo]] + (e - cursor[lo])];
-    }
-    __syncthreads();
 
     const FrameDesc& fd = tab.f[img];
     // region of the source frame shown by the detector input: x in [x_lo, x_hi], y likewise

@@ -233,6 +233,34 @@ def test_max_det_cap_is_hit():
     assert res.counts.tolist() == [37, 37]
 
 
+def test_max_det_cap_is_hit_with_few_candidates():
+    """The cap inside the short path (at most 256 candidates per image)."""
+    b = _small_case(200, 200, batch=3, max_det=11)
+    res, ref = _run_and_compare(b)
+    assert int(ref.n_cand.max()) <= 256 and res.counts.tolist() == [11, 11, 11]
+
+
+@pytest.mark.parametrize("n_raised", [255, 256, 257, 300])
+def test_candidate_counts_around_the_short_path_limit(n_raised):
+    b = _small_case(n_raised, 30, batch=2)
+    res, ref = _run_and_compare(b)
+    assert abs(int(ref.n_cand.max()) - n_raised) <= 3
+
+
+def test_class_agnostic_with_few_candidates():
+    """One class of up to 256 candidates in the short path (survivor set wider than one word)."""
+    b = _small_case(180, 25, batch=2)
+    wl = b.workload
+    st = make_stage(wl, b.n, class_agnostic=True)
+    try:
+        ref = _oracle(b, agnostic=True, do_letterbox=False, do_crops=False)
+        res = run_stage_gpu(st, b.frames, b.sizes, b.head, max_items=[8])
+        assert 100 < int(ref.n_cand.max()) <= 256
+        _check_dets(res, ref)
+    finally:
+        st.close()
+
+
 def test_score_ties_break_by_anchor():
     b = _small_case(40, 40, batch=1)
     h = b.head
