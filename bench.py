@@ -43,13 +43,13 @@ NCU_TRAFFIC = {
     # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md); decode_planes on the
     # anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "30c103e879ad76e5", 487372.0, "crop"),
+             "30c103e879ad76e5", 486995.0, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                  "e8dcf55213e0dc25", 3701808.0, "frame"),
+                  "e8dcf55213e0dc25", 3694980.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "75e75da9f5c5fef2", 1701316.0, "frame"),
+               "c2fb71b4332d2670", 1700720.0, "frame"),
     "decode_planes": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                      "75e75da9f5c5fef2", 2812624.0, "frame"),
+                      "c2fb71b4332d2670", 2813744.0, "frame"),
 }
 
 
