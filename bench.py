@@ -460,8 +460,11 @@ def run_octo(args):
         h_crops = [torch.empty((max(totals[b][1], 1) + len(chunks), 3, oh, ow), dtype=torch.float16).pin_memory()
                    for b, (ow, oh) in enumerate(wl.branches)]
         for ln in lanes:
-            ln.dev_frames = [torch.empty_like(h_frames[0], device=dev) for _ in range(c)]
+            ln.dev_block = torch.empty((c,) + tuple(h_frames[0].shape), dtype=torch.uint8, device=dev)
+            ln.dev_frames = [ln.dev_block[k] for k in range(c)]
         same_shape = all(f.shape == h_frames[0].shape for f in h_frames)
+        # frames of one shape travel as one pinned block per sub-batch (one copy instead of one per frame)
+        h_block = torch.stack(h_frames).pin_memory() if same_shape else None
         d2h = [0]
 
         def enqueue(ci):
@@ -473,8 +476,11 @@ def run_octo(args):
                     fr = ln.dev_frames[:m]
                 else:
                     fr = [torch.empty_like(h_frames[lo + k], device=dev) for k in range(m)]
-                for k in range(m):
-                    fr[k].copy_(h_frames[lo + k], non_blocking=True)
+                if same_shape:
+                    ln.dev_block[:m].copy_(h_block[lo:hi], non_blocking=True)
+                else:
+                    for k in range(m):
+                        fr[k].copy_(h_frames[lo + k], non_blocking=True)
                 ln.head[:m].copy_(h_head[lo:hi], non_blocking=True)
                 ln.stage.preprocess(fr, batch.sizes[lo:hi], out=ln.det_in[:m], stream=ln.stream)
                 ln.stage.postprocess(ln.head[:m], dets=ln.dets[:m], counts=ln.counts[:m], stream=ln.stream)
