@@ -39,6 +39,7 @@ constexpr int kCropTilePx = 5300;
 constexpr int kCropMaxPassRows = 32;
 constexpr int kCropCtasPerSm = 3;
 constexpr int kCropConsumerWarps = 8;
+constexpr int kCropTailBands = 4;     // finer tiles for the last crops of a launch
 constexpr int kCropTilesPerCta = 4;  // measured: 4 > 8 > 16 > 1 for small batches; a tile switch costs about 1 us
 constexpr unsigned kCropProducerSleepNs = 200;  // between the producer's polls of an "empty" barrier
 constexpr int kCropKernelThreads = 32 * (kCropConsumerWarps + 1);  // + one producer warp
@@ -126,6 +127,14 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
     const int bands_req = min(max(bands_want, 1), (oh + 7) >> 3);
     const int band_rows = min(((oh + bands_req - 1) / bands_req + 7) & ~7, oh);
     const int bands = (oh + band_rows - 1) / band_rows;
+    // With whole crops as tiles the grid would end up to one crop apart, so the last crops (one
+    // per CTA) are cut into up to kCropTailBands finer tiles that even the end out.
+    const int tail_req = min(kCropTailBands, (oh + 7) >> 3);
+    const int tail_rows = min(((oh + tail_req - 1) / tail_req + 7) & ~7, oh);
+    const int tail_bands = (oh + tail_rows - 1) / tail_rows;
+    const int tail_crops = (bands == 1 && tail_bands > 1) ? min(packed, (int)gridDim.x) : 0;
+    const long long coarse_tiles = (long long)(packed - tail_crops) * bands;
+    const long long all_tiles = coarse_tiles + (long long)tail_crops * tail_bands;
     const size_t plane = (size_t)ow * (size_t)oh;
 
     if (warp == kCropConsumerWarps) {
@@ -139,7 +148,7 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         // round trips of a tile's resolution (counter -> detection index -> detection) are hidden
         // behind the passes that are already staged in the ring.
         int w_tiles = 0;  // tiles opened so far
-        int w_slot = 0, w_band = 0;
+        int w_slot = 0, w_band = 0, w_band_rows = band_rows;
         int w_pitch = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
         const uint8_t* w_data = nullptr;
         int w_row_lo = 0, w_row_hi = 0, w_tile_cols = ow;
@@ -170,7 +179,7 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             w_seg_lo = lo;
             w_seg = hi - lo;
             w_stride = w_seg + 16;
-            w_pass_rows = max(1, min(min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows), band_rows));
+            w_pass_rows = max(1, min(min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows), w_band_rows));
         };
         // first pass of the next tile, if there is one; every lane resolves the same item
         auto open_tile = [&]() {
@@ -181,10 +190,18 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 tile = (long long)gridDim.x + (long long)__shfl_sync(0xffffffffu, t, 0);
             }
             w_tiles += 1;
-            w_valid = tile < (long long)packed * bands;
+            w_valid = tile < all_tiles;
             if (!w_valid) return;
-            w_slot = (int)(tile / bands);
-            w_band = (int)(tile - (long long)w_slot * bands);
+            if (tile < coarse_tiles) {
+                w_slot = (int)(tile / bands);
+                w_band = (int)(tile - (long long)w_slot * bands);
+                w_band_rows = band_rows;
+            } else {
+                const long long u = tile - coarse_tiles;
+                w_slot = (packed - tail_crops) + (int)(u / tail_bands);
+                w_band = (int)(u % tail_bands);
+                w_band_rows = tail_rows;
+            }
             int rx0, ry0, rx1, ry1;
             if (QUEUE) {
                 const QRecord rec = qrec[w_slot];
@@ -239,8 +256,8 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 (full_seg + 16 > kCropMaxStride) ? max(2, (int)((long long)kCropTilePx * w_nw / w_cw) & ~1) : ow;
             w_c0 = 0;
             set_tile();
-            w_row_lo = w_band * band_rows;
-            w_row_hi = min(w_row_lo + band_rows, oh);
+            w_row_lo = w_band * w_band_rows;
+            w_row_hi = min(w_row_lo + w_band_rows, oh);
             w_r0 = w_row_lo;
             w_nr = min(w_pass_rows, w_row_hi - w_r0);
             w_new = true;
