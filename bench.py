@@ -43,7 +43,7 @@ NCU_TRAFFIC = {
     # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md); decode_planes on the
     # anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "5c118b0e6c587331", 473898.6, "crop"),
+             "b45affcf6a21acdf", 473898.6, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
                   "e8dcf55213e0dc25", 3694980.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),

@@ -7,10 +7,12 @@
 // detection through the branch's index list, -> outward-rounded integer rectangle.  The item
 // table entry of a slot is written by the CTA that processes the slot's first row band.
 //
-// Crop-resize: bound by instruction issue, then HBM (the fp16 output is as large as the
-// source rectangles).  A persistent grid strides over (slot, row band) tiles, so no host
-// synchronisation sits between NMS and cropping.  Inside a CTA one producer warp walks the
-// tiles: it resolves the item, builds the table of horizontal taps (byte offset + exact
+// Crop-resize: bound by instruction issue and shared-memory wavefronts, then HBM (the fp16
+// output is as large as the source rectangles).  A persistent grid works through (slot, row
+// band) tiles that an atomic counter hands out (whole crops, except that the last crops of a
+// launch are cut into bands so that the grid ends together), so no host synchronisation sits
+// between NMS and cropping.  Inside a CTA one producer warp walks its tiles: it resolves the
+// item, builds the table of horizontal taps (byte offset + exact
 // integer weights per output column) and has the bulk-copy engine stage the 16-byte aligned
 // segments of the source rows a pass taps into one of two shared-memory buffers (mbarrier
 // "full" / "empty" ring, every wait bounded).  The 256 threads of the eight consumer warps
