@@ -80,3 +80,44 @@ def test_workspace_and_stats(stage):
     s = stage.stats()
     assert s["candidates"] == 0 and s["kept"] == 0 and s["status_word"] == 0
     assert stage.status() == 0
+
+
+def test_repeated_passes_are_bit_identical():
+    """Candidate append order, tile hand-out and the scheduler words change from launch to launch;
+    the results must not: 40 passes over the same batch, two stages interleaved on two streams."""
+    import numpy as np
+    import workloads
+    from gpu_harness import make_stage
+
+    b = workloads.make_batch("traffic_1080p", batch=3)
+    wl = b.workload
+    dev = torch.device("cuda", 0)
+    stages = [make_stage(wl, b.n), make_stage(wl, b.n)]
+    streams = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    try:
+        frames = [torch.from_numpy(f).to(dev) for f in b.frames]
+        head = torch.from_numpy(b.head).to(dev)
+        first = None
+        for it in range(40):
+            st, s = stages[it % 2], streams[it % 2]
+            with torch.cuda.stream(s):
+                det_in = st.preprocess(frames, b.sizes, stream=s)
+                dets, counts = st.postprocess(head, stream=s)
+                crops, offsets, n_items = st.crop(0, 200, stream=s)
+                crops2, _, _ = st.crop(0, 7, first_item=5, stream=s)  # a second window on the same stage
+            s.synchronize()
+            packed = int(n_items[0])
+            cur = (det_in.view(torch.int16).cpu().numpy(), dets.cpu().numpy()[:, :40], counts.cpu().numpy(),
+                   crops[:packed].view(torch.int16).cpu().numpy(), offsets.cpu().numpy(),
+                   crops2.view(torch.int16).cpu().numpy())
+            if first is None:
+                first = cur
+                assert packed > 20
+            else:
+                for x, y in zip(cur, first):
+                    assert np.array_equal(x, y)
+            assert np.array_equal(cur[5], cur[3][5:12])
+            assert st.status(s) & ~0x2 == 0  # the small second window is truncated by design
+    finally:
+        for st in stages:
+            st.close()
