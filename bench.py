@@ -43,13 +43,13 @@ NCU_TRAFFIC = {
     # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md); decode_planes on the
     # anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "b45affcf6a21acdf", 473898.6, "crop"),
+             "e28c1196c4fd4154", 473086.2, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                  "e8dcf55213e0dc25", 3694980.0, "frame"),
+                  "3423e26f20e7cf7a", 3699516.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "c2fb71b4332d2670", 1700720.0, "frame"),
+               "1b4ca10d57b78340", 1707712.0, "frame"),
     "decode_planes": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                      "c2fb71b4332d2670", 2813744.0, "frame"),
+                      "1b4ca10d57b78340", 2816568.0, "frame"),
 }
 
 

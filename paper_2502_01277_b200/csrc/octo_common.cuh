@@ -154,6 +154,58 @@ __device__ __forceinline__ void sample_px(uint32_t row0, uint32_t row_step, cons
     }
 }
 
+// Packed binary32 arithmetic (two independent IEEE operations per instruction, sm_100): the
+// two pixels of a pair go through the vertical lerp together.
+__device__ __forceinline__ unsigned long long f32x2(float lo, float hi) {
+    unsigned long long v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// binary16 pair from a packed binary32 pair (low element in the low half)
+__device__ __forceinline__ uint32_t half2_of_f32x2(unsigned long long v) {
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// Two neighbouring destination pixels (table entries ea, eb) of one output row: the integer
+// horizontal lerps as in sample_px, then the vertical lerp and scaling of both pixels in packed
+// arithmetic.  p0 / p1 / p2 receive (pixel a, pixel b) of the three input channels; every
+// element goes through the same individually rounded operations as in sample_px.
+template <bool LERP_Y>
+__device__ __forceinline__ void sample_pair(uint32_t row0, uint32_t row_step, uint32_t offa, uint32_t wtsa,
+                                            uint32_t offb, uint32_t wtsb, float wx, float nwx, float wy,
+                                            unsigned long long& p0, unsigned long long& p1, unsigned long long& p2) {
+    const uint32_t addra = row0 + (offa & ~3u), sha = offa << 3;
+    const uint32_t addrb = row0 + (offb & ~3u), shb = offb << 3;
+    float a0, a1, a2, b0, b1, b2;
+    hsample(addra, sha, wtsa, a0, a1, a2);
+    hsample(addrb, shb, wtsb, b0, b1, b2);
+    const unsigned long long wx2 = f32x2(wx, wx), nwx2 = f32x2(nwx, nwx);
+    p0 = fma_f32x2(f32x2(a0, b0), wx2, nwx2);
+    p1 = fma_f32x2(f32x2(a1, b1), wx2, nwx2);
+    p2 = fma_f32x2(f32x2(a2, b2), wx2, nwx2);
+    if (LERP_Y) {
+        hsample(addra + row_step, sha, wtsa, a0, a1, a2);
+        hsample(addrb + row_step, shb, wtsb, b0, b1, b2);
+        const unsigned long long wy2 = f32x2(wy, wy), m2 = f32x2(-kF32IntValue, -kF32IntValue);
+        p0 = fma_f32x2(add_f32x2(f32x2(a0, b0), m2), wy2, p0);
+        p1 = fma_f32x2(add_f32x2(f32x2(a1, b1), m2), wy2, p1);
+        p2 = fma_f32x2(add_f32x2(f32x2(a2, b2), m2), wy2, p2);
+    }
+}
+
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
     __half2 h = __floats2half2_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);

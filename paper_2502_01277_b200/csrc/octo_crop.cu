@@ -394,30 +394,40 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 const uint4 ee = lds128(xt + 16u * (uint32_t)pair);
                 const float wx = __uint_as_float(rw.z), wy = __uint_as_float(rw.w);
                 const float nwx = -kF32IntValue * wx;
-                float a0, a1, a2, b0, b1, b2;
-                if (GENERAL && (int)rw.y < 0) {  // canvas row
-                    a0 = b0 = opts.fill[0]; a1 = b1 = opts.fill[1]; a2 = b2 = opts.fill[2];
+                if (!GENERAL) {
+                    unsigned long long p0, p1, p2;
+                    if (wy != 0.0f) sample_pair<true>(rows + rw.x, rw.y, ee.x, ee.y, ee.z, ee.w, wx, nwx, wy, p0, p1, p2);
+                    else sample_pair<false>(rows + rw.x, rw.y, ee.x, ee.y, ee.z, ee.w, wx, nwx, wy, p0, p1, p2);
+                    const uint32_t o = (uint32_t)(r * ow + 2 * pair);
+                    *reinterpret_cast<uint32_t*>(t0 + o) = half2_of_f32x2(p0);
+                    *reinterpret_cast<uint32_t*>(t1 + o) = half2_of_f32x2(p1);
+                    *reinterpret_cast<uint32_t*>(t2 + o) = half2_of_f32x2(p2);
                 } else {
-                    if (wy != 0.0f) {
-                        sample_px<true>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
-                        sample_px<true>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+                    float a0, a1, a2, b0, b1, b2;
+                    if (GENERAL && (int)rw.y < 0) {  // canvas row
+                        a0 = b0 = opts.fill[0]; a1 = b1 = opts.fill[1]; a2 = b2 = opts.fill[2];
                     } else {
-                        sample_px<false>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
-                        sample_px<false>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+                        if (wy != 0.0f) {
+                            sample_px<true>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
+                            sample_px<true>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+                        } else {
+                            sample_px<false>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
+                            sample_px<false>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+                        }
+                        if (GENERAL) {
+                            a0 = ee.y ? fmaf(a0, opts.sc[0], opts.of[0]) : opts.fill[0];
+                            a1 = ee.y ? fmaf(a1, opts.sc[1], opts.of[1]) : opts.fill[1];
+                            a2 = ee.y ? fmaf(a2, opts.sc[2], opts.of[2]) : opts.fill[2];
+                            b0 = ee.w ? fmaf(b0, opts.sc[0], opts.of[0]) : opts.fill[0];
+                            b1 = ee.w ? fmaf(b1, opts.sc[1], opts.of[1]) : opts.fill[1];
+                            b2 = ee.w ? fmaf(b2, opts.sc[2], opts.of[2]) : opts.fill[2];
+                        }
                     }
-                    if (GENERAL) {
-                        a0 = ee.y ? fmaf(a0, opts.sc[0], opts.of[0]) : opts.fill[0];
-                        a1 = ee.y ? fmaf(a1, opts.sc[1], opts.of[1]) : opts.fill[1];
-                        a2 = ee.y ? fmaf(a2, opts.sc[2], opts.of[2]) : opts.fill[2];
-                        b0 = ee.w ? fmaf(b0, opts.sc[0], opts.of[0]) : opts.fill[0];
-                        b1 = ee.w ? fmaf(b1, opts.sc[1], opts.of[1]) : opts.fill[1];
-                        b2 = ee.w ? fmaf(b2, opts.sc[2], opts.of[2]) : opts.fill[2];
-                    }
+                    const uint32_t o = (uint32_t)(r * ow + 2 * pair);
+                    *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(a0, b0);
+                    *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(a1, b1);
+                    *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(a2, b2);
                 }
-                const uint32_t o = (uint32_t)(r * ow + 2 * pair);
-                *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(a0, b0);
-                *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(a1, b1);
-                *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(a2, b2);
                 r += dr;
                 pair += dp;
                 if (pair >= pairs) { pair -= pairs; ++r; }
