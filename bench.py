@@ -199,6 +199,16 @@ def oracle_pass(batch, frames_used: int, threads: int) -> float:
     return time.perf_counter() - t0
 
 
+def cpu_model() -> str:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.lower().startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def cpu_sample_frames(batch_n: int, cores: int) -> int:
     # about 0.25 s of single-core work per 1080p frame -> roughly 5-20 s of wall time
     return max(1, min(batch_n, 64 * cores))
@@ -531,8 +541,12 @@ def run_octo(args):
         cores = len(os.sched_getaffinity(0))
         sample = cpu_sample_frames(n, cores)
         t = oracle_pass(batch, sample, cores)
+        one = min(n, 8)
+        t1 = oracle_pass(batch, one, 1)
         cpu = {"value": sample / t, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"first {sample} of {n} frames, whole stage, {cores} threads, {t:.1f} s"}
+               "sample": f"first {sample} of {n} frames, whole stage, {cores} threads, {t:.1f} s",
+               "single_thread": {"value": one / t1, "unit": UNIT, "sample": f"first {one} frames, {t1:.1f} s"},
+               "cpu_model": cpu_model()}
 
     if rank == 0:
         line = {
