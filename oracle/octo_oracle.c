@@ -411,6 +411,27 @@ int32_t orc_postprocess_region(const float* head, int32_t A, int32_t C, int32_t 
     return k;
 }
 
+/* The same for the decode variants of orc_decode_ex (head layout, multi-label candidates). */
+int32_t orc_postprocess_region_v2(const float* head, int32_t A, int32_t C, int32_t logits, float conf,
+                                  float iou_thr, int32_t max_det, int32_t S, int32_t ox, int32_t oy,
+                                  int32_t rw, int32_t rh, int32_t layout, int32_t multi_label,
+                                  orc_det_t* dets, int32_t* n_cand) {
+    const size_t cap = (size_t)(A > 0 ? A : 1) * (size_t)(multi_label ? (C > 0 ? C : 1) : 1);
+    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * cap);
+    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
+    int32_t n = orc_decode_ex(head, A, C, logits, conf, layout, multi_label, cand, (int32_t)cap);
+    orc_sort(cand, n);
+    int32_t k = orc_nms(cand, n, iou_thr, max_det, keep);
+    for (int32_t t = 0; t < k; ++t) {
+        dets[t] = cand[keep[t]];
+        orc_scale_back_region(&dets[t], S, S, 0, 0, ox, oy, rw, rh);
+    }
+    if (n_cand) *n_cand = n;
+    free(cand);
+    free(keep);
+    return k;
+}
+
 /* R7: integer crop rectangle of a frame-space box: rx0 = clamp(floor(X1), 0, w-1),
  * rx1 = clamp(ceil(X2), rx0+1, w), same in y.  rect = {rx0, ry0, rx1, ry1}. */
 void orc_crop_rect(const orc_det_t* d, int32_t w, int32_t h, int32_t* rect) {

@@ -70,6 +70,8 @@ def _load():
     lib.orc_postprocess_image.restype = i32
     lib.orc_postprocess_region.argtypes = [vp, i32, i32, i32, f32, f32, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.orc_postprocess_region.restype = i32
+    lib.orc_postprocess_region_v2.argtypes = [vp, i32, i32, i32, f32, f32, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp]
+    lib.orc_postprocess_region_v2.restype = i32
     lib.orc_crop_rect.argtypes = [vp, i32, i32, vp]
     lib.orc_crop_rect.restype = None
     lib.orc_crop.argtypes = [vp, i32, i32, i32, vp, i32, i32, i32, vp]
@@ -219,17 +221,25 @@ def postprocess_image(head: np.ndarray, w: int, h: int, s: int, logits: bool = T
 
 
 def postprocess_region(head: np.ndarray, region: Tuple[int, int, int, int], s: int, logits: bool = True,
-                       conf: float = 0.25, iou_thr: float = 0.45, max_det: int = 300):
-    """Chained stage: head [A, 5+C] of one upstream crop (rectangle region = (rx0, ry0, rx1, ry1)
-    stretched to s x s) -> (dets in ORIGINAL-frame pixels [kept], candidate count)."""
+                       conf: float = 0.25, iou_thr: float = 0.45, max_det: int = 300, layout: str = "rows",
+                       multi_label: bool = False):
+    """Chained stage: head (rows [A, 5+C] or planes [4+C, A]) of one upstream crop (rectangle
+    region = (rx0, ry0, rx1, ry1) stretched to s x s) -> (dets in ORIGINAL-frame pixels [kept],
+    candidate count)."""
     hd = np.ascontiguousarray(head, dtype=np.float32)
-    a, row = hd.shape
     dets = np.zeros(max(max_det, 1), dtype=DET_DTYPE)
     ncand = np.zeros(1, dtype=np.int32)
     rx0, ry0, rx1, ry1 = (int(v) for v in region)
-    k = _load().orc_postprocess_region(_ptr(hd), a, row - 5, 1 if logits else 0, np.float32(conf),
-                                       np.float32(iou_thr), max_det, s, rx0, ry0, rx1 - rx0, ry1 - ry0,
-                                       _ptr(dets), _ptr(ncand))
+    if layout == "rows" and not multi_label:
+        a, row = hd.shape
+        k = _load().orc_postprocess_region(_ptr(hd), a, row - 5, 1 if logits else 0, np.float32(conf),
+                                           np.float32(iou_thr), max_det, s, rx0, ry0, rx1 - rx0, ry1 - ry0,
+                                           _ptr(dets), _ptr(ncand))
+    else:
+        a, c = _head_dims(hd, layout)
+        k = _load().orc_postprocess_region_v2(_ptr(hd), a, c, 1 if logits else 0, np.float32(conf),
+                                              np.float32(iou_thr), max_det, s, rx0, ry0, rx1 - rx0, ry1 - ry0,
+                                              LAYOUTS[layout], 1 if multi_label else 0, _ptr(dets), _ptr(ncand))
     return dets[:k].copy(), int(ncand[0])
 
 

@@ -19,7 +19,13 @@ from oracle import DET_DTYPE
 pytestmark = pytest.mark.gpu
 
 
-def test_two_level_cascade_matches_oracle():
+MEAN, STD = (0.485, 0.456, 0.406), (0.229, 0.224, 0.225)
+
+
+@pytest.mark.parametrize("layout2,opts2", [("rows", None), ("planes", {"keep_aspect": True, "mean": MEAN, "std": STD})])
+def test_two_level_cascade_matches_oracle(layout2, opts2):
+    """Second level with a row head and plain crops, and with an anchor-free planes head whose
+    crops keep their aspect ratio and are normalised."""
     wl = replace(workloads.WORKLOADS["traffic_1080p"], branches=((256, 256),))
     b = workloads.make_batch(wl, batch=3, seed=31)
     s2, c2, max_det2 = 256, 6, 12
@@ -43,8 +49,10 @@ def test_two_level_cascade_matches_oracle():
                               ref1.rects[0])
         # ---- level 2: the 256x256 crops are the detector input; heads are synthetic
         head2 = workloads.make_heads(77, n1, s2, num_classes=c2, n_raised=14, n_groups=4)
+        if layout2 == "planes":
+            head2 = np.stack([workloads.rows_to_planes(h) for h in head2])
         st2 = octo.Stage(net_size=s2, max_batch=n1, num_anchors=a2, num_classes=c2, max_det=max_det2,
-                         branches=((64, 32),))
+                         branches=((64, 32),), head_layout=layout2, crop_options=[opts2])
         st2.adopt_regions(frames, b.sizes, items1)
         dets2, counts2 = st2.postprocess(torch.from_numpy(head2).cuda())
         cap2 = n1 * max_det2
@@ -61,7 +69,7 @@ def test_two_level_cascade_matches_oracle():
         ref_c = np.zeros(n1, dtype=np.int32)
         for i in range(n1):
             r = ref1.rects[0][i]
-            d, _ = oracle.postprocess_region(head2[i], tuple(int(v) for v in r), s2, max_det=max_det2)
+            d, _ = oracle.postprocess_region(head2[i], tuple(int(v) for v in r), s2, max_det=max_det2, layout=layout2)
             ref_d[i, : len(d)] = d
             ref_c[i] = len(d)
         assert np.array_equal(c2n, ref_c) and int(ref_c.sum()) > n1
@@ -79,7 +87,7 @@ def test_two_level_cascade_matches_oracle():
             w, h = b.sizes[f]
             rect = oracle.crop_rect(ref_d[i, j], w, h)
             assert (int(items2["rx0"][k]), int(items2["ry0"][k]), int(items2["rx1"][k]), int(items2["ry1"][k])) == rect
-            want = oracle.crop(b.frames[f], w, h, ref_d[i, j], 64, 32)
+            want = oracle.crop(b.frames[f], w, h, ref_d[i, j], 64, 32, **(opts2 or {}))
             assert half_absdiff(got[k], want) <= 2e-3
         assert np.all(got[packed2:] == 0x7BFF)
     finally:

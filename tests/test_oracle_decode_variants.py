@@ -138,3 +138,16 @@ def test_anchor_free_workload_counts():
         dets, ncand = o.postprocess_image(b.head[i], 1920, 1080, 640, layout="planes")
         assert ncand == wl.n_raised and 15 <= len(dets) <= 60
         assert np.all(np.diff(dets["score"]) <= 0)
+
+
+def test_chained_stage_with_planes_head_reduces_to_the_row_form():
+    """A chained stage's planes head equals the row head with unit objectness (sigma(30) == 1.0f):
+    same detections, mapped into the same upstream rectangle."""
+    h = workloads.make_heads(77, 2, 256, num_classes=6, n_raised=14, n_groups=4)
+    h[:, :, 4] = 30.0
+    for i in range(2):
+        region = (10 + i, 20, 200, 150 + i)
+        want, nw = o.postprocess_region(h[i], region, 256, max_det=12)
+        got, ng = o.postprocess_region(workloads.rows_to_planes(h[i]), region, 256, max_det=12, layout="planes")
+        assert nw == ng and len(want) > 3 and np.array_equal(got, want)
+        assert np.all((want["x1"] >= region[0]) & (want["x2"] <= region[2]))
