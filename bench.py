@@ -43,7 +43,7 @@ NCU_TRAFFIC = {
     # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md); decode_planes on the
     # anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "e28c1196c4fd4154", 473086.2, "crop"),
+             "b86f4bd9895afd72", 473086.2, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
                   "3423e26f20e7cf7a", 3699516.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),

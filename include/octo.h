@@ -279,6 +279,11 @@ OCTO_API int octo_queue_create(int32_t device, int32_t capacity, int32_t out_w, 
                                int32_t max_bz, octo_queue_t** out);
 OCTO_API int octo_queue_destroy(octo_queue_t* q);
 
+/* Crop options of the queue's downstream model: keep_aspect, normalize, mean and std of *options
+ * are used as in octo_branch_cfg_t (its other fields are ignored), pad_value (0..255) fills the
+ * canvas of aspect-preserving crops.  Takes effect from the next pop.  Errors: OCTO_E_INVALID_ARG. */
+OCTO_API int octo_queue_set_options(octo_queue_t* q, const octo_branch_cfg_t* options, int32_t pad_value);
+
 /* Append the items of `branch` of the stage's current batch (after octo_postprocess_batch;
  * same item order and rectangles as octo_crop_batch would use).  Enqueues one kernel.
  * Errors: OCTO_E_INVALID_ARG, OCTO_E_NO_PREPROCESS, OCTO_E_NO_POSTPROCESS, OCTO_E_CUDA. */

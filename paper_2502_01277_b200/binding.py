@@ -47,7 +47,7 @@ EXPORTS = (
     "octo_stage_workspace_bytes", "octo_stage_launch_count",
     "octo_strerror", "octo_last_cuda_error", "octo_version", "octo_postprocess_frame_static",
     "octo_adopt_regions", "octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop",
-    "octo_queue_pop_due", "octo_coral_schedule",
+    "octo_queue_pop_due", "octo_coral_schedule", "octo_queue_set_options",
 )
 
 
@@ -170,6 +170,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_queue_destroy.argtypes = [vp]
     lib.octo_queue_push.argtypes = [vp, vp, i32, vp]
     lib.octo_queue_pop.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.octo_queue_set_options.argtypes = [vp, ctypes.POINTER(BranchCfg), i32]
+    lib.octo_queue_set_options.restype = ctypes.c_int
     lib.octo_queue_pop_due.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     lib.octo_queue_pop_due.restype = ctypes.c_int
     for name in ("octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop"):
@@ -473,6 +475,19 @@ class Queue:
         if stream is None:
             stream = self._torch.cuda.current_stream(self.device)
         return int(stream.cuda_stream)
+
+    def set_options(self, keep_aspect: bool = False, mean=None, std=None, pad_value: int = 114) -> None:
+        """Crop options of the downstream model (see octo_branch_cfg_t)."""
+        br = BranchCfg()
+        br.keep_aspect = 1 if keep_aspect else 0
+        if mean is not None or std is not None:
+            br.normalize = 1
+            for k in range(3):
+                br.mean[k] = float((mean or (0.0, 0.0, 0.0))[k])
+                br.std[k] = float((std or (1.0, 1.0, 1.0))[k])
+        rc = load_library().octo_queue_set_options(self.handle, ctypes.byref(br), pad_value)
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_queue_set_options")
 
     def push(self, stage: "Stage", branch: int = 0, stream=None) -> None:
         rc = load_library().octo_queue_push(self.handle, stage.handle, branch, self._stream(stream))

@@ -479,7 +479,7 @@ cudaError_t prepare_crop() {
         (const void*)crop_kernel<8, false, false>,   (const void*)crop_kernel<8, false, true>,
         (const void*)crop_kernel<64, false, false>,  (const void*)crop_kernel<64, false, true>,
         (const void*)crop_kernel<512, false, false>, (const void*)crop_kernel<512, false, true>,
-        (const void*)crop_kernel<8, true, false>,
+        (const void*)crop_kernel<8, true, false>,    (const void*)crop_kernel<8, true, true>,
     };
     for (const void* k : kernels) {
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -497,7 +497,8 @@ cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream) {
 
 // Crop the records staged by a queue pop (at most bz of them) into the downstream batch.
 cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int bz, void* d_out, int out_w,
-                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, int* d_sched, cudaStream_t stream) {
+                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, int* d_sched,
+                              const CropOpts* general, cudaStream_t stream) {
     static FrameTable<8> tab;  // unused in queue mode
     const long long cap = (long long)sm_count * kCropCtasPerSm;
     const long long work = (long long)bz * ((out_h + 7) / 8);
@@ -505,9 +506,14 @@ cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int
     const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)out_w;
     CropOpts opts;
     memset(&opts, 0, sizeof(opts));
-    crop_kernel<8, true, false><<<grid, kCropKernelThreads, smem, stream>>>(
-        tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
-        out_w, out_h, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched, opts);
+    if (general)
+        crop_kernel<8, true, true><<<grid, kCropKernelThreads, smem, stream>>>(
+            tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
+            out_w, out_h, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched, *general);
+    else
+        crop_kernel<8, true, false><<<grid, kCropKernelThreads, smem, stream>>>(
+            tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
+            out_w, out_h, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched, opts);
     return cudaGetLastError();
 }
 

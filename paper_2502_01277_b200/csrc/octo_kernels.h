@@ -73,6 +73,10 @@ struct CropArgs {
     CropOpts opts;
 };
 
+// Branch options -> kernel form (per input channel, see CropOpts).
+void fill_crop_opts(const octo_branch_cfg_t& br, int swap_rb, int pad_value, CropOpts* out);
+int validate_branch_options(const octo_branch_cfg_t& br);  // OCTO_OK or OCTO_E_INVALID_ARG
+
 // Opt the kernels of every table capacity into the shared memory they need (current device).
 cudaError_t prepare_letterbox();
 cudaError_t prepare_nms();
@@ -84,7 +88,8 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
 cudaError_t launch_nms(const NmsArgs& a, cudaStream_t stream);
 cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream);  // batch assembler + crop-resize
 cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int bz, void* d_out, int out_w,
-                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, int* d_sched, cudaStream_t stream);
+                              int out_h, int swap_rb, int sm_count, unsigned int* d_status, int* d_sched,
+                              const CropOpts* general, cudaStream_t stream);
 
 constexpr int kLetterboxMaxWidth = 8192;  // widest frame the row staging supports
 

@@ -136,6 +136,8 @@ struct octo_queue {
     QRecord* d_staged;
     QueueState* d_state;
     int* d_qpacked;
+    bool general;   // crop options set (octo_queue_set_options)
+    CropOpts opts;
 };
 
 static void queue_free(octo_queue* q) {
@@ -175,6 +177,14 @@ extern "C" int octo_queue_create(int32_t device, int32_t capacity, int32_t out_w
         return OCTO_E_CUDA;
     }
     *out = q;
+    return OCTO_OK;
+}
+
+extern "C" int octo_queue_set_options(octo_queue_t* q, const octo_branch_cfg_t* options, int32_t pad_value) {
+    if (!q || !options || pad_value < 0 || pad_value > 255) return OCTO_E_INVALID_ARG;
+    if (validate_branch_options(*options) != OCTO_OK) return OCTO_E_INVALID_ARG;
+    q->general = options->keep_aspect != 0 || options->normalize != 0;
+    fill_crop_opts(*options, q->swap_rb, pad_value, &q->opts);
     return OCTO_OK;
 }
 
@@ -218,6 +228,6 @@ extern "C" int octo_queue_pop_due(octo_queue_t* q, int32_t bz, int32_t max_wait,
                                            reinterpret_cast<QRecord*>(d_items_out), d_info, q->d_qpacked);
     if (cudaGetLastError() != cudaSuccess) return OCTO_E_CUDA;
     cudaError_t e = launch_crop_queue(q->d_staged, q->d_qpacked, bz, d_out_f16, q->out_w, q->out_h, q->swap_rb,
-                                      q->sm_count, &q->d_state->status, q->d_state->sched, stream);
+                                      q->sm_count, &q->d_state->status, q->d_state->sched, q->general ? &q->opts : nullptr, stream);
     return e == cudaSuccess ? OCTO_OK : OCTO_E_CUDA;
 }

@@ -62,17 +62,37 @@ static int validate_config(const octo_stage_config_t* c) {
         const octo_branch_cfg_t& br = c->branch[b];
         if (br.out_w < 8 || br.out_w > 2048 || (br.out_w & 7)) return OCTO_E_INVALID_ARG;
         if (br.out_h < 1 || br.out_h > 2048) return OCTO_E_INVALID_ARG;
-        if (br.keep_aspect != 0 && br.keep_aspect != 1) return OCTO_E_INVALID_ARG;
-        if (br.normalize != 0 && br.normalize != 1) return OCTO_E_INVALID_ARG;
-        if (br.normalize) {
-            for (int k = 0; k < 3; ++k) {
-                if (!(fabsf(br.mean[k]) <= 1e6f)) return OCTO_E_INVALID_ARG;          // finite, sane
-                if (!(br.std[k] >= 1e-6f) || !(br.std[k] <= 1e6f)) return OCTO_E_INVALID_ARG;
-            }
+        if (octo::validate_branch_options(br) != OCTO_OK) return OCTO_E_INVALID_ARG;
+    }
+    return OCTO_OK;
+}
+
+namespace octo {
+// branch options, expressed per input channel c (it lands in output plane swap ? 2 - c : c)
+void fill_crop_opts(const octo_branch_cfg_t& br, int swap_rb, int pad_value, CropOpts* out) {
+    out->keep_aspect = br.keep_aspect;
+    for (int ch = 0; ch < 3; ++ch) {
+        const int p = swap_rb ? 2 - ch : ch;
+        const double m = br.normalize ? (double)br.mean[p] : 0.0, sd = br.normalize ? (double)br.std[p] : 1.0;
+        out->sc[ch] = (float)(1.0 / sd);
+        out->of[ch] = (float)(-m / sd);
+        out->fill[ch] = (float)(((double)pad_value / 255.0 - m) / sd);
+    }
+}
+
+// shared by octo_stage_create and octo_queue_set_options
+int validate_branch_options(const octo_branch_cfg_t& br) {
+    if (br.keep_aspect != 0 && br.keep_aspect != 1) return OCTO_E_INVALID_ARG;
+    if (br.normalize != 0 && br.normalize != 1) return OCTO_E_INVALID_ARG;
+    if (br.normalize) {
+        for (int k = 0; k < 3; ++k) {
+            if (!(fabsf(br.mean[k]) <= 1e6f)) return OCTO_E_INVALID_ARG;          // finite, sane
+            if (!(br.std[k] >= 1e-6f) || !(br.std[k] <= 1e6f)) return OCTO_E_INVALID_ARG;
         }
     }
     return OCTO_OK;
 }
+}  // namespace octo
 
 template <typename T>
 static cudaError_t dev_alloc(T** p, size_t count, int64_t* total) {
@@ -346,19 +366,8 @@ extern "C" int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_i
     a.swap_rb = c.swap_rb;
     a.sm_count = st->sm_count;
     a.d_ctr = st->d_ctr;
-    {
-        // branch options, expressed per input channel c (it lands in output plane swap ? 2 - c : c)
-        const octo_branch_cfg_t& br = c.branch[branch];
-        a.general = br.keep_aspect != 0 || br.normalize != 0;
-        a.opts.keep_aspect = br.keep_aspect;
-        for (int ch = 0; ch < 3; ++ch) {
-            const int p = c.swap_rb ? 2 - ch : ch;
-            const double m = br.normalize ? (double)br.mean[p] : 0.0, sd = br.normalize ? (double)br.std[p] : 1.0;
-            a.opts.sc[ch] = (float)(1.0 / sd);
-            a.opts.of[ch] = (float)(-m / sd);
-            a.opts.fill[ch] = (float)(((double)c.pad_value / 255.0 - m) / sd);
-        }
-    }
+    a.general = c.branch[branch].keep_aspect != 0 || c.branch[branch].normalize != 0;
+    fill_crop_opts(c.branch[branch], c.swap_rb, c.pad_value, &a.opts);
     OCTO_CUDA(cudaSetDevice(c.device));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     {

@@ -16,12 +16,14 @@ pytestmark = pytest.mark.gpu
 OW, OH = 64, 48
 
 
-def _run(capacity, bz, pops_between, final_pops, max_wait=-1):
+def _run(capacity, bz, pops_between, final_pops, max_wait=-1, options=None):
     wl = workloads.WORKLOADS["traffic_1080p"]
     batches = [workloads.make_batch("traffic_1080p", batch=nb, first_frame=ff) for nb, ff in ((2, 0), (3, 10), (1, 20))]
     st = make_stage(wl, 4, branches=((OW, OH),))
     q = octo.Queue(capacity, OW, OH, max_bz=bz)
     oq = oracle.OracleQueue(capacity)
+    if options:
+        q.set_options(**options)
     got, want = [], []
     try:
         keep = []
@@ -58,7 +60,7 @@ def _run(capacity, bz, pops_between, final_pops, max_wait=-1):
                 box = np.zeros(1, dtype=oracle.DET_DTYPE)
                 box["x1"], box["y1"], box["x2"], box["y2"] = rect  # integer box -> the same rectangle
                 assert oracle.crop_rect(box, w, h) == rect
-                assert half_absdiff(crops[i], oracle.crop(pix, w, h, box, OW, OH)) <= 2e-3
+                assert half_absdiff(crops[i], oracle.crop(pix, w, h, box, OW, OH, **(options or {}))) <= 2e-3
             assert np.all(crops[len(orecs):] == 0x7BFF)
         return want
     finally:
@@ -88,6 +90,19 @@ def test_queue_release_rule_decided_on_the_device():
     assert infos[0][0] == 0 and infos[0][1] > 0          # first batch alone: not full, not due
     assert any(i[0] == 64 for i in infos) or infos[2][0] > 0
     assert sum(i[0] for i in infos) > 0
+
+
+def test_queue_with_crop_options():
+    _run(capacity=96, bz=32, pops_between=(1, 1, 0), final_pops=2,
+         options=dict(keep_aspect=True, mean=(0.485, 0.456, 0.406), std=(0.229, 0.224, 0.225), pad_value=30))
+    q = octo.Queue(16, 64, 48, max_bz=8)
+    try:
+        with pytest.raises(octo.OctoError):
+            q.set_options(std=(0.2, 0.0, 0.2))
+        with pytest.raises(octo.OctoError):
+            q.set_options(pad_value=300)
+    finally:
+        q.close()
 
 
 def test_queue_argument_errors():
