@@ -474,8 +474,9 @@ def run_octo(args):
         "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})", "unit": "GB/s",
         "frac": kern[dominant]["gbs"] / hbm_peak, "frac_of_nominal_8TBs": kern[dominant]["gbs"] / 8000.0,
         "alg_bytes_per_launch": alg[dominant], "ms_per_launch": kern[dominant]["ms_per_launch"],
-        "traffic": traffic_for("decode_planes" if dominant == "decode" and wl.head_layout == "planes" else dominant,
-                               units),
+        # the per-unit ncu figures were taken on 1080p frames and 224x224 crops: other shapes get none
+        "traffic": (traffic_for("decode_planes" if dominant == "decode" and wl.head_layout == "planes" else dominant,
+                                units) if name in ("sweep", "anchor_free") else None),
     }
 
     # ---- end to end from pinned host buffers ----
