@@ -43,13 +43,13 @@ NCU_TRAFFIC = {
     # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md); decode_planes on the
     # anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "b86f4bd9895afd72", 473086.2, "crop"),
+             "a2adfd8f629814cc", 472654.6, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                  "3423e26f20e7cf7a", 3699516.0, "frame"),
+                  "ad30360af87ae8e6", 3695876.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "1b4ca10d57b78340", 1707712.0, "frame"),
+               "2f5c19fd5c24faad", 1699900.0, "frame"),
     "decode_planes": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                      "1b4ca10d57b78340", 2816568.0, "frame"),
+                      "2f5c19fd5c24faad", 2811836.0, "frame"),
 }
 
 

@@ -216,25 +216,30 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
 // and the warp writes 128 contiguous bytes per plane and step.  row0 / xt are shared-space
 // addresses of the first staged row and of the tile's first table entry; o0 / o1 / o2 point
 // at the row's first pixel in the planes of input channels 0 / 1 / 2.  With FILL, columns
-// whose table entry has zero weights (canvas outside the image) receive fill_f.
+// whose table entry has zero weights (canvas outside the image) receive the binary16 fill value
+// (fill_h2 holds it in both halves).
 template <bool LERP_Y, bool FILL>
 __device__ __forceinline__ void sample_row(uint32_t row0, uint32_t row_step, float wx, float wy, uint32_t xt,
                                            int pairs, int lane, __half* __restrict__ o0, __half* __restrict__ o1,
-                                           __half* __restrict__ o2, float fill_f) {
+                                           __half* __restrict__ o2, uint32_t fill_h2) {
     const float nwx = -kF32IntValue * wx;
     for (int pair = lane; pair < pairs; pair += 32) {
         const uint4 ee = lds128(xt + 16u * (uint32_t)pair);  // two XEntry: {off, wts} x 2
-        float a0, a1, a2, b0, b1, b2;
-        sample_px<LERP_Y>(row0, row_step, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
-        sample_px<LERP_Y>(row0, row_step, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
+        unsigned long long p0, p1, p2;
+        sample_pair<LERP_Y>(row0, row_step, ee.x, ee.y, ee.z, ee.w, wx, nwx, wy, p0, p1, p2);
+        uint32_t h0 = half2_of_f32x2(p0), h1 = half2_of_f32x2(p1), h2 = half2_of_f32x2(p2);
         if (FILL) {
-            if (ee.y == 0u) { a0 = fill_f; a1 = fill_f; a2 = fill_f; }
-            if (ee.w == 0u) { b0 = fill_f; b1 = fill_f; b2 = fill_f; }
+            // canvas columns: replace the half of the pair that lies outside the image
+            const uint32_t keep = (ee.y == 0u ? 0u : 0x0000ffffu) | (ee.w == 0u ? 0u : 0xffff0000u);
+            const uint32_t fill = fill_h2 & ~keep;
+            h0 = (h0 & keep) | fill;
+            h1 = (h1 & keep) | fill;
+            h2 = (h2 & keep) | fill;
         }
         const uint32_t o = 2u * (uint32_t)pair;
-        *reinterpret_cast<uint32_t*>(o0 + o) = pack_half2(a0, b0);
-        *reinterpret_cast<uint32_t*>(o1 + o) = pack_half2(a1, b1);
-        *reinterpret_cast<uint32_t*>(o2 + o) = pack_half2(a2, b2);
+        *reinterpret_cast<uint32_t*>(o0 + o) = h0;
+        *reinterpret_cast<uint32_t*>(o1 + o) = h1;
+        *reinterpret_cast<uint32_t*>(o2 + o) = h2;
     }
 }
 

@@ -20,7 +20,7 @@ constexpr int kLbRows = 8;  // most output rows a CTA produces; fewer for very w
 template <int CAP>
 __global__ void __launch_bounds__(kLbThreads)
 letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict__ out, int S, int band_rows,
-                 int slot_bytes, uint32_t fill_h2, float fill_f, int swap_rb, unsigned int* __restrict__ status) {
+                 int slot_bytes, uint32_t fill_h2, int swap_rb, unsigned int* __restrict__ status) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t bar;
     __shared__ __align__(16) RowInfo s_row[kLbRows];  // per-row data; step < 0 marks a canvas (pad) row
@@ -122,10 +122,10 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
             }
         } else if (ri.wy != 0.0f) {
             sample_row<true, true>(rows_s + (uint32_t)ri.row0, (uint32_t)ri.step, ri.wx, ri.wy, xtab_s, pairs, lane,
-                                   out0 + o, out1 + o, out2 + o, fill_f);
+                                   out0 + o, out1 + o, out2 + o, fill_h2);
         } else {
             sample_row<false, true>(rows_s + (uint32_t)ri.row0, (uint32_t)ri.step, ri.wx, ri.wy, xtab_s, pairs, lane,
-                                    out0 + o, out1 + o, out2 + o, fill_f);
+                                    out0 + o, out1 + o, out2 + o, fill_h2);
         }
     }
 }
@@ -163,10 +163,9 @@ static cudaError_t launch_cap(const FrameDesc* frames, int n, void* d_out, int S
     const __half hf = __double2half((double)pad_value / 255.0);  // one rounding, nearest even
     const uint32_t fb = *reinterpret_cast<const unsigned short*>(&hf);
     const uint32_t fill_h2 = fb | (fb << 16);
-    const float fill_f = __half2float(hf);
     dim3 grid((S + band_rows - 1) / band_rows, n);
     letterbox_kernel<CAP><<<grid, kLbThreads, smem, stream>>>(tab, reinterpret_cast<__half*>(d_out), S, band_rows, slot_bytes,
-                                                             fill_h2, fill_f, swap_rb, d_status);
+                                                             fill_h2, swap_rb, d_status);
     return cudaGetLastError();
 }
 
