@@ -40,8 +40,7 @@ UNIT = "frames/s"
 # reported as null.
 NCU_TRAFFIC = {
     # kernel: (source files, sha256[:16] of their concatenation at capture time, bytes per unit, unit)
-    # captured on the sweep workload at B = 64 (profiles/*_kernel_sweep.md); decode_planes on the
-    # anchor_free workload at B = 64
+    # captured on the sweep workload at B = 64; decode_planes on the anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
              "a2adfd8f629814cc", 472654.6, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
@@ -103,6 +102,25 @@ def crop_bytes(items: np.ndarray, ow: int, oh: int) -> int:
     cw = (items["rx1"] - items["rx0"]).astype(np.int64)
     ch = (items["ry1"] - items["ry0"]).astype(np.int64)
     return int(len(items) * 3 * ow * oh * 2 + int((cw * ch * 3).sum()))
+
+
+def crop_compulsory_bytes(items: np.ndarray, sizes, ow: int, oh: int) -> int:
+    """What a crop launch cannot avoid moving through DRAM: the fp16 output of every packed crop +
+    every source byte that at least one rectangle covers, counted once per frame (rectangles of a
+    frame overlap; the second reader of a byte is served by L2)."""
+    total = int(len(items)) * 3 * ow * oh * 2
+    order = np.argsort(items["frame"], kind="stable")
+    it = items[order]
+    bounds = np.flatnonzero(np.diff(it["frame"])) + 1
+    for grp in np.split(it, bounds):
+        if len(grp) == 0:
+            continue
+        w, h = sizes[int(grp["frame"][0])]
+        mask = np.zeros((h, w), dtype=bool)
+        for r in grp:
+            mask[r["ry0"]:r["ry1"], r["rx0"]:r["rx1"]] = True
+        total += 3 * int(mask.sum())
+    return total
 
 
 def decode_bytes(n: int, a: int, c: int, candidates: int, logits: bool, layout: str = "rows") -> int:
@@ -325,17 +343,24 @@ def run_octo(args):
         if world > 1:
             dist.barrier()
 
-    def timed(nsteps, fn):
+    def timed(nsteps, fn, per_step=None):
+        """Device time of nsteps steps (max over ranks).  With per_step (a list), an event is also
+        recorded after every step and the step-to-step times (ms, this rank) are appended to it."""
         barrier()
         torch.cuda.synchronize(dev)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(nsteps + 1 if per_step is not None else 2)]
+        ev[0].record(stream)
         for i in range(nsteps):
             fn(i)
-        e1.record(stream)
+            if per_step is not None:
+                ev[i + 1].record(stream)
+        if per_step is None:
+            ev[1].record(stream)
         torch.cuda.synchronize(dev)
         barrier()
-        ms = e0.elapsed_time(e1)
+        ms = ev[0].elapsed_time(ev[-1])
+        if per_step is not None:
+            per_step.extend(ev[i].elapsed_time(ev[i + 1]) for i in range(nsteps))
         if world > 1:
             t = torch.tensor([ms], dtype=torch.float64, device=dev)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -372,13 +397,35 @@ def run_octo(args):
         for i in range(3):
             replay(i)
         launches0 = stage.launch_count
+        run_step = replay
         ms_total = timed(args.steps, replay)
         gpu_launches = launches_per_step * args.steps  # kernels run from the graph, not counted by the stage
     else:
-        ms_total = timed(args.steps, lambda i: step(sets[i % n_sets]))
+        run_step = lambda i: step(sets[i % n_sets])  # noqa: E731
+        ms_total = timed(args.steps, run_step)
         gpu_launches = stage.launch_count - launches0
     ms_per_step = ms_total / args.steps
     value = world * n / (ms_per_step * 1e-3)
+
+    # ---- distribution over single steps: >= 50 steps, an event after each one ----
+    # (informational: `value` above is the plain K-step figure; a per-step event keeps the next
+    # launch from overlapping the end of the step, which costs small batches a few microseconds)
+    dist_steps = max(50, args.steps)
+    per = []
+    timed(dist_steps, run_step, per_step=per)
+    step_stats = {"steps": dist_steps, "ms_median": statistics.median(per), "ms_min": min(per),
+                  "us_per_pass_median": 1e3 * statistics.median(per), "us_per_pass_min": 1e3 * min(per)}
+    # the L2-warm figure of small batches: one input/output set over and over (it fits L2)
+    l2_warm = None
+    if n <= 16 and n_sets > 1:
+        warm_fn = (lambda i: replay(0)) if args.graph else (lambda i: step(sets[0]))
+        for i in range(3):
+            warm_fn(i)
+        perw = []
+        timed(dist_steps, warm_fn, per_step=perw)
+        l2_warm = {"steps": dist_steps, "ms_median": statistics.median(perw), "ms_min": min(perw),
+                   "frames_per_s_median": world * n / (statistics.median(perw) * 1e-3),
+                   "note": "one input/output set reused every step: the working set stays in L2"}
 
     # ---- two stage instances interleaved on two streams (informational) ----
     # Co-located instances fill each other's gaps: the latency-bound decode and NMS kernels of one
@@ -469,15 +516,27 @@ def run_octo(args):
         kern[k]["share"] = kt[k][0] / tot_ms if tot_ms > 0 else None
     dominant = max((k for k in kern if k in alg), key=lambda k: kt[k][0])
     units = {"letterbox": n, "decode": n, "crop": len(items[0])}[dominant]
+    # the per-unit ncu figures were taken on 1080p frames and 224x224 crops: other shapes get none
+    traffic = (traffic_for("decode_planes" if dominant == "decode" and wl.head_layout == "planes" else dominant, units)
+               if name in ("sweep", "anchor_free") else None)
+    dom_ms = kern[dominant]["ms_per_launch"]
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": kern[dominant]["gbs"], "peak": hbm_peak,
         "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})", "unit": "GB/s",
         "frac": kern[dominant]["gbs"] / hbm_peak, "frac_of_nominal_8TBs": kern[dominant]["gbs"] / 8000.0,
-        "alg_bytes_per_launch": alg[dominant], "ms_per_launch": kern[dominant]["ms_per_launch"],
-        # the per-unit ncu figures were taken on 1080p frames and 224x224 crops: other shapes get none
-        "traffic": (traffic_for("decode_planes" if dominant == "decode" and wl.head_layout == "planes" else dominant,
-                                units) if name in ("sweep", "anchor_free") else None),
+        "basis": "algorithmic bytes per launch / CUDA-event time"
+                 + (": fp16 output + the source rectangle of every crop, each rectangle counted once per crop "
+                    "although rectangles of a frame overlap and repeats are served by L2" if dominant == "crop" else ""),
+        "alg_bytes_per_launch": alg[dominant], "ms_per_launch": dom_ms,
+        "traffic": traffic,
+        # the same launch on the bytes that reach DRAM (ncu dram__bytes, scaled by the units processed)
+        "frac_dram": (traffic / (dom_ms * 1e-3) / 1e9 / hbm_peak) if traffic else None,
     }
+    if dominant == "crop":
+        comp = sum(crop_compulsory_bytes(items[b], batch.sizes, *wl.branches[b]) for b in range(len(wl.branches))) \
+            / len(wl.branches)
+        roofline["compulsory_bytes"] = comp  # output + every covered source byte once per frame
+        roofline["frac_compulsory"] = comp / (dom_ms * 1e-3) / 1e9 / hbm_peak
 
     # ---- end to end from pinned host buffers ----
     # The batch is streamed as sub-batches of up to 32 frames over two lanes (stage + stream +
@@ -619,6 +678,8 @@ def run_octo(args):
             "roofline": roofline,
             "kernels": kern,
             "ms_per_step_with_kernel_events": ms_ev_total / args.steps,
+            "step_times": step_stats,
+            "l2_warm": l2_warm,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)
@@ -629,8 +690,9 @@ def run_octo(args):
 
 def run_two_level(args):
     """Two-level cascade (frames -> detector stage -> 256x256 crops -> chained detector stage ->
-    64x32 crops).  One step = level-1 pass, host hand-off of the item table, level-2 pass.  The
-    hand-off synchronises, as it does between two serving containers.  Single GPU."""
+    64x32 crops).  One step = level-1 pass, hand-off of the item table, level-2 passes.  Timed with
+    the hand-off on the device (the reported value) and through the host (stream synchronised and
+    item table read back, as between two serving containers).  Single GPU."""
     import torch
     from dataclasses import replace
 
@@ -676,39 +738,53 @@ def run_two_level(args):
         crops2 = torch.empty((c2n * max_det2, 3, 32, 64), dtype=torch.float16, device=dev)
         off2 = torch.zeros((c2n + 1,), dtype=torch.int32, device=dev)
         ni2 = torch.zeros((2,), dtype=torch.int32, device=dev)
-    items2_total = [0]
 
-    def step(_i):
+    def level1():
         st1.preprocess_array(desc, n, det_in, stream=stream, keepalive=frames)
         st1.postprocess(head1, dets=dets1, counts=counts1, stream=stream)
         st1.crop(0, cap1, out=crops1, offsets=off1, n_items=ni1, stream=stream)
+
+    def level2(lo, hi):
+        st2.postprocess(head2[lo:hi], dets=dets2[: hi - lo], counts=counts2[: hi - lo], stream=stream)
+        st2.crop(0, (hi - lo) * max_det2, out=crops2, offsets=off2[: hi - lo + 1], n_items=ni2, stream=stream)
+
+    def step_host(_i):
+        level1()
         stream.synchronize()  # hand-off: the downstream stage learns its inputs from the host
         m = int(ni1[0])
         items = st1.item_table(0, m)
-        tot = 0
         for lo in range(0, m, c2n):
             hi = min(lo + c2n, m)
             st2.adopt_regions(frames, batch.sizes, items[lo:hi], stream=stream)
-            st2.postprocess(head2[lo:hi], dets=dets2[: hi - lo], counts=counts2[: hi - lo], stream=stream)
-            st2.crop(0, (hi - lo) * max_det2, out=crops2, offsets=off2[: hi - lo + 1], n_items=ni2, stream=stream)
-            tot += hi - lo
-        items2_total[0] = tot
+            level2(lo, hi)
 
-    for i in range(max(args.warmup, 3)):
-        step(i)
-    torch.cuda.synchronize(dev)
+    def step_device(_i):
+        level1()
+        # hand-off on the device: the chained stage reads the upstream item table where it lies;
+        # the level-2 batches are provisioned for the n1 items a pass of this workload yields
+        for lo in range(0, n1, c2n):
+            hi = min(lo + c2n, n1)
+            st2.adopt_items_device(st1, 0, hi - lo, first=lo, stream=stream)
+            level2(lo, hi)
+
+    def measure(step):
+        for i in range(max(args.warmup, 3)):
+            step(i)
+        torch.cuda.synchronize(dev)
+        l0 = st1.launch_count + st2.launch_count
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / args.steps, st1.launch_count + st2.launch_count - l0
+
     sampler = ClockSampler(0)
     sampler.start()
     time.sleep(0.3)
-    l0 = st1.launch_count + st2.launch_count
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
-    torch.cuda.synchronize(dev)
-    ms = e0.elapsed_time(e1) / args.steps
-    launches = st1.launch_count + st2.launch_count - l0
+    ms_host, _ = measure(step_host)
+    ms, launches = measure(step_device)
     clocks = sampler.stop()
     for st in (st1, st2):
         if st.status(stream) & ~0xA:
@@ -719,8 +795,11 @@ def run_two_level(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"two_level B={n}", "level1": "1920x1080 -> 640, crops 256x256",
                    "level1_items": n1, "level2": f"head [{n1}, {a2}, {5 + c2}], crops 64x32",
-                   "level2_items_last_batch": int(ni2[1]), "handoff": "host (item table read back, stream sync)",
+                   "level2_items_last_batch": int(ni2[1]),
+                   "handoff": "device (octo_adopt_items_device: no host synchronisation between the levels)",
                    "l2": f"working set {(sum(f.numel() for f in frames) + head1.numel() * 4 + crops1.numel() * 2) / 2**20:.0f} MiB"},
+        "host_handoff": {"value": n / (ms_host * 1e-3), "unit": UNIT, "ms_per_step": ms_host,
+                         "mode": "item table read back, stream synchronised, octo_adopt_regions"},
         "e2e": None, "gpu_launches": int(launches), "clocks": clocks, "roofline": None, "cpu_baseline": None,
     }
     print(json.dumps(line), flush=True)

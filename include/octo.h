@@ -24,7 +24,10 @@
  *     passed to octo_preprocess_batch are read again by octo_crop_batch (see there).
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).  The three
  *     batch calls only enqueue work on it and return; they never synchronise.
- *   - A stage is not re-entrant: use it from one host thread and one stream at a time.
+ *   - A stage (or queue) object is not re-entrant: use it from one host thread and one stream
+ *     at a time.  Different objects are independent: the library keeps no state outside them
+ *     (apart from the fixed workspace of octo_postprocess_frame_static), so several host
+ *     threads may each drive their own stage, on one GPU or on several.
  *   - Every function returns OCTO_OK (0) or a negative octo_status_t.  No exception
  *     crosses the boundary and nothing aborts the process.  Conditions detected on the
  *     device (non-finite head values, a wait that ran out) set bits in a status word read
@@ -57,7 +60,8 @@ typedef enum {
     OCTO_E_NO_PREPROCESS = -4, /* post/crop called before any octo_preprocess_batch       */
     OCTO_E_CUDA = -5,          /* a CUDA runtime call failed (octo_last_cuda_error)       */
     OCTO_E_DEVICE_TIMEOUT = -6,/* a bounded device-side wait gave up (status word)        */
-    OCTO_E_NO_POSTPROCESS = -7 /* crop called before octo_postprocess_batch of this batch */
+    OCTO_E_NO_POSTPROCESS = -7,/* crop called before octo_postprocess_batch of this batch */
+    OCTO_E_NO_MEMORY = -8      /* host or device memory could not be allocated            */
 } octo_status_t;
 
 /* Bits of the device status word. */
@@ -68,6 +72,8 @@ typedef enum {
                                         /* took the slower global-memory path (informational)  */
 #define OCTO_STATUS_CAND_OVERFLOW 0x10u /* multi-label decode found more candidates in an image */
                                         /* than the workspace holds; the excess was dropped    */
+#define OCTO_STATUS_BOUNDS 0x20u        /* checked build only (-DOCTO_BOUNDS_CHECK): an index    */
+                                        /* left its range; the access was skipped               */
 
 /* Head layouts (octo_stage_config_t.head_layout). */
 #define OCTO_HEAD_ROWS 0   /* [n, A, 5 + C]: rows (cx, cy, w, h, obj, class_0 ..)              */
@@ -192,6 +198,26 @@ typedef struct {
 OCTO_API int octo_adopt_regions(octo_stage_t* st, const octo_region_t* regions, int32_t n, void* cuda_stream);
 
 /*
+ * The same hand-off without the host (Section I: the cascade continues below the first detector;
+ * Section III-B, Observation 1: what a detector emits is what its downstream models receive).
+ * This stage's batch becomes entries [first, first + n) of the item table that the LAST
+ * octo_crop_batch of `branch` on `upstream` built (entry k = slot k of that call's window), read
+ * on the device: one small kernel on `cuda_stream` writes this stage's frame table into its own
+ * workspace, and the following octo_postprocess_batch / octo_crop_batch / octo_queue_push read it
+ * there.  Nothing synchronises and no item travels through host memory, so a chained detector
+ * can be enqueued right behind the upstream pass.  n is the batch size the downstream detector
+ * runs with (the head has n images); if the upstream call packed fewer than first + n items,
+ * the surplus entries are empty: they yield no detections whatever their head holds.
+ * Requirements: both stages on one device; upstream.branch[branch] is net_size x net_size of
+ * this stage; the upstream crop call was enqueued before this call, on the same stream or
+ * ordered with it; the buffer that call wrote {packed, total} to (d_n_items) and the upstream
+ * frames stay valid until this stage's batch is done.  Mapping rule and errors as
+ * octo_adopt_regions, plus OCTO_E_NO_POSTPROCESS (the branch has not been cropped yet).
+ */
+OCTO_API int octo_adopt_items_device(octo_stage_t* st, const octo_stage_t* upstream, int32_t branch, int32_t first,
+                                     int32_t n, void* cuda_stream);
+
+/*
  * Decode the detector head of the batch last given to octo_preprocess_batch (n must match)
  * into detections (stage output Out_m of Table II; the per-frame count is what drives the
  * downstream request rate, Section III-B Observation 1).
@@ -309,6 +335,13 @@ OCTO_API int octo_queue_pop_due(octo_queue_t* q, int32_t bz, int32_t max_wait, v
 /* Synchronise `cuda_stream`, then read (and keep) the device status word. */
 OCTO_API int octo_stage_status(octo_stage_t* st, uint32_t* status_word, void* cuda_stream);
 
+/* Test support for the time-out path: enqueue a one-thread kernel that arms a barrier for bytes
+ * that never arrive (no copy is issued), polls it `polls` times (1 .. 2^20) and then sets
+ * OCTO_STATUS_COPY_TIMEOUT, exactly as the bulk-copy waits of the letterbox and crop kernels do
+ * when they give up.  Afterwards octo_stage_status returns OCTO_E_DEVICE_TIMEOUT until the status
+ * word is cleared; the context stays usable. */
+OCTO_API int octo_stage_selftest_wait(octo_stage_t* st, int32_t polls, void* cuda_stream);
+
 /* Clear the device status word (enqueued on the stream). */
 OCTO_API int octo_stage_clear_status(octo_stage_t* st, void* cuda_stream);
 
@@ -385,6 +418,11 @@ OCTO_API int octo_postprocess_frame_static(int32_t device, const float* d_head, 
                                            float iou_thresh, int32_t max_det, int32_t net_size,
                                            int32_t frame_w, int32_t frame_h, octo_det_t* d_dets,
                                            int32_t* d_count, void* cuda_stream);
+
+/* Synchronise `cuda_stream`, then read the status word of the last octo_postprocess_frame_static
+ * call on `device` (OCTO_STATUS_NONFINITE, OCTO_STATUS_BIG_NMS; every call starts from zero).
+ * Allocates nothing.  (Part of the same addition; no counterpart in the paper.) */
+OCTO_API int octo_static_status(int32_t device, uint32_t* status_word, void* cuda_stream);
 
 /* ---- placement of model instances on GPU inference streams (host only) ---------------------
  * The paper's co-location scheduler (Section III-C "Inference Stream", Algorithm 2): a GPU runs

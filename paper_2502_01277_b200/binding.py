@@ -29,12 +29,14 @@ OCTO_E_NO_PREPROCESS = -4
 OCTO_E_CUDA = -5
 OCTO_E_DEVICE_TIMEOUT = -6
 OCTO_E_NO_POSTPROCESS = -7
+OCTO_E_NO_MEMORY = -8
 
 OCTO_STATUS_NONFINITE = 0x1
 OCTO_STATUS_TRUNCATED = 0x2
 OCTO_STATUS_COPY_TIMEOUT = 0x4
 OCTO_STATUS_BIG_NMS = 0x8
 OCTO_STATUS_CAND_OVERFLOW = 0x10
+OCTO_STATUS_BOUNDS = 0x20
 
 OCTO_HEAD_ROWS = 0
 OCTO_HEAD_PLANES = 1
@@ -48,6 +50,7 @@ EXPORTS = (
     "octo_strerror", "octo_last_cuda_error", "octo_version", "octo_postprocess_frame_static",
     "octo_adopt_regions", "octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop",
     "octo_queue_pop_due", "octo_coral_schedule", "octo_queue_set_options",
+    "octo_adopt_items_device", "octo_stage_selftest_wait", "octo_static_status",
 )
 
 
@@ -152,6 +155,12 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_postprocess_batch.argtypes = [vp, vp, i32, vp, vp, vp]
     lib.octo_adopt_regions.argtypes = [vp, ctypes.POINTER(Region), i32, vp]
     lib.octo_adopt_regions.restype = ctypes.c_int
+    lib.octo_adopt_items_device.argtypes = [vp, vp, i32, i32, i32, vp]
+    lib.octo_adopt_items_device.restype = ctypes.c_int
+    lib.octo_stage_selftest_wait.argtypes = [vp, i32, vp]
+    lib.octo_stage_selftest_wait.restype = ctypes.c_int
+    lib.octo_static_status.argtypes = [i32, ctypes.POINTER(ctypes.c_uint32), vp]
+    lib.octo_static_status.restype = ctypes.c_int
     lib.octo_crop_batch.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.octo_stage_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     lib.octo_stage_clear_status.argtypes = [vp, vp]
@@ -281,6 +290,15 @@ def octo_postprocess_frame_static(device: int, d_head: int, num_anchors: int, nu
         raise OctoError(rc, "octo_postprocess_frame_static")
 
 
+def octo_static_status(device: int = 0, stream: int = 0) -> int:
+    """Status word of the last octo_postprocess_frame_static call on the device (synchronises)."""
+    w = ctypes.c_uint32(0)
+    rc = load_library().octo_static_status(device, ctypes.byref(w), stream)
+    if rc != OCTO_OK:
+        raise OctoError(rc, "octo_static_status")
+    return int(w.value)
+
+
 def octo_stage_status(handle, stream: int = 0) -> int:
     w = ctypes.c_uint32(0)
     rc = load_library().octo_stage_status(handle, ctypes.byref(w), stream)
@@ -378,6 +396,22 @@ class Stage:
         self._frames_keepalive = list(frames)
         self.n = n
 
+    def adopt_items_device(self, upstream: "Stage", branch: int, n: int, first: int = 0, stream=None) -> None:
+        """Chained stage without a host hand-off: this batch = entries [first, first + n) of the item
+        table the upstream stage's last crop call of `branch` built (octo_adopt_items_device)."""
+        rc = load_library().octo_adopt_items_device(self.handle, upstream.handle, branch, first, n,
+                                                    self._stream(stream))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_adopt_items_device")
+        self._frames_keepalive = list(upstream._frames_keepalive)
+        self._upstream_keepalive = upstream
+        self.n = n
+
+    def selftest_wait(self, polls: int = 256, stream=None) -> None:
+        rc = load_library().octo_stage_selftest_wait(self.handle, polls, self._stream(stream))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_stage_selftest_wait")
+
     def postprocess(self, head, dets=None, counts=None, stream=None):
         """head: float32 CUDA tensor [n, A, 5+C].  Returns (dets uint8 [n, max_det, 32], counts int32 [n])."""
         t = self._torch
@@ -440,10 +474,6 @@ class Stage:
     @property
     def launch_count(self) -> int:
         return int(load_library().octo_stage_launch_count(self.handle))
-
-    @property
-    def workspace_bytes(self) -> int:
-        return int(load_library().octo_stage_workspace_bytes(self.handle))
 
     @property
     def workspace_bytes(self) -> int:

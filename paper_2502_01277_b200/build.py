@@ -1,5 +1,12 @@
 """Build the CUDA library (sm_100a) in-tree with nvcc.  No JIT cache, no torch extension:
-the result is a plain C-ABI shared object next to the sources."""
+the result is a plain C-ABI shared object next to the sources.
+
+    python -m paper_2502_01277_b200.build [--force] [--ptxas] [--checked]
+
+--checked builds liboctostage_checked.so with -DOCTO_BOUNDS_CHECK: the same library with every
+computed shared- and global-memory index of the kernels range-checked; a miss sets
+OCTO_STATUS_BOUNDS in the status word and skips the access (no trap).  It stands in for a
+memory checker where none can be run; tests load it with load_library(path)."""
 from __future__ import annotations
 
 import os
@@ -11,6 +18,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "liboctostage.so")
+LIB_CHECKED = os.path.join(HERE, "liboctostage_checked.so")
 OBJ_DIR = os.path.join(HERE, "_build")
 
 NVCC_FLAGS = [
@@ -32,22 +40,24 @@ def _deps():
     return out
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB):
+def is_stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(p) > t for p in _deps())
 
 
-def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) -> str:
-    if not force and not is_stale():
-        return LIB
+def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False, checked: bool = False) -> str:
+    lib = LIB_CHECKED if checked else LIB
+    if not force and not is_stale(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "nvcc")
-    os.makedirs(OBJ_DIR, exist_ok=True)
-    flags = list(NVCC_FLAGS) + (["-Xptxas", "-v"] if ptxas_info else [])
+    obj_dir = OBJ_DIR + ("_checked" if checked else "")
+    os.makedirs(obj_dir, exist_ok=True)
+    flags = list(NVCC_FLAGS) + (["-Xptxas", "-v"] if ptxas_info else []) + (["-DOCTO_BOUNDS_CHECK"] if checked else [])
 
     def compile_one(src: str) -> str:
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         cmd = [nvcc] + flags + ["-c", src, "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if verbose or ptxas_info or r.returncode != 0:
@@ -58,15 +68,16 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
 
     with ThreadPoolExecutor(max_workers=4) as ex:
         objs = list(ex.map(compile_one, sources()))
-    tmp = LIB + f".{os.getpid()}.tmp"
+    tmp = lib + f".{os.getpid()}.tmp"
     cmd = [nvcc, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a", "-cudart", "static"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         sys.stderr.write(r.stdout + r.stderr)
         raise RuntimeError("link failed")
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose=True, ptxas_info="--ptxas" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose=True, ptxas_info="--ptxas" in sys.argv,
+                checked="--checked" in sys.argv))

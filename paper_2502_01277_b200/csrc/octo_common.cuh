@@ -50,6 +50,27 @@ struct StageCounters {
     int sched[2];  // crop kernel: tiles handed out beyond each CTA's first, CTAs finished (both zero between launches)
 };
 
+// Range checks of the checked build (-DOCTO_BOUNDS_CHECK): an index outside its range sets the
+// OCTO_STATUS_BOUNDS bit of the status word and the access is skipped; nothing traps.  In the
+// normal build the condition is not evaluated.  Use as  if (OCTO_IN_RANGE(i < n, status)) a[i] = v;
+#ifdef OCTO_BOUNDS_CHECK
+#define OCTO_IN_RANGE(cond, status_ptr) ((cond) ? true : (atomicOr((status_ptr), 0x20u), false))
+#else
+#define OCTO_IN_RANGE(cond, status_ptr) (true)
+#endif
+
+// Programmatic dependent launch.  Every kernel of the library starts with pdl_enter: it waits
+// until the kernel before it in the stream has completed and its writes are visible (a no-op
+// for a launch without the programmatic attribute); with `early` set it then lets the next
+// kernel of the stream be scheduled right away, where that kernel waits at its own pdl_enter.
+// The hosts sets `early` (and the launch attribute) for small batches only: there the launch
+// latency between the kernels of a pass is most of the pass, while a large grid loses more to
+// the waiting CTAs of its successor than it gains.
+__device__ __forceinline__ void pdl_enter(int early) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 constexpr int kKeyAnchorBits = 25;  // anchor index field of a candidate key
 constexpr unsigned long long kKeySentinel = ~0ull;
 
@@ -164,6 +185,11 @@ __device__ __forceinline__ unsigned long long f32x2(float lo, float hi) {
 __device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
     unsigned long long d;
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long mul_f32x2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
 __device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {

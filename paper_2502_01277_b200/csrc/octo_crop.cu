@@ -12,16 +12,21 @@
 // band) tiles that an atomic counter hands out (whole crops, except that the last crops of a
 // launch are cut into bands so that the grid ends together), so no host synchronisation sits
 // between NMS and cropping.  Inside a CTA one producer warp walks its tiles: it resolves the
-// item, builds the table of horizontal taps (byte offset + exact
-// integer weights per output column) and has the bulk-copy engine stage the 16-byte aligned
-// segments of the source rows a pass taps into one of two shared-memory buffers (mbarrier
-// "full" / "empty" ring, every wait bounded).  The 256 threads of the eight consumer warps
-// walk a pass as a flat, row-major list of pixel pairs, so every lane is busy and
-// neighbouring lanes read neighbouring table entries and row words; the horizontal lerp is
-// an exact integer two-way dot product per channel, the vertical lerp and all scaling are two
-// fp32 operations, and a warp writes up to 128 contiguous bytes per plane straight into the
-// downstream slot.  Measured: large passes matter more than occupancy (2 x 32 KB buffers at
-// 3 CTAs/SM beat 2 x 24 KB at 4, 3 x 22 KB at 3 and 4 x 12 KB at 4).
+// item, builds the table of horizontal taps (byte offset + exact integer weights per output
+// column) and has the bulk-copy engine stage the source rows a pass taps into one of two
+// shared-memory buffers (mbarrier "full" / "empty" ring, every wait bounded).  Every tapped
+// source row is staged ONCE per pass: output rows that share a source row (always when the
+// vertical scale is below 2) point at the same staged copy, so a pass covers as many output
+// rows as its distinct source rows fit the buffer.
+//
+// Consumers own columns.  A consumer thread keeps one pair of neighbouring output columns
+// (its two tap-table entries live in registers) and walks a run of consecutive output rows of
+// the pass.  The horizontal integer lerp of a staged row (an exact two-way dot product per
+// channel) is kept in registers and reused by the next output row whenever that row taps the
+// same source row: per output row only the NEW source rows cost a horizontal pass, i.e. about
+// min(2, vertical scale) instead of 2.  The vertical lerp and all scaling are two packed fp32
+// operations per channel, and a warp writes 128 contiguous bytes per plane and row straight
+// into the downstream slot.
 #include "octo_common.cuh"
 #include <cstring>
 
@@ -29,22 +34,22 @@
 
 namespace octo {
 
-// Shared memory for staged source rows.  A pass stages two row segments per output row; a
-// segment longer than kCropMaxStride - 16 bytes (a rectangle wider than about 5300 pixels)
-// is split into column tiles, so one row pair always fits.  Two buffers form a ring between
-// the producer warp and the consumer warps.
+// Shared memory for staged source rows.  A row segment longer than kCropMaxStride - 16 bytes
+// (a rectangle wider than about 5300 pixels) is split into column tiles, so two rows always
+// fit.  Two buffers form a ring between the producer warp and the consumer warps.
 constexpr int kCropStages = 2;         // ring depth (row buffers)
 constexpr int kCropTables = kCropStages + 1;  // tap tables, one more than ring slots
 constexpr int kCropRowBudget = 32768;  // bytes per ring buffer
 constexpr int kCropMaxStride = kCropRowBudget / 2;
 constexpr int kCropTilePx = 5300;
-constexpr int kCropMaxPassRows = 32;
+constexpr int kCropMaxPassRows = 32;   // one producer lane per output row of a pass
 constexpr int kCropCtasPerSm = 3;
 constexpr int kCropConsumerWarps = 8;
+constexpr int kCropConsumers = 32 * kCropConsumerWarps;
 constexpr int kCropTailBands = 4;     // finer tiles for the last crops of a launch
 constexpr int kCropTilesPerCta = 4;  // measured: 4 > 8 > 16 > 1 for small batches; a tile switch costs about 1 us
 constexpr unsigned kCropProducerSleepNs = 200;  // between the producer's polls of an "empty" barrier
-constexpr int kCropKernelThreads = 32 * (kCropConsumerWarps + 1);  // + one producer warp
+constexpr int kCropKernelThreads = kCropConsumers + 32;  // + one producer warp
 
 // One pass of a CTA: output rows [r0, r0 + nr) x columns [c0, c0 + ncols) of one item.  The
 // producer warp walks the CTA's sequence of passes and publishes each one for the consumers.
@@ -52,8 +57,37 @@ struct __align__(16) CropPass {
     int32_t valid;  // 0: no more passes
     int32_t table;  // which tap table the pass uses
     int32_t slot, r0, nr, c0, ncols;
-    int32_t _pad;
+    uint32_t magic;  // floor(2^32 / pairs) + 1: unit index -> row run by one multiplication
+    int32_t run_rows;  // the pass is cut into runs of this many consecutive rows ...
+    int32_t units;     // ... and (run, column pair) units are dealt to the consumer threads
+    int32_t _pad[2];
 };
+
+// Per output row of a staged pass (RowInfo): row0 = byte offset of the staged copy of the top
+// tap row, relative to the ring buffer and to the tap table's offsets; step = kRowStep bits:
+// distance to the staged bottom tap row (0: the row has a single tap row) | reuse code << 16,
+// or negative for a canvas row (nothing staged).  The reuse code tells a consumer that comes
+// from the previous output row what it already holds:
+//   0 both tap rows, 1 its bottom row is this row's top row, 2 nothing, 3 the top row only.
+constexpr uint32_t kRowStepMask = 0xffffu;
+
+// Horizontal integer lerp of one staged row for a pair of output columns, as exact binary32
+// integers (the 2^23 offset of hsample is taken off again).
+__device__ __forceinline__ void hpair(uint32_t addra, uint32_t sha, uint32_t wtsa, uint32_t addrb, uint32_t shb,
+                                      uint32_t wtsb, unsigned long long& q0, unsigned long long& q1,
+                                      unsigned long long& q2) {
+    float a0, a1, a2, b0, b1, b2;
+    hsample(addra, sha, wtsa, a0, a1, a2);
+    hsample(addrb, shb, wtsb, b0, b1, b2);
+    const unsigned long long m2 = f32x2(-kF32IntValue, -kF32IntValue);
+    q0 = add_f32x2(f32x2(a0, b0), m2);
+    q1 = add_f32x2(f32x2(a1, b1), m2);
+    q2 = add_f32x2(f32x2(a2, b2), m2);
+}
+
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
 
 // QUEUE = false: items come from the stage's current batch through the assembler above.
 // QUEUE = true: items are self-contained records popped from a device queue (qrec[0, *qpacked));
@@ -63,15 +97,21 @@ struct __align__(16) CropPass {
 // offsets inside the slot, canvas columns marked by zero weights in the tap table, canvas rows by a
 // negative row step) and per-plane normalisation (one fused multiply-add per value).  The plain
 // form carries none of that code.
+//
+// The frame table comes either by value in kernel parameter space (`tab`, first-level stages:
+// no table copy on the critical path) or from device memory (`gtab`, chained stages whose
+// table an upstream stage's items define on the device).
 template <int CAP, bool QUEUE, bool GENERAL>
 __global__ void __launch_bounds__(kCropKernelThreads, kCropCtasPerSm)
-crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int first_item, int max_items,
+crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restrict__ gtab, int n, int max_det,
+            int first_item, int max_items,
             const int* __restrict__ bcount, const int* __restrict__ bidx, const octo_det_t* __restrict__ dets,
             int* __restrict__ offsets, int* __restrict__ n_items, octo_item_t* __restrict__ items,
             __half* __restrict__ out, int ow, int oh, int swap_rb, StageCounters* __restrict__ ctr,
             const QRecord* __restrict__ qrec, const int* __restrict__ qpacked, unsigned int* __restrict__ qstatus,
-            int* __restrict__ sched, const CropOpts opts) {
+            int* __restrict__ sched, const CropOpts opts, int pdl) {
     extern __shared__ __align__(128) unsigned char smem[];
+    pdl_enter(pdl);
     __shared__ __align__(8) uint64_t full[kCropStages], empty[kCropStages];
     __shared__ CropPass s_pass[kCropStages];
     __shared__ __align__(16) RowInfo s_row[kCropStages][kCropMaxPassRows];  // per-row data of the staged passes
@@ -154,13 +194,18 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
         int w_pitch = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
         const uint8_t* w_data = nullptr;
         int w_row_lo = 0, w_row_hi = 0, w_tile_cols = ow;
-        int w_c0 = 0, w_ncols = 0, w_r0 = 0, w_nr = 0;
-        int w_seg_lo = 0, w_seg = 0, w_stride = 16, w_pass_rows = 1;
+        int w_c0 = 0, w_ncols = 0, w_r0 = 0;
+        int w_seg_lo = 0, w_seg = 0, w_stride = 16, w_cap_slots = 2;
+        int w_runs = 1;           // row runs that fit the consumer threads side by side
+        uint32_t w_run_magic = 0, w_pair_magic = 0;  // divisions by w_runs / by the pair count, as multiplications
         bool w_valid = false, w_new = false;
         // size and offset of the resized rectangle inside the slot: the whole slot unless the
         // branch keeps the aspect ratio
         int w_nw = ow, w_nh = oh, w_pl = 0, w_pt = 0;
         float w_inv_dx = inv_dx, w_inv_dy = inv_dy, w_inv_all = inv_all;
+#ifdef OCTO_BOUNDS_CHECK
+        int w_fh = 0;  // frame height, for the range check of the staged rows
+#endif
 
         // geometry of the column tile starting at w_c0
         auto set_tile = [&]() {
@@ -181,7 +226,14 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             w_seg_lo = lo;
             w_seg = hi - lo;
             w_stride = w_seg + 16;
-            w_pass_rows = max(1, min(min(kCropRowBudget / (2 * w_stride), kCropMaxPassRows), w_band_rows));
+            w_cap_slots = kCropRowBudget / w_stride;  // >= 2
+            // Work units of a pass: (run of consecutive rows, column pair).  A pass is cut into as
+            // many runs as fit the consumer threads side by side (224 columns: 2 runs x 112
+            // pairs), so that a warp works on one run and its reuse decisions are uniform.
+            const uint32_t pairs = (uint32_t)max(w_ncols >> 1, 1);
+            w_runs = max(1, min(kCropConsumers / (int)pairs, kCropMaxPassRows));
+            w_run_magic = w_runs > 1 ? 0xffffffffu / (uint32_t)w_runs + 1u : 0u;
+            w_pair_magic = pairs > 1u ? 0xffffffffu / pairs + 1u : 0u;
         };
         // first pass of the next tile, if there is one; every lane resolves the same item
         auto open_tile = [&]() {
@@ -209,6 +261,9 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 const QRecord rec = qrec[w_slot];
                 w_data = rec.data; w_pitch = rec.pitch;
                 rx0 = rec.rx0; ry0 = rec.ry0; rx1 = rec.rx1; ry1 = rec.ry1;
+#ifdef OCTO_BOUNDS_CHECK
+                w_fh = rec.h;
+#endif
             } else {
                 const int item = first_item + w_slot;
                 int lo = 0, hi = n;  // largest f with s_off[f] <= item (frames without items are skipped)
@@ -217,9 +272,12 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                     if (s_off[mid] <= item) lo = mid; else hi = mid;
                 }
                 const int f = lo;
-                const int det = bidx[(size_t)f * max_det + (item - s_off[f])];
+                int det = 0;
+                if (OCTO_IN_RANGE(item - s_off[f] >= 0 && item - s_off[f] < max_det, status))
+                    det = bidx[(size_t)f * max_det + (item - s_off[f])];
+                if (!OCTO_IN_RANGE(det >= 0 && det < max_det, status)) det = 0;
                 const octo_det_t d = dets[(size_t)f * max_det + det];
-                const FrameDesc& fd = tab.f[f];
+                const FrameDesc fd = gtab ? gtab[f] : tab.f[f];
                 // outward-rounded rectangle, clamped so that it is never empty
                 rx0 = (int)floorf(d.x1); ry0 = (int)floorf(d.y1);
                 rx1 = (int)ceilf(d.x2); ry1 = (int)ceilf(d.y2);
@@ -227,7 +285,8 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                 ry0 = min(max(ry0, 0), fd.h - 1);
                 rx1 = min(max(rx1, rx0 + 1), fd.w);
                 ry1 = min(max(ry1, ry0 + 1), fd.h);
-                if (w_band == 0 && lane == 0) {  // the tile of a slot's first band records the item
+                if (w_band == 0 && lane == 0 && OCTO_IN_RANGE(w_slot >= 0 && w_slot < max_items, status)) {
+                    // the tile of a slot's first band records the item
                     octo_item_t it;
                     it.frame = f; it.det = det;
                     it.rx0 = rx0; it.ry0 = ry0; it.rx1 = rx1; it.ry1 = ry1;
@@ -235,6 +294,9 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                     items[w_slot] = it;
                 }
                 w_data = fd.data; w_pitch = fd.pitch;
+#ifdef OCTO_BOUNDS_CHECK
+                w_fh = fd.h;
+#endif
             }
             w_rx0 = rx0; w_ry0 = ry0; w_cw = rx1 - rx0; w_ch = ry1 - ry0;
             if (GENERAL && opts.keep_aspect) {
@@ -261,22 +323,20 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             w_row_lo = w_band * w_band_rows;
             w_row_hi = min(w_row_lo + w_band_rows, oh);
             w_r0 = w_row_lo;
-            w_nr = min(w_pass_rows, w_row_hi - w_r0);
             w_new = true;
         };
-        auto advance = [&]() {
+        // the pass that was just published covered nr rows
+        auto advance = [&](int nr) {
             w_new = false;
-            if (w_r0 + w_nr < w_row_hi) {
-                w_r0 += w_nr;
+            if (w_r0 + nr < w_row_hi) {
+                w_r0 += nr;
             } else if (w_c0 + w_ncols < ow) {
                 w_c0 += w_ncols;
                 set_tile();
                 w_r0 = w_row_lo;
             } else {
                 open_tile();
-                return;
             }
-            w_nr = min(w_pass_rows, w_row_hi - w_r0);
         };
 
         open_tile();
@@ -305,33 +365,59 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
                     }
                 }
             }
-            CropPass p;
-            p.valid = w_valid ? 1 : 0;
-            p.table = tb;
-            p.slot = w_slot; p.r0 = w_r0; p.nr = w_nr; p.c0 = w_c0; p.ncols = w_ncols;
-            p._pad = 0;
-            // lane r owns output row w_r0 + r of the pass
-            int ry = 0;
-            uint32_t bytes = 0;
+            // lane r stands for output row w_r0 + r; the pass takes the first nr of them
+            const bool cand = w_valid && (w_r0 + lane < w_row_hi);
+            const int iy = w_r0 + lane - w_pt;  // row inside the resized rectangle
+            const bool has_row = cand && (!GENERAL || (iy >= 0 && iy < w_nh));
+            int y0 = 0, ry = 0;
+            if (has_row) src_coord(iy, w_ch, w_nh, w_inv_dy, y0, ry);
+            const int need2 = ry != 0 ? 1 : 0;
+            // Which of this row's tap rows (y0, and y0 + 1 if need2) did the row before it not
+            // tap already?  Source rows never decrease from one output row to the next, so the
+            // row before is the only one that can share them.
+            const int maxrow = y0 + need2;
+            int p_has = __shfl_up_sync(0xffffffffu, has_row ? 1 : 0, 1);
+            const int p_max = __shfl_up_sync(0xffffffffu, maxrow, 1);
+            const int p_need2 = __shfl_up_sync(0xffffffffu, need2, 1);
+            if (lane == 0) p_has = 0;
+            int newrows = 0, back = 0;
+            uint32_t code = 2u;
+            if (has_row) {
+                if (!p_has || y0 > p_max) { newrows = 1 + need2; }
+                else if (y0 == p_max) { newrows = need2; back = 1; code = p_need2 ? 1u : (need2 ? 3u : 0u); }
+                else { back = 2; code = 0u; }  // y0 == p_max - 1: both rows are staged
+            }
+            int incl = newrows;  // inclusive scan: staged rows up to and including this output row
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += t;
+            }
+            const int nr = __popc(__ballot_sync(0xffffffffu, cand && incl <= w_cap_slots));  // >= 1 when valid
+            const bool in_pass = lane < nr;
+            const int slot_top = incl - newrows - back;
             RowInfo ri;
             ri.row0 = 0; ri.step = 0; ri.wx = 0.0f; ri.wy = 0.0f;
-            const uint8_t* src = nullptr;
-            const bool in_pass = w_valid && lane < w_nr;
-            const int iy = w_r0 + lane - w_pt;  // row inside the resized rectangle
-            const bool has_row = in_pass && (!GENERAL || (iy >= 0 && iy < w_nh));
-            if (has_row) {
-                int y0;
-                src_coord(iy, w_ch, w_nh, w_inv_dy, y0, ry);
-                bytes = (uint32_t)w_seg * (ry != 0 ? 2u : 1u);
-                ri.row0 = 2 * lane * w_stride - w_seg_lo;  // table offsets are relative to the frame row
-                ri.step = w_stride;
+            uint32_t bytes = 0;
+            if (in_pass && has_row) {
+                bytes = (uint32_t)(newrows * w_seg);
+                ri.row0 = slot_top * w_stride - w_seg_lo;  // table offsets are relative to the frame row
+                ri.step = (int32_t)((need2 ? (uint32_t)w_stride : 0u) | (code << 16));
                 ri.wx = (float)(2 * w_nh - ry) * w_inv_all;
                 ri.wy = (float)ry * w_inv_all;
-                src = w_data + (size_t)(w_ry0 + y0) * (size_t)w_pitch + w_seg_lo;
             } else if (GENERAL) {
                 ri.step = -1;  // canvas row: nothing is staged for it
             }
-            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+            const uint32_t total_tx = __reduce_add_sync(0xffffffffu, bytes);
+            CropPass p;
+            p.valid = w_valid ? 1 : 0;
+            p.table = tb;
+            p.slot = w_slot; p.r0 = w_r0; p.nr = nr; p.c0 = w_c0; p.ncols = w_ncols;
+            p.magic = w_pair_magic;
+            // rows per run = ceil(nr / runs); runs that start past the last row stay empty
+            p.run_rows = w_runs > 1 ? (int)__umulhi((uint32_t)(nr + w_runs - 1), w_run_magic) : nr;
+            p.units = (w_ncols >> 1) * w_runs;
+            p._pad[0] = 0; p._pad[1] = 0;
             // ---- ring slot b: wait until the consumers have finished the pass that used it ----
             if (k >= kCropStages) {
                 const uint32_t par = (ephase >> b) & 1u;
@@ -350,14 +436,31 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             if (in_pass) s_row[b][lane] = ri;
             fence_proxy_async();
             __syncwarp();  // table, pass record and row data are written before the barrier is armed
-            if (lane == 0) mbar_expect_tx(&full[b], total);
+            if (lane == 0) mbar_expect_tx(&full[b], total_tx);
             __syncwarp();
-            if (has_row) {
-                unsigned char* dst = s_rows0 + (size_t)b * kCropRowBudget + (size_t)(2 * lane) * w_stride;
-                bulk_g2s(dst, src, (uint32_t)w_seg, &full[b]);
-                if (ry != 0) bulk_g2s(dst + w_stride, src + w_pitch, (uint32_t)w_seg, &full[b]);
+            if (in_pass && newrows > 0) {
+                // the new rows are the last `newrows` of {y0, y0 + 1}
+                const int first_new = need2 + 1 - newrows;  // 0: y0 is new, 1: only y0 + 1
+                const int slot_new = slot_top + first_new;
+                const uint8_t* src = w_data + (size_t)(w_ry0 + y0 + first_new) * (size_t)w_pitch + w_seg_lo;
+                unsigned char* dst = s_rows0 + (size_t)b * kCropRowBudget + (size_t)slot_new * w_stride;
+                bool ok = true;
+#ifdef OCTO_BOUNDS_CHECK
+                ok = OCTO_IN_RANGE(slot_new >= 0 && slot_new + newrows <= w_cap_slots &&
+                                   (slot_new + newrows) * w_stride <= kCropRowBudget &&
+                                   w_ry0 + y0 + first_new + newrows <= w_fh && w_seg_lo >= 0 &&
+                                   w_seg_lo + w_seg <= w_pitch && (w_seg & 15) == 0, status);
+                if (!ok) {  // keep the barrier's byte count right without touching memory
+                    asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full[b])),
+                                 "r"((uint32_t)(newrows * w_seg)) : "memory");
+                }
+#endif
+                if (ok) {
+                    bulk_g2s(dst, src, (uint32_t)w_seg, &full[b]);
+                    if (newrows == 2) bulk_g2s(dst + w_stride, src + w_pitch, (uint32_t)w_seg, &full[b]);
+                }
             }
-            advance();
+            advance(nr);
         }
     } else {
         // =============================== consumer warps ==================================
@@ -375,7 +478,6 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             fphase ^= 1u << b;
             const CropPass cur = s_pass[b];
             if (!cur.valid) break;
-            // flat list of pixel pairs (row-major); thread t of the consumers owns pairs t, t+256, ...
             const uint32_t xt = smem_u32(s_xtab0) + (uint32_t)(cur.table * ow + cur.c0) * (uint32_t)sizeof(XEntry);
             const uint32_t rows = smem_u32(s_rows0) + (uint32_t)b * kCropRowBudget;
             const uint32_t rinfo = smem_u32(&s_row[b][0]);
@@ -383,54 +485,70 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
             __half* const t0 = out0 + tile_off;
             __half* const t1 = out1 + tile_off;
             __half* const t2 = out2 + tile_off;
+            // work units (run of rows, column pair), laid out by the producer
             const int pairs = cur.ncols >> 1;
-            const int npairs = cur.nr * pairs;
-            // (row, pair) of this thread's first element, then advanced by the stride in place
-            constexpr int kStride = 32 * kCropConsumerWarps;
-            const int dr = kStride / pairs, dp = kStride - dr * pairs;
-            int r = (int)threadIdx.x / pairs, pair = (int)threadIdx.x - r * pairs;
-            for (int idx = threadIdx.x; idx < npairs; idx += kStride) {
-                const uint4 rw = lds128(rinfo + 16u * (uint32_t)r);
-                const uint4 ee = lds128(xt + 16u * (uint32_t)pair);
-                const float wx = __uint_as_float(rw.z), wy = __uint_as_float(rw.w);
-                const float nwx = -kF32IntValue * wx;
-                if (!GENERAL) {
-                    unsigned long long p0, p1, p2;
-                    if (wy != 0.0f) sample_pair<true>(rows + rw.x, rw.y, ee.x, ee.y, ee.z, ee.w, wx, nwx, wy, p0, p1, p2);
-                    else sample_pair<false>(rows + rw.x, rw.y, ee.x, ee.y, ee.z, ee.w, wx, nwx, wy, p0, p1, p2);
-                    const uint32_t o = (uint32_t)(r * ow + 2 * pair);
-                    *reinterpret_cast<uint32_t*>(t0 + o) = half2_of_f32x2(p0);
-                    *reinterpret_cast<uint32_t*>(t1 + o) = half2_of_f32x2(p1);
-                    *reinterpret_cast<uint32_t*>(t2 + o) = half2_of_f32x2(p2);
-                } else {
-                    float a0, a1, a2, b0, b1, b2;
+            for (int u = threadIdx.x; u < cur.units; u += kCropConsumers) {
+                const int run = pairs > 1 ? (int)__umulhi((uint32_t)u, cur.magic) : u;
+                const int pair = u - run * pairs;
+                const int ra = run * cur.run_rows, rb = min(ra + cur.run_rows, cur.nr);
+                const uint4 ee = lds128(xt + 16u * (uint32_t)pair);  // two XEntry: {off, wts} x 2
+                const uint32_t basea = rows + (ee.x & ~3u), sha = ee.x << 3;
+                const uint32_t baseb = rows + (ee.z & ~3u), shb = ee.z << 3;
+                // horizontal lerps of the current top (T) and bottom (B) tap rows, three channels x two pixels
+                unsigned long long T0 = 0ull, T1 = 0ull, T2 = 0ull, B0 = 0ull, B1 = 0ull, B2 = 0ull;
+                uint32_t o = (uint32_t)(ra * ow + 2 * pair);
+                for (int r = ra; r < rb; ++r, o += (uint32_t)ow) {
+                    const uint4 rw = lds128(rinfo + 16u * (uint32_t)r);
                     if (GENERAL && (int)rw.y < 0) {  // canvas row
-                        a0 = b0 = opts.fill[0]; a1 = b1 = opts.fill[1]; a2 = b2 = opts.fill[2];
-                    } else {
-                        if (wy != 0.0f) {
-                            sample_px<true>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
-                            sample_px<true>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
-                        } else {
-                            sample_px<false>(rows + rw.x, rw.y, ee.x, ee.y, wx, nwx, wy, a0, a1, a2);
-                            sample_px<false>(rows + rw.x, rw.y, ee.z, ee.w, wx, nwx, wy, b0, b1, b2);
-                        }
-                        if (GENERAL) {
-                            a0 = ee.y ? fmaf(a0, opts.sc[0], opts.of[0]) : opts.fill[0];
-                            a1 = ee.y ? fmaf(a1, opts.sc[1], opts.of[1]) : opts.fill[1];
-                            a2 = ee.y ? fmaf(a2, opts.sc[2], opts.of[2]) : opts.fill[2];
-                            b0 = ee.w ? fmaf(b0, opts.sc[0], opts.of[0]) : opts.fill[0];
-                            b1 = ee.w ? fmaf(b1, opts.sc[1], opts.of[1]) : opts.fill[1];
-                            b2 = ee.w ? fmaf(b2, opts.sc[2], opts.of[2]) : opts.fill[2];
-                        }
+                        *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(opts.fill[0], opts.fill[0]);
+                        *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(opts.fill[1], opts.fill[1]);
+                        *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(opts.fill[2], opts.fill[2]);
+                        continue;
                     }
-                    const uint32_t o = (uint32_t)(r * ow + 2 * pair);
-                    *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(a0, b0);
-                    *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(a1, b1);
-                    *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(a2, b2);
+                    const uint32_t code = r == ra ? 2u : (rw.y >> 16) & 3u;
+                    const uint32_t step = rw.y & kRowStepMask;
+#ifdef OCTO_BOUNDS_CHECK
+                    {
+                        // every tap reads 12 bytes from its aligned word: both rows must lie in the buffer
+                        const long long lo = (long long)(int)rw.x + (long long)min(ee.x & ~3u, ee.z & ~3u);
+                        const long long hi = (long long)(int)rw.x + (long long)max(ee.x & ~3u, ee.z & ~3u) + step + 12;
+                        if (!OCTO_IN_RANGE(lo >= 0 && hi <= kCropRowBudget && r < kCropMaxPassRows &&
+                                           cur.slot >= 0 && cur.slot < max_items && cur.r0 + r < oh &&
+                                           cur.c0 + 2 * pair + 1 < ow, status))
+                            continue;
+                    }
+#endif
+                    if (code == 2u) hpair(basea + rw.x, sha, ee.y, baseb + rw.x, shb, ee.w, T0, T1, T2);
+                    else if (code == 1u) { T0 = B0; T1 = B1; T2 = B2; }
+                    if (code != 0u && step != 0u)
+                        hpair(basea + rw.x + step, sha, ee.y, baseb + rw.x + step, shb, ee.w, B0, B1, B2);
+                    const float wx = __uint_as_float(rw.z), wy = __uint_as_float(rw.w);
+                    const unsigned long long wx2 = f32x2(wx, wx), wy2 = f32x2(wy, wy);
+                    // fl(fl(v0 * wx) + v1 * wy) per element (B is finite and wy = 0 when the row has one tap row)
+                    const unsigned long long p0 = fma_f32x2(B0, wy2, mul_f32x2(T0, wx2));
+                    const unsigned long long p1 = fma_f32x2(B1, wy2, mul_f32x2(T1, wx2));
+                    const unsigned long long p2 = fma_f32x2(B2, wy2, mul_f32x2(T2, wx2));
+                    if (!GENERAL) {
+                        *reinterpret_cast<uint32_t*>(t0 + o) = half2_of_f32x2(p0);
+                        *reinterpret_cast<uint32_t*>(t1 + o) = half2_of_f32x2(p1);
+                        *reinterpret_cast<uint32_t*>(t2 + o) = half2_of_f32x2(p2);
+                    } else {
+                        float a0, a1, a2, b0, b1, b2;
+                        unpack_f32x2(p0, a0, b0);
+                        unpack_f32x2(p1, a1, b1);
+                        unpack_f32x2(p2, a2, b2);
+                        // zero weights mark a canvas column
+                        a0 = ee.y ? fmaf(a0, opts.sc[0], opts.of[0]) : opts.fill[0];
+                        a1 = ee.y ? fmaf(a1, opts.sc[1], opts.of[1]) : opts.fill[1];
+                        a2 = ee.y ? fmaf(a2, opts.sc[2], opts.of[2]) : opts.fill[2];
+                        b0 = ee.w ? fmaf(b0, opts.sc[0], opts.of[0]) : opts.fill[0];
+                        b1 = ee.w ? fmaf(b1, opts.sc[1], opts.of[1]) : opts.fill[1];
+                        b2 = ee.w ? fmaf(b2, opts.sc[2], opts.of[2]) : opts.fill[2];
+                        *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(a0, b0);
+                        *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(a1, b1);
+                        *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(a2, b2);
+                    }
                 }
-                r += dr;
-                pair += dp;
-                if (pair >= pairs) { pair -= pairs; ++r; }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[b]);  // this warp is done with ring slot b
@@ -448,38 +566,42 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, int
     }
 }
 
-template <int CAP>
-static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
-    static FrameTable<CAP> tab;
-    for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
+static size_t crop_smem_bytes(int out_w) {
+    return (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)out_w;
+}
+
+static int crop_grid(int sm_count, int slots, int out_h) {
     // The kernel cuts crops into row bands itself once it knows how many items there are; the
     // grid only has to be large enough for the finest cut.
-    const long long cap = (long long)a.sm_count * kCropCtasPerSm;
-    const long long work = (long long)a.max_items * ((a.out_h + 7) / 8);
-    int grid = (int)(work < cap ? work : cap);
-    if (grid < 1) grid = 1;  // a zero-slot window still gets its offsets and totals
-    const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)a.out_w;
-    if (a.general)
-        crop_kernel<CAP, false, true><<<grid, kCropKernelThreads, smem, stream>>>(
-            tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
-            a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, a.swap_rb, a.d_ctr, nullptr, nullptr,
-            nullptr, a.d_ctr->sched, a.opts);
-    else
-        crop_kernel<CAP, false, false><<<grid, kCropKernelThreads, smem, stream>>>(
-            tab, a.n, a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
-            a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, a.swap_rb, a.d_ctr, nullptr, nullptr,
-            nullptr, a.d_ctr->sched, a.opts);
-    return cudaGetLastError();
+    const long long cap = (long long)sm_count * kCropCtasPerSm;
+    const long long work = (long long)slots * ((out_h + 7) / 8);
+    const int grid = (int)(work < cap ? work : cap);
+    return grid < 1 ? 1 : grid;  // a zero-slot window still gets its offsets and totals
+}
+
+template <int CAP>
+static cudaError_t launch_crop_cap(const CropArgs& a, cudaStream_t stream) {
+    FrameTable<CAP> tab;  // built per call (copied into kernel parameter space by the launch)
+    if (!a.d_tab)
+        for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
+    const int grid = crop_grid(a.sm_count, a.max_items, a.out_h);
+    const size_t smem = crop_smem_bytes(a.out_w);
+    auto kernel = a.general ? crop_kernel<CAP, false, true> : crop_kernel<CAP, false, false>;
+    return launch_kernel(kernel, dim3(grid), dim3(kCropKernelThreads), smem, stream, a.pdl, tab, a.d_tab, a.n,
+                         a.max_det, a.first_item, a.max_items, a.d_bcount, a.d_bidx, a.d_dets, a.d_offsets, a.d_n_items,
+                         a.d_items, reinterpret_cast<__half*>(a.d_out), a.out_w, a.out_h, a.swap_rb, a.d_ctr,
+                         (const QRecord*)nullptr, (const int*)nullptr, (unsigned int*)nullptr, a.d_ctr->sched, a.opts,
+                         a.pdl ? 1 : 0);
 }
 
 cudaError_t prepare_crop() {
-    const int smem = kCropStages * kCropRowBudget + kCropTables * (int)sizeof(XEntry) * 2048;
+    const int smem = (int)crop_smem_bytes(2048);
     cudaError_t e;
     const void* kernels[] = {
         (const void*)crop_kernel<8, false, false>,   (const void*)crop_kernel<8, false, true>,
         (const void*)crop_kernel<64, false, false>,  (const void*)crop_kernel<64, false, true>,
         (const void*)crop_kernel<512, false, false>, (const void*)crop_kernel<512, false, true>,
-        (const void*)crop_kernel<8, true, false>,    (const void*)crop_kernel<8, true, true>,
+        (const void*)crop_kernel<1, true, false>,    (const void*)crop_kernel<1, true, true>,
     };
     for (const void* k : kernels) {
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -488,7 +610,9 @@ cudaError_t prepare_crop() {
     return cudaSuccess;
 }
 
-// Assembler + crop-resize of one branch window (a.max_items may be 0).
+// Assembler + crop-resize of one branch window (a.max_items may be 0).  The capacity also sizes
+// the shared-memory scan of the per-frame counts, so it follows n even when the frame table is
+// read from device memory.
 cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream) {
     if (a.n <= 8) return launch_crop_cap<8>(a, stream);
     if (a.n <= 64) return launch_crop_cap<64>(a, stream);
@@ -499,22 +623,19 @@ cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream) {
 cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int bz, void* d_out, int out_w,
                               int out_h, int swap_rb, int sm_count, unsigned int* d_status, int* d_sched,
                               const CropOpts* general, cudaStream_t stream) {
-    static FrameTable<8> tab;  // unused in queue mode
-    const long long cap = (long long)sm_count * kCropCtasPerSm;
-    const long long work = (long long)bz * ((out_h + 7) / 8);
-    const int grid = (int)(work < cap ? work : cap);
-    const size_t smem = (size_t)kCropStages * kCropRowBudget + (size_t)kCropTables * sizeof(XEntry) * (size_t)out_w;
+    FrameTable<1> tab;  // unused in queue mode
+    memset(&tab, 0, sizeof(tab));
+    const int grid = crop_grid(sm_count, bz, out_h);
+    const size_t smem = crop_smem_bytes(out_w);
     CropOpts opts;
     memset(&opts, 0, sizeof(opts));
-    if (general)
-        crop_kernel<8, true, true><<<grid, kCropKernelThreads, smem, stream>>>(
-            tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
-            out_w, out_h, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched, *general);
-    else
-        crop_kernel<8, true, false><<<grid, kCropKernelThreads, smem, stream>>>(
-            tab, 0, 0, 0, bz, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, reinterpret_cast<__half*>(d_out),
-            out_w, out_h, swap_rb, nullptr, d_staged, d_qpacked, d_status, d_sched, opts);
-    return cudaGetLastError();
+    if (general) opts = *general;
+    auto kernel = general ? crop_kernel<1, true, true> : crop_kernel<1, true, false>;
+    return launch_kernel(kernel, dim3(grid), dim3(kCropKernelThreads), smem, stream, false, tab,
+                         (const FrameDesc*)nullptr, 0, 0, 0, bz, (const int*)nullptr, (const int*)nullptr,
+                         (const octo_det_t*)nullptr, (int*)nullptr, (int*)nullptr, (octo_item_t*)nullptr,
+                         reinterpret_cast<__half*>(d_out), out_w, out_h, swap_rb, (StageCounters*)nullptr, d_staged,
+                         d_qpacked, d_status, d_sched, opts, 0);
 }
 
 }  // namespace octo

@@ -46,7 +46,8 @@ template <int kDecPerThread>
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf, int key_stride,
               unsigned long long* __restrict__ keys, int* __restrict__ cand_count,
-              unsigned int* __restrict__ status) {
+              unsigned int* __restrict__ status, int pdl) {
+    pdl_enter(pdl);
     // mode bit 0: obj / class values are logits; bit 1: class-agnostic NMS (key class field 0);
     // bit 2: multi-label candidates
     const int logits = mode & 1;
@@ -171,7 +172,8 @@ template <int VEC>
 __global__ void __launch_bounds__(kDecThreads)
 decode_planes_kernel(const float* __restrict__ head, int A, int C, int mode, float conf, float pre, int key_stride,
                      unsigned long long* __restrict__ keys, int* __restrict__ cand_count,
-                     unsigned int* __restrict__ status) {
+                     unsigned int* __restrict__ status, int pdl) {
+    pdl_enter(pdl);
     constexpr int kCtaAnchors = kPlaneAnchorWarps * 32 * VEC;
     __shared__ float s_best[kPlaneClassWarps][kCtaAnchors];
     __shared__ int s_k[kPlaneClassWarps][kCtaAnchors];
@@ -274,6 +276,7 @@ decode_planes_kernel(const float* __restrict__ head, int A, int C, int mode, flo
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
     // d_cand_count is zero on entry: zeroed at stage creation and re-zeroed by the NMS kernel.
     const int mode = (a.logits ? 1 : 0) | (a.class_agnostic ? 2 : 0) | (a.multi_label ? 4 : 0);
+    const int pdl = a.pdl ? 1 : 0;
     if (a.layout == OCTO_HEAD_PLANES) {
         // Multi-label prefilter in the head's own units: for probabilities the threshold itself;
         // for logits the threshold's logit lowered by a margin that dwarfs the few-ulp error of
@@ -288,26 +291,23 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
         }
         if ((a.A & 3) == 0 && (reinterpret_cast<uintptr_t>(a.d_head) & 15) == 0) {
             dim3 grid((a.A + 128 * kPlaneAnchorWarps - 1) / (128 * kPlaneAnchorWarps), a.n);
-            decode_planes_kernel<4><<<grid, kDecThreads, 0, stream>>>(a.d_head, a.A, a.C, mode, a.conf, pre,
-                                                                     a.key_stride, a.d_keys, a.d_cand_count, a.d_status);
+            return launch_kernel(decode_planes_kernel<4>, grid, dim3(kDecThreads), 0, stream, a.pdl, a.d_head, a.A, a.C,
+                                 mode, a.conf, pre, a.key_stride, a.d_keys, a.d_cand_count, a.d_status, pdl);
         } else {
             dim3 grid((a.A + 32 * kPlaneAnchorWarps - 1) / (32 * kPlaneAnchorWarps), a.n);
-            decode_planes_kernel<1><<<grid, kDecThreads, 0, stream>>>(a.d_head, a.A, a.C, mode, a.conf, pre,
-                                                                     a.key_stride, a.d_keys, a.d_cand_count, a.d_status);
+            return launch_kernel(decode_planes_kernel<1>, grid, dim3(kDecThreads), 0, stream, a.pdl, a.d_head, a.A, a.C,
+                                 mode, a.conf, pre, a.key_stride, a.d_keys, a.d_cand_count, a.d_status, pdl);
         }
-        return cudaGetLastError();
     }
     const int per_cta4 = kDecThreads * 4;
     if ((long long)a.n * ((a.A + per_cta4 - 1) / per_cta4) >= 296) {
         dim3 grid((a.A + per_cta4 - 1) / per_cta4, a.n);
-        decode_kernel<4><<<grid, kDecThreads, 0, stream>>>(a.d_head, a.A, a.C, mode, a.conf, a.key_stride, a.d_keys,
-                                                          a.d_cand_count, a.d_status);
-    } else {
-        dim3 grid((a.A + kDecThreads - 1) / kDecThreads, a.n);
-        decode_kernel<1><<<grid, kDecThreads, 0, stream>>>(a.d_head, a.A, a.C, mode, a.conf, a.key_stride, a.d_keys,
-                                                          a.d_cand_count, a.d_status);
+        return launch_kernel(decode_kernel<4>, grid, dim3(kDecThreads), 0, stream, a.pdl, a.d_head, a.A, a.C, mode,
+                             a.conf, a.key_stride, a.d_keys, a.d_cand_count, a.d_status, pdl);
     }
-    return cudaGetLastError();
+    dim3 grid((a.A + kDecThreads - 1) / kDecThreads, a.n);
+    return launch_kernel(decode_kernel<1>, grid, dim3(kDecThreads), 0, stream, a.pdl, a.d_head, a.A, a.C, mode, a.conf,
+                         a.key_stride, a.d_keys, a.d_cand_count, a.d_status, pdl);
 }
 
 }  // namespace octo

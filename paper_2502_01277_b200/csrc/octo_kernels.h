@@ -25,10 +25,13 @@ struct DecodeArgs {
     unsigned long long* d_keys;
     int* d_cand_count;
     unsigned int* d_status;
+    bool pdl;  // launch with programmatic stream serialisation (small batches)
 };
 
 struct NmsArgs {
     const FrameDesc* frames;  // host
+    const FrameDesc* d_tab;   // device-resident frame table of a chained stage, or null
+    bool pdl;                 // launch with programmatic stream serialisation (small batches)
     int n;
     const float* d_head;
     int A, C;
@@ -58,6 +61,8 @@ struct CropOpts {
 
 struct CropArgs {
     const FrameDesc* frames;  // host
+    const FrameDesc* d_tab;   // device-resident frame table of a chained stage, or null
+    bool pdl;                 // launch with programmatic stream serialisation (small batches)
     int n;
     int max_det, first_item, max_items;
     const int* d_bcount;  // this branch's [max_batch]
@@ -77,13 +82,16 @@ struct CropArgs {
 void fill_crop_opts(const octo_branch_cfg_t& br, int swap_rb, int pad_value, CropOpts* out);
 int validate_branch_options(const octo_branch_cfg_t& br);  // OCTO_OK or OCTO_E_INVALID_ARG
 
+// Records the text that octo_last_cuda_error returns on this thread; returns OCTO_E_CUDA.
+int report_cuda_error(cudaError_t e, const char* what);
+
 // Opt the kernels of every table capacity into the shared memory they need (current device).
 cudaError_t prepare_letterbox();
 cudaError_t prepare_nms();
 cudaError_t prepare_crop();
 
 cudaError_t launch_letterbox(const FrameDesc* frames, int n, void* d_out, int S, int max_w, int pad_value,
-                             int swap_rb, unsigned int* d_status, cudaStream_t stream);
+                             int swap_rb, unsigned int* d_status, bool pdl, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
 cudaError_t launch_nms(const NmsArgs& a, cudaStream_t stream);
 cudaError_t launch_crop(const CropArgs& a, cudaStream_t stream);  // batch assembler + crop-resize
@@ -92,5 +100,27 @@ cudaError_t launch_crop_queue(const QRecord* d_staged, const int* d_qpacked, int
                               const CropOpts* general, cudaStream_t stream);
 
 constexpr int kLetterboxMaxWidth = 8192;  // widest frame the row staging supports
+
+// Batches up to this size are launched with programmatic dependent launch (see pdl_enter).
+constexpr int kPdlMaxBatch = 16;
+
+// One kernel launch; with `pdl` the launch carries the programmatic stream serialisation
+// attribute, so the kernel may be scheduled while its predecessor in the stream still runs (it
+// waits for that predecessor in pdl_enter before it touches memory).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 bool pdl, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1u : 0u;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 }  // namespace octo

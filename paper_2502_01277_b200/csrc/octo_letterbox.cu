@@ -20,8 +20,10 @@ constexpr int kLbRows = 8;  // most output rows a CTA produces; fewer for very w
 template <int CAP>
 __global__ void __launch_bounds__(kLbThreads)
 letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict__ out, int S, int band_rows,
-                 int slot_bytes, uint32_t fill_h2, int swap_rb, unsigned int* __restrict__ status) {
+                 int slot_bytes, int nslots, uint32_t fill_h2, int swap_rb, unsigned int* __restrict__ status,
+                 int pdl) {
     extern __shared__ __align__(128) unsigned char smem[];
+    pdl_enter(pdl);
     __shared__ __align__(8) uint64_t bar;
     __shared__ __align__(16) RowInfo s_row[kLbRows];  // per-row data; step < 0 marks a canvas (pad) row
 
@@ -83,6 +85,16 @@ letterbox_kernel(const __grid_constant__ FrameTable<CAP> tab, __half* __restrict
             int y0, ry;
             src_coord(iy, h, nh, inv_dy, y0, ry);
             const uint8_t* src = fd.data + (size_t)y0 * (size_t)fd.pitch;
+#ifdef OCTO_BOUNDS_CHECK
+            if (!OCTO_IN_RANGE(slot + (ry != 0 ? 2 : 1) <= nslots && (int)row_bytes + 16 <= slot_bytes &&
+                               y0 + (ry != 0 ? 1 : 0) < h && (int)row_bytes <= fd.pitch, status)) {
+                // keep the barrier's byte count right without touching memory
+                asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&bar)),
+                             "r"(row_bytes * (ry != 0 ? 2u : 1u)) : "memory");
+                slot += ry != 0 ? 2 : 1;
+                continue;
+            }
+#endif
             bulk_g2s(s_rows + (size_t)slot * slot_bytes, src, row_bytes, &bar);
             if (ry != 0) bulk_g2s(s_rows + (size_t)(slot + 1) * slot_bytes, src + fd.pitch, row_bytes, &bar);
             slot += ry != 0 ? 2 : 1;
@@ -147,10 +159,10 @@ static size_t lb_smem_bytes(int S, int slots, int slot_bytes) {
 
 template <int CAP>
 static cudaError_t launch_cap(const FrameDesc* frames, int n, void* d_out, int S, int max_w, int pad_value,
-                              int swap_rb, unsigned int* d_status, cudaStream_t stream) {
-    static FrameTable<CAP> tab;  // host staging; a stage is used from one thread at a time
+                              int swap_rb, unsigned int* d_status, bool pdl, cudaStream_t stream) {
+    FrameTable<CAP> tab;  // built per call (copied into kernel parameter space by the launch)
     for (int i = 0; i < n; ++i) tab.f[i] = frames[i];
-    const int slot_bytes = ((3 * max_w + 15) & ~15) + 16;
+    const int slot_bytes = ((3 * max_w + 15) & ~15) + 16;  // 16 bytes of slack: a tap reads 12 bytes from its word
     // rows per CTA: as many as fit about 56 KB of shared memory (four CTAs per SM), at most
     // kLbRows, at least one (a single row of the widest supported frame still fits)
     const int per_row = slots_per_row(frames, n) * slot_bytes;
@@ -164,9 +176,9 @@ static cudaError_t launch_cap(const FrameDesc* frames, int n, void* d_out, int S
     const uint32_t fb = *reinterpret_cast<const unsigned short*>(&hf);
     const uint32_t fill_h2 = fb | (fb << 16);
     dim3 grid((S + band_rows - 1) / band_rows, n);
-    letterbox_kernel<CAP><<<grid, kLbThreads, smem, stream>>>(tab, reinterpret_cast<__half*>(d_out), S, band_rows, slot_bytes,
-                                                             fill_h2, swap_rb, d_status);
-    return cudaGetLastError();
+    return launch_kernel(letterbox_kernel<CAP>, grid, dim3(kLbThreads), smem, stream, pdl, tab,
+                         reinterpret_cast<__half*>(d_out), S, band_rows, slot_bytes,
+                         band_rows * slots_per_row(frames, n), fill_h2, swap_rb, d_status, pdl ? 1 : 0);
 }
 
 // largest dynamic shared memory a launch may ask for (see kLetterboxMaxWidth)
@@ -182,10 +194,10 @@ cudaError_t prepare_letterbox() {
 }
 
 cudaError_t launch_letterbox(const FrameDesc* frames, int n, void* d_out, int S, int max_w, int pad_value,
-                             int swap_rb, unsigned int* d_status, cudaStream_t stream) {
-    if (n <= 8) return launch_cap<8>(frames, n, d_out, S, max_w, pad_value, swap_rb, d_status, stream);
-    if (n <= 64) return launch_cap<64>(frames, n, d_out, S, max_w, pad_value, swap_rb, d_status, stream);
-    return launch_cap<512>(frames, n, d_out, S, max_w, pad_value, swap_rb, d_status, stream);
+                             int swap_rb, unsigned int* d_status, bool pdl, cudaStream_t stream) {
+    if (n <= 8) return launch_cap<8>(frames, n, d_out, S, max_w, pad_value, swap_rb, d_status, pdl, stream);
+    if (n <= 64) return launch_cap<64>(frames, n, d_out, S, max_w, pad_value, swap_rb, d_status, pdl, stream);
+    return launch_cap<512>(frames, n, d_out, S, max_w, pad_value, swap_rb, d_status, pdl, stream);
 }
 
 }  // namespace octo

@@ -75,16 +75,21 @@ __device__ __forceinline__ float4 gather_box(const float* __restrict__ p, size_t
 
 template <int CAP>
 __global__ void __launch_bounds__(kNmsThreads, 1)
-nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict__ head, int A, int C, int layout,
+nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restrict__ gtab,
+           const float* __restrict__ head, int A, int C, int layout,
            const IouTest iou_test, int max_det, int key_stride, unsigned long long* __restrict__ gkeys,
            float4* __restrict__ gboxes, int* __restrict__ cand_count, octo_det_rec* __restrict__ dets,
            int* __restrict__ counts, int num_branches, int class_agnostic,
            const __grid_constant__ BranchMasks masks,
-           int* __restrict__ bcount, int* __restrict__ bidx, int max_batch, StageCounters* __restrict__ ctr) {
+           int* __restrict__ bcount, int* __restrict__ bidx, int max_batch, StageCounters* __restrict__ ctr,
+           int pdl) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    pdl_enter(pdl);
     __shared__ int seg_start[128], seg_cnt[128], cursor[128], nkept[128];
     __shared__ int live[128];  // classes with survivors
-    __shared__ int s_total, s_live, s_big;
+    __shared__ int s_total, s_live, s_big, s_nout;
+    unsigned int* const status = &ctr->status;
+    (void)status;  // referenced by the range checks of the checked build only
 
     const int img = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -94,8 +99,12 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
     const size_t as = layout == OCTO_HEAD_PLANES ? 1 : (size_t)(nbox + C);  // anchor to anchor
     const float* __restrict__ hbase = head + (size_t)img * (size_t)A * (size_t)(nbox + C);
 
+    // The frame table comes by value (first-level stages) or from device memory (chained stages,
+    // where an entry without a frame stands for an unused slot of the batch: no detections).
+    const FrameDesc fd = gtab ? gtab[img] : tab.f[img];
     int cnt = cand_count[img];
     cnt = min(cnt, key_stride);
+    if (gtab && fd.data == nullptr) cnt = 0;
     if (threadIdx.x < 128) { seg_cnt[threadIdx.x] = 0; nkept[threadIdx.x] = 0; }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -140,109 +149,120 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
         unsigned int* const sup = reinterpret_cast<unsigned int*>(sbox + kSmallMax);  // [kSmallMax][kSmallWords]
         unsigned char* const alive = reinterpret_cast<unsigned char*>(sup + kSmallMax * kSmallWords);
         const int t = threadIdx.x;
-        unsigned long long k = kKeySentinel;
-        float4 box = make_float4(0.f, 0.f, 0.f, 0.f);
-        int cls = 0;
-        if (t == 0) s_m = 0;
-        if (t < cnt) {
-            k = gk[t];
-            cls = (int)(k >> 57);
-            atomicAdd(&seg_cnt[cls], 1);
-            box = gather_box(hbase + (size_t)(k & ((1ull << kKeyAnchorBits) - 1)) * as, es);
-        }
-        __syncthreads();
-        if (warp == 0) {
-            int run = 0;
-#pragma unroll
-            for (int base = 0; base < 128; base += 32) {
-                const int v = seg_cnt[base + lane];
-                int inc = v;
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const int u = __shfl_up_sync(0xffffffffu, inc, off);
-                    if (lane >= off) inc += u;
-                }
-                seg_start[base + lane] = run + inc - v;
-                cursor[base + lane] = run + inc - v;
-                run += __shfl_sync(0xffffffffu, inc, 31);
+        // Only the first kSmallMax threads work here; they meet at a barrier of their own, so the
+        // phases are not paced by the 24 warps that have nothing to do.
+        auto bar_small = []() { asm volatile("bar.sync 1, %0;" ::"n"(kSmallMax) : "memory"); };
+        if (t < kSmallMax) {
+            unsigned long long k = kKeySentinel;
+            float4 box = make_float4(0.f, 0.f, 0.f, 0.f);
+            int cls = 0;
+            if (t == 0) s_m = 0;
+            if (t < cnt) {
+                k = gk[t];
+                cls = (int)(k >> 57);
+                atomicAdd(&seg_cnt[cls], 1);
+                box = gather_box(hbase + (size_t)(k & ((1ull << kKeyAnchorBits) - 1)) * as, es);
             }
-        }
-        __syncthreads();
-        if (t < cnt) {
-            const int pos = atomicAdd(&cursor[cls], 1);
-            ukey[pos] = k;
-            ubox[pos] = box;
-        }
-        __syncthreads();
-        int start = 0;
-        if (t < cnt) {  // from here on thread t owns bucket position t
-            k = ukey[t];
-            box = ubox[t];
-            cls = (int)(k >> 57);
-            start = seg_start[cls];
-            const int m = seg_cnt[cls];
-            int r = 0;
-            for (int j = start; j < start + m; ++j) r += ukey[j] < k;
-            skey[start + r] = k;
-            sbox[start + r] = box;
-        }
-        __syncthreads();
-        if (t < cnt) {  // ... and ordered position t (same class, hence the same start)
-            const float4 bi = sbox[t];
-            const int words = (t - start + 31) >> 5;  // words that hold predecessors
-            for (int w = 0; w < words; ++w) {
-                unsigned bits = 0u;
-                const int j0 = start + (w << 5), j1 = min(j0 + 32, t);
-                for (int j = j0; j < j1; ++j)
-                    if (iou_above(sbox[j], bi, iou_test)) bits |= 1u << (j - j0);
-                sup[t * kSmallWords + w] = bits;
-            }
-        }
-        __syncthreads();
-        if (t < cnt && t == start) {  // first position of a class: walk the class in order
-            const int m = seg_cnt[cls];
-            if (m <= 32) {
-                unsigned kept = 0u;
-                alive[t] = 1;
-                kept = 1u;
-                for (int i = 1; i < m; ++i) {
-                    const bool ok = (sup[(t + i) * kSmallWords] & kept) == 0u;
-                    alive[t + i] = ok ? 1 : 0;
-                    if (ok) kept |= 1u << i;
-                }
-            } else {
-                unsigned kept[kSmallWords];
-#pragma unroll
-                for (int w = 0; w < kSmallWords; ++w) kept[w] = 0u;
-                for (int i = 0; i < m; ++i) {
-                    bool ok = true;
-#pragma unroll
-                    for (int w = 0; w < kSmallWords; ++w)
-                        if (w < ((i + 31) >> 5) && (sup[(t + i) * kSmallWords + w] & kept[w]) != 0u) ok = false;
-                    alive[t + i] = ok ? 1 : 0;
-#pragma unroll
-                    for (int w = 0; w < kSmallWords; ++w)
-                        if (ok && w == (i >> 5)) kept[w] |= 1u << (i & 31);
+            bar_small();
+            if (warp == 0) {
+                int run = 0;
+    #pragma unroll
+                for (int base = 0; base < 128; base += 32) {
+                    const int v = seg_cnt[base + lane];
+                    int inc = v;
+    #pragma unroll
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const int u = __shfl_up_sync(0xffffffffu, inc, off);
+                        if (lane >= off) inc += u;
+                    }
+                    seg_start[base + lane] = run + inc - v;
+                    cursor[base + lane] = run + inc - v;
+                    run += __shfl_sync(0xffffffffu, inc, 31);
                 }
             }
+            bar_small();
+            if (t < cnt) {
+                const int pos = atomicAdd(&cursor[cls], 1);
+                if (OCTO_IN_RANGE(pos >= 0 && pos < kSmallMax, status)) {
+                    ukey[pos] = k;
+                    ubox[pos] = box;
+                }
+            }
+            bar_small();
+            int start = 0;
+            if (t < cnt) {  // from here on thread t owns bucket position t
+                k = ukey[t];
+                box = ubox[t];
+                cls = (int)(k >> 57);
+                start = seg_start[cls];
+                const int m = seg_cnt[cls];
+                int r = 0;
+                for (int j = start; j < start + m; ++j) r += ukey[j] < k;
+                if (OCTO_IN_RANGE(start + r >= 0 && start + r < kSmallMax, status)) {
+                    skey[start + r] = k;
+                    sbox[start + r] = box;
+                }
+            }
+            bar_small();
+            if (t < cnt) {  // ... and ordered position t (same class, hence the same start)
+                const float4 bi = sbox[t];
+                const int words = (t - start + 31) >> 5;  // words that hold predecessors
+                for (int w = 0; w < words; ++w) {
+                    unsigned bits = 0u;
+                    const int j0 = start + (w << 5), j1 = min(j0 + 32, t);
+                    for (int j = j0; j < j1; ++j)
+                        if (iou_above(sbox[j], bi, iou_test)) bits |= 1u << (j - j0);
+                    sup[t * kSmallWords + w] = bits;
+                }
+            }
+            bar_small();
+            if (t < cnt && t == start) {  // first position of a class: walk the class in order
+                const int m = seg_cnt[cls];
+                if (m <= 32) {
+                    unsigned kept = 0u;
+                    alive[t] = 1;
+                    kept = 1u;
+                    for (int i = 1; i < m; ++i) {
+                        const bool ok = (sup[(t + i) * kSmallWords] & kept) == 0u;
+                        alive[t + i] = ok ? 1 : 0;
+                        if (ok) kept |= 1u << i;
+                    }
+                } else {
+                    unsigned kept[kSmallWords];
+    #pragma unroll
+                    for (int w = 0; w < kSmallWords; ++w) kept[w] = 0u;
+                    for (int i = 0; i < m; ++i) {
+                        bool ok = true;
+    #pragma unroll
+                        for (int w = 0; w < kSmallWords; ++w)
+                            if (w < ((i + 31) >> 5) && (sup[(t + i) * kSmallWords + w] & kept[w]) != 0u) ok = false;
+                        alive[t + i] = ok ? 1 : 0;
+    #pragma unroll
+                        for (int w = 0; w < kSmallWords; ++w)
+                            if (ok && w == (i >> 5)) kept[w] |= 1u << (i & 31);
+                    }
+                }
+            }
+            bar_small();
+            unsigned long long g = kKeySentinel;
+            const bool mine = t < cnt && alive[t] != 0;
+            if (mine) {
+                const unsigned long long ks = skey[t];
+                g = ((ks & ((1ull << 57) - 1)) << 7) | (ks >> 57);  // inverted score | anchor | class
+                const int q = atomicAdd(&s_m, 1);
+                if (OCTO_IN_RANGE(q >= 0 && q < kSmallMax, status)) surv[q] = g;
+            }
+            bar_small();
+            const int m_all = s_m;
+            if (mine) {
+                int r = 0;
+                for (int j = 0; j < m_all; ++j) r += surv[j] < g;
+                if (r < max_det && OCTO_IN_RANGE(r < kSmallMax, status)) ordered[r] = g;
+            }
+            if (t == 0) s_nout = min(m_all, max_det);
         }
         __syncthreads();
-        unsigned long long g = kKeySentinel;
-        const bool mine = t < cnt && alive[t] != 0;
-        if (mine) {
-            const unsigned long long ks = skey[t];
-            g = ((ks & ((1ull << 57) - 1)) << 7) | (ks >> 57);  // inverted score | anchor | class
-            surv[atomicAdd(&s_m, 1)] = g;
-        }
-        __syncthreads();
-        const int m_all = s_m;
-        if (mine) {
-            int r = 0;
-            for (int j = 0; j < m_all; ++j) r += surv[j] < g;
-            if (r < max_det) ordered[r] = g;
-        }
-        nout = min(m_all, max_det);
-        __syncthreads();
+        nout = s_nout;
     } else {
         // ---- bucket the keys by class: histogram, scan, scatter ----
         for (int i = threadIdx.x; i < cnt; i += kNmsThreads) atomicAdd(&seg_cnt[(int)(gk[i] >> 57)], 1);
@@ -270,7 +290,8 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
             unsigned long long* const dst = on_chip ? keys : reinterpret_cast<unsigned long long*>(boxes);
             for (int i = threadIdx.x; i < cnt; i += kNmsThreads) {
                 const unsigned long long k = gk[i];
-                dst[atomicAdd(&cursor[(int)(k >> 57)], 1)] = k;
+                const int pos = atomicAdd(&cursor[(int)(k >> 57)], 1);
+                if (OCTO_IN_RANGE(pos >= 0 && pos < cnt, status)) dst[pos] = k;
             }
             __syncthreads();
             if (!on_chip) {
@@ -353,7 +374,7 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
                 const int allowed = min(__popc(keptmask), max_det - nk);
                 if ((keptmask >> lane) & 1u) {
                     const int r = __popc(keptmask & ((1u << lane) - 1u));
-                    if (r < allowed) {
+                    if (r < allowed && OCTO_IN_RANGE(s + nk + r < e, status)) {
                         boxes[s + nk + r] = b;
                         // re-key for the global order: inverted score | anchor | class
                         keys[s + nk + r] = ((k & ((1ull << 57) - 1)) << 7) | (k >> 57);
@@ -422,7 +443,7 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
                 const int mid = (l2 + h2) >> 1;
                 if (list[mid] < g) l2 = mid + 1; else h2 = mid;
             }
-            if (l2) atomicAdd(&rank[e], l2);
+            if (l2 && OCTO_IN_RANGE(e >= 0 && e < total, status)) atomicAdd(&rank[e], l2);
         }
         __syncthreads();
         for (int e = threadIdx.x; e < total; e += kNmsThreads) {
@@ -433,13 +454,13 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
                 const int mid = (lo + hi) >> 1;
                 if (cursor[mid] <= e) lo = mid; else hi = mid;
             }
-            ordered[r] = keys[seg_start[live[lo]] + (e - cursor[lo])];
+            if (OCTO_IN_RANGE(r >= 0 && r < min(max_det, cnt), status))
+                ordered[r] = keys[seg_start[live[lo]] + (e - cursor[lo])];
         }
         __syncthreads();
         nout = min(s_total, max_det);
     }
 
-    const FrameDesc& fd = tab.f[img];
     // region of the source frame shown by the detector input: x in [x_lo, x_hi], y likewise
     const float fpl = (float)fd.pad_l, fpt = (float)fd.pad_t;
     const float x_lo = (float)fd.ox, y_lo = (float)fd.oy;
@@ -490,7 +511,8 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const float* __restrict_
                 take = (masks.m[warp][cls >> 5] >> (cls & 31u)) & 1u;
             }
             const unsigned bal = __ballot_sync(0xffffffffu, take);
-            if (take) list[m + __popc(bal & ((1u << lane) - 1u))] = r;
+            if (take && OCTO_IN_RANGE(m + __popc(bal & ((1u << lane) - 1u)) < max_det, status))
+                list[m + __popc(bal & ((1u << lane) - 1u))] = r;
             m += __popc(bal);
         }
         if (lane == 0) bcount[warp * max_batch + img] = m;
@@ -510,8 +532,9 @@ cudaError_t prepare_nms() {
 
 template <int CAP>
 static cudaError_t launch_cap(const NmsArgs& a, cudaStream_t stream) {
-    static FrameTable<CAP> tab;
-    for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
+    FrameTable<CAP> tab;  // built per call (copied into kernel parameter space by the launch)
+    if (!a.d_tab)
+        for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
     const size_t smem = kNmsSmemBytes;
     // rounding boundary of the IoU test (see iou_above)
     const float up = nextafterf(a.iou_thr, INFINITY);
@@ -520,12 +543,10 @@ static cudaError_t launch_cap(const NmsArgs& a, cudaStream_t stream) {
     unsigned int up_bits;
     memcpy(&up_bits, &up, sizeof(up_bits));
     iou_test.tie_up = (up_bits & 1u) == 0u ? 1 : 0;
-    nms_kernel<CAP><<<a.n, kNmsThreads, smem, stream>>>(tab, a.d_head, a.A, a.C, a.layout, iou_test, a.max_det, a.key_stride,
-                                                       a.d_keys, a.d_boxes, a.d_cand_count,
-                                                       reinterpret_cast<octo_det_rec*>(a.d_dets), a.d_counts,
-                                                       a.num_branches, a.class_agnostic, a.masks, a.d_bcount, a.d_bidx, a.max_batch,
-                                                       a.d_ctr);
-    return cudaGetLastError();
+    return launch_kernel(nms_kernel<CAP>, dim3(a.n), dim3(kNmsThreads), smem, stream, a.pdl, tab, a.d_tab, a.d_head, a.A,
+                         a.C, a.layout, iou_test, a.max_det, a.key_stride, a.d_keys, a.d_boxes, a.d_cand_count,
+                         reinterpret_cast<octo_det_rec*>(a.d_dets), a.d_counts, a.num_branches, a.class_agnostic,
+                         a.masks, a.d_bcount, a.d_bidx, a.max_batch, a.d_ctr, a.pdl ? 1 : 0);
 }
 
 cudaError_t launch_nms(const NmsArgs& a, cudaStream_t stream) {

@@ -115,10 +115,10 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
         return OCTO_E_ALIGNMENT;
 
     cudaError_t e = cudaSetDevice(device);
-    if (e != cudaSuccess) return OCTO_E_CUDA;
+    if (e != cudaSuccess) return report_cuda_error(e, "cudaSetDevice");
     unsigned char* base = nullptr;
     e = setup_device(device, &base);
-    if (e != cudaSuccess) return OCTO_E_CUDA;
+    if (e != cudaSuccess) return report_cuda_error(e, "workspace set-up (cudaGetSymbolAddress)");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     unsigned long long* d_keys = reinterpret_cast<unsigned long long*>(base + kOffKeys);
@@ -131,7 +131,7 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
     // The array keeps whatever the previous call left: the candidate counter and the counter
     // block must start at zero; keys and boxes are overwritten before they are read.
     e = cudaMemsetAsync(base + kOffBcount, 0, kScratchBytes - kOffBcount, stream);
-    if (e != cudaSuccess) return OCTO_E_CUDA;
+    if (e != cudaSuccess) return report_cuda_error(e, "cudaMemsetAsync");
 
     int key_stride = 2;
     while (key_stride < num_anchors) key_stride <<= 1;  // <= kStaticMaxAnchors
@@ -144,13 +144,16 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
     da.conf = conf_thresh;
     da.key_stride = key_stride;
     da.d_keys = d_keys; da.d_cand_count = d_cand; da.d_status = &d_ctr->status;
+    da.pdl = false;
     e = launch_decode(da, stream);
-    if (e != cudaSuccess) return OCTO_E_CUDA;
+    if (e != cudaSuccess) return report_cuda_error(e, "decode_kernel");
 
     FrameDesc fd;
     frame_geometry(frame_w, frame_h, net_size, &fd);
     NmsArgs a;
     a.frames = &fd;
+    a.d_tab = nullptr;
+    a.pdl = false;
     a.n = 1;
     a.d_head = d_head;
     a.A = num_anchors;
@@ -172,6 +175,22 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
     a.max_batch = 1;
     a.d_ctr = d_ctr;
     e = launch_nms(a, stream);
-    if (e != cudaSuccess) return OCTO_E_CUDA;
+    if (e != cudaSuccess) return report_cuda_error(e, "nms_kernel");
+    return OCTO_OK;
+}
+
+extern "C" int octo_static_status(int32_t device, uint32_t* status_word, void* cuda_stream) {
+    if (!status_word || device < 0 || device >= kMaxDevices) return OCTO_E_INVALID_ARG;
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) return report_cuda_error(e, "cudaSetDevice");
+    unsigned char* base = nullptr;
+    e = setup_device(device, &base);
+    if (e != cudaSuccess) return report_cuda_error(e, "workspace set-up (cudaGetSymbolAddress)");
+    e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return report_cuda_error(e, "cudaStreamSynchronize");
+    unsigned int w = 0;
+    e = cudaMemcpy(&w, &reinterpret_cast<StageCounters*>(base + kOffCtr)->status, sizeof(w), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return report_cuda_error(e, "cudaMemcpy");
+    *status_word = w;
     return OCTO_OK;
 }

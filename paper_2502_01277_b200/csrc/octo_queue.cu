@@ -28,10 +28,12 @@ constexpr int kQueueThreads = 1024;
 
 template <int CAP>
 __global__ void __launch_bounds__(kQueueThreads)
-queue_push_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_det, const int* __restrict__ bcount,
+queue_push_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restrict__ gtab, int n, int max_det,
+                  const int* __restrict__ bcount,
                   const int* __restrict__ bidx, const octo_det_t* __restrict__ dets, QRecord* __restrict__ ring,
                   int cap, QueueState* __restrict__ state) {
     __shared__ int s_off[CAP + 1];
+    pdl_enter(0);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (warp == 0) {
         int run = 0;
@@ -64,7 +66,7 @@ queue_push_kernel(const __grid_constant__ FrameTable<CAP> tab, int n, int max_de
         const int f = lo;
         const int det = bidx[(size_t)f * max_det + (item - s_off[f])];
         const octo_det_t d = dets[(size_t)f * max_det + det];
-        const FrameDesc& fd = tab.f[f];
+        const FrameDesc fd = gtab ? gtab[f] : tab.f[f];
         // outward-rounded rectangle, clamped so that it is never empty
         int rx0 = (int)floorf(d.x1), ry0 = (int)floorf(d.y1);
         int rx1 = (int)ceilf(d.x2), ry1 = (int)ceilf(d.y2);
@@ -90,6 +92,7 @@ __global__ void __launch_bounds__(256)
 queue_pop_kernel(const QRecord* __restrict__ ring, int cap, QueueState* __restrict__ state, int bz, int max_wait,
                  QRecord* __restrict__ staged, QRecord* __restrict__ items_out, int* __restrict__ info,
                  int* __restrict__ qpacked) {
+    pdl_enter(0);
     const long long head = state->head, tail = state->tail;
     const long long pending = tail - head;
     // max_wait < 0: release whatever is pending.  Otherwise a batch is released when it is full, or
@@ -119,11 +122,12 @@ queue_pop_kernel(const QRecord* __restrict__ ring, int cap, QueueState* __restri
 template <int CAP>
 static cudaError_t push_cap(const octo_stage* st, int branch, QRecord* ring, int cap, QueueState* state,
                             cudaStream_t stream) {
-    static FrameTable<CAP> tab;
-    for (int i = 0; i < st->n_frames; ++i) tab.f[i] = st->frames[i];
+    FrameTable<CAP> tab;  // built per call (copied into kernel parameter space by the launch)
+    if (!st->tab_on_device)
+        for (int i = 0; i < st->n_frames; ++i) tab.f[i] = st->frames[i];
     const octo_stage_config_t& c = st->cfg;
     queue_push_kernel<CAP><<<1, kQueueThreads, 0, stream>>>(
-        tab, st->n_frames, c.max_det, st->d_bcount + (size_t)branch * c.max_batch,
+        tab, st->tab_on_device ? st->d_tab : nullptr, st->n_frames, c.max_det, st->d_bcount + (size_t)branch * c.max_batch,
         st->d_bidx + (size_t)branch * c.max_batch * c.max_det, st->d_dets, ring, cap, state);
     return cudaGetLastError();
 }

@@ -30,10 +30,14 @@ struct ScopedKernelTimer {
 
 static thread_local char g_cuda_err[256] = "";
 
-static int cuda_fail(cudaError_t e, const char* what) {
+namespace octo {
+// Records the text octo_last_cuda_error returns on this thread; always returns OCTO_E_CUDA.
+int report_cuda_error(cudaError_t e, const char* what) {
     snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
     return OCTO_E_CUDA;
 }
+}  // namespace octo
+static int cuda_fail(cudaError_t e, const char* what) { return octo::report_cuda_error(e, what); }
 #define OCTO_CUDA(call)                                     \
     do {                                                    \
         cudaError_t e__ = (call);                           \
@@ -113,6 +117,7 @@ static void free_all(octo_stage* st) {
     cudaFree(st->d_bidx);
     for (int b = 0; b < OCTO_MAX_BRANCHES; ++b) cudaFree(st->d_items[b]);
     cudaFree(st->d_ctr);
+    cudaFree(st->d_tab);
     for (int i = 0; i < 2 * kEventPairs; ++i)
         if (st->ev[i]) cudaEventDestroy(st->ev[i]);
 }
@@ -129,17 +134,20 @@ extern "C" int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** 
     OCTO_CUDA(cudaSetDevice(cfg->device));
 
     octo_stage* st = new (std::nothrow) octo_stage();
-    if (!st) return OCTO_E_INVALID_ARG;
+    if (!st) return OCTO_E_NO_MEMORY;
     memset(st, 0, sizeof(*st));
     st->cfg = *cfg;
-    OCTO_CUDA(cudaDeviceGetAttribute(&st->sm_count, cudaDevAttrMultiProcessorCount, cfg->device));
+    cudaError_t e = cudaDeviceGetAttribute(&st->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
+    if (e != cudaSuccess) {
+        delete st;
+        return cuda_fail(e, "cudaDeviceGetAttribute");
+    }
     int ks = 2;
     while (ks < cfg->num_anchors) ks <<= 1;
     if (cfg->multi_label) ks <<= 1;  // an anchor can yield several candidates
     st->key_stride = ks;
 
     const size_t mb = (size_t)cfg->max_batch;
-    cudaError_t e = cudaSuccess;
     if (e == cudaSuccess) e = dev_alloc(&st->d_keys, mb * ks, &st->workspace_bytes);
     if (e == cudaSuccess) e = dev_alloc(&st->d_boxes, mb * ks, &st->workspace_bytes);
     if (e == cudaSuccess) e = dev_alloc(&st->d_cand_count, mb, &st->workspace_bytes);
@@ -149,13 +157,16 @@ extern "C" int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** 
     for (int b = 0; b < cfg->num_branches && e == cudaSuccess; ++b)
         e = dev_alloc(&st->d_items[b], mb * cfg->max_det, &st->workspace_bytes);
     if (e == cudaSuccess) e = dev_alloc(&st->d_ctr, 1, &st->workspace_bytes);
+    if (e == cudaSuccess) e = dev_alloc(&st->d_tab, mb, &st->workspace_bytes);
     if (e == cudaSuccess) e = prepare_letterbox();
     if (e == cudaSuccess) e = prepare_nms();
     if (e == cudaSuccess) e = prepare_crop();
     if (e != cudaSuccess) {
         free_all(st);
         delete st;
-        return cuda_fail(e, "octo_stage_create");
+        cuda_fail(e, "octo_stage_create");
+        (void)cudaGetLastError();  // the failure is reported here, not by a later call
+        return e == cudaErrorMemoryAllocation ? OCTO_E_NO_MEMORY : OCTO_E_CUDA;
     }
     *out = st;
     return OCTO_OK;
@@ -211,6 +222,7 @@ extern "C" int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frame
     }
     st->n_frames = 0;
     st->have_dets = false;
+    st->tab_on_device = false;
     for (int i = 0; i < n; ++i) {
         FrameDesc& fd = st->frames[i];
         fd.data = frames[i].d_data;
@@ -224,7 +236,8 @@ extern "C" int octo_preprocess_batch(octo_stage_t* st, const octo_frame_t* frame
     {
         ScopedKernelTimer t(st, OCTO_K_LETTERBOX, static_cast<cudaStream_t>(cuda_stream));
         OCTO_CUDA(launch_letterbox(st->frames, n, d_out_f16_nchw, st->cfg.net_size, max_w, st->cfg.pad_value,
-                                   st->cfg.swap_rb, &st->d_ctr->status, static_cast<cudaStream_t>(cuda_stream)));
+                                   st->cfg.swap_rb, &st->d_ctr->status, n <= kPdlMaxBatch,
+                                   static_cast<cudaStream_t>(cuda_stream)));
     }
     st->launches += 1;
     st->n_frames = n;
@@ -247,6 +260,7 @@ extern "C" int octo_adopt_regions(octo_stage_t* st, const octo_region_t* regions
     }
     st->n_frames = 0;
     st->have_dets = false;
+    st->tab_on_device = false;
     for (int i = 0; i < n; ++i) {
         const octo_region_t& r = regions[i];
         FrameDesc& fd = st->frames[i];
@@ -267,6 +281,101 @@ extern "C" int octo_adopt_regions(octo_stage_t* st, const octo_region_t* regions
     }
     st->max_w = 0;
     st->n_frames = n;
+    return OCTO_OK;
+}
+
+// ---- device-side hand-off between cascade levels ---------------------------------------------
+// One thread per entry of the chained stage's batch: entry i becomes item first + i of the
+// upstream branch (original frame + rectangle, stretched to S x S, no padding), or an empty
+// entry (no frame: the NMS kernel reports no detections for it) when the upstream branch packed
+// fewer items.  The arithmetic is the host's (octo_adopt_regions): gains by IEEE division.
+namespace octo {
+template <int CAP>
+__global__ void __launch_bounds__(256)
+adopt_items_kernel(const __grid_constant__ FrameTable<CAP> up_tab, const FrameDesc* __restrict__ up_gtab,
+                   const octo_item_t* __restrict__ items, const int* __restrict__ up_n_items, int first, int n, int S,
+                   FrameDesc* __restrict__ out) {
+    pdl_enter(0);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    FrameDesc fd;
+    memset(&fd, 0, sizeof(fd));
+    const int slot = first + i;
+    if (slot < up_n_items[0]) {
+        const octo_item_t it = items[slot];
+        const FrameDesc src = up_gtab ? up_gtab[it.frame] : up_tab.f[it.frame];
+        fd.data = src.data;
+        fd.w = src.w; fd.h = src.h; fd.pitch = src.pitch;
+        fd.nw = S; fd.nh = S;
+        fd.ox = (uint16_t)it.rx0; fd.oy = (uint16_t)it.ry0;
+        fd.rw = (uint16_t)(it.rx1 - it.rx0); fd.rh = (uint16_t)(it.ry1 - it.ry0);
+        fd.gx = __fdiv_rn(__int2float_rn(it.rx1 - it.rx0), __int2float_rn(S));
+        fd.gy = __fdiv_rn(__int2float_rn(it.ry1 - it.ry0), __int2float_rn(S));
+    }
+    out[i] = fd;
+}
+
+template <int CAP>
+static cudaError_t launch_adopt(const octo_stage* up, const octo_item_t* d_items, const int* d_n_items, int first,
+                                int n, int S, FrameDesc* d_out, cudaStream_t stream) {
+    FrameTable<CAP> tab;
+    if (!up->tab_on_device)
+        for (int i = 0; i < up->n_frames; ++i) tab.f[i] = up->frames[i];
+    return launch_kernel(adopt_items_kernel<CAP>, dim3((n + 255) / 256), dim3(256), 0, stream, false, tab,
+                         up->tab_on_device ? up->d_tab : (const FrameDesc*)nullptr, d_items, d_n_items, first, n, S,
+                         d_out);
+}
+
+// Test support: a wait that nothing ends.  One thread arms an mbarrier for `bytes` bytes that no
+// copy will ever deliver, polls it `polls` times, reports the timeout in the status word and
+// returns.  No copy is in flight at any point and the shared memory dies with the CTA.
+__global__ void wait_selftest_kernel(unsigned int* __restrict__ status, int polls) {
+    __shared__ __align__(8) uint64_t bar;
+    pdl_enter(0);
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+        mbar_expect_tx(&bar, 64u);
+        if (!mbar_wait_bounded(&bar, 0, polls)) atomicOr(status, 0x4u);
+    }
+}
+}  // namespace octo
+
+extern "C" int octo_adopt_items_device(octo_stage_t* st, const octo_stage_t* upstream, int32_t branch, int32_t first,
+                                       int32_t n, void* cuda_stream) {
+    if (!st || !upstream || st == upstream || n < 1 || first < 0) return OCTO_E_INVALID_ARG;
+    if (branch < 0 || branch >= upstream->cfg.num_branches) return OCTO_E_INVALID_ARG;
+    if (upstream->cfg.device != st->cfg.device) return OCTO_E_INVALID_ARG;
+    if (n > st->cfg.max_batch) return OCTO_E_CAPACITY;
+    if ((long long)first + n > (long long)upstream->cfg.max_batch * upstream->cfg.max_det) return OCTO_E_CAPACITY;
+    if (upstream->n_frames < 1) return OCTO_E_NO_PREPROCESS;
+    if (!upstream->d_last_n_items[branch]) return OCTO_E_NO_POSTPROCESS;  // the branch was never cropped
+    // the upstream crop (a plain stretch of the rectangle to S x S) is this stage's detector input
+    if (upstream->cfg.branch[branch].out_w != st->cfg.net_size || upstream->cfg.branch[branch].out_h != st->cfg.net_size)
+        return OCTO_E_INVALID_ARG;
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st->n_frames = 0;
+    st->have_dets = false;
+    cudaError_t e;
+    const int un = upstream->tab_on_device ? 1 : upstream->n_frames;
+    if (un <= 8) e = launch_adopt<8>(upstream, upstream->d_items[branch], upstream->d_last_n_items[branch], first, n, st->cfg.net_size, st->d_tab, stream);
+    else if (un <= 64) e = launch_adopt<64>(upstream, upstream->d_items[branch], upstream->d_last_n_items[branch], first, n, st->cfg.net_size, st->d_tab, stream);
+    else e = launch_adopt<512>(upstream, upstream->d_items[branch], upstream->d_last_n_items[branch], first, n, st->cfg.net_size, st->d_tab, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "adopt_items_kernel");
+    st->launches += 1;
+    st->tab_on_device = true;
+    st->max_w = 0;
+    st->n_frames = n;
+    return OCTO_OK;
+}
+
+extern "C" int octo_stage_selftest_wait(octo_stage_t* st, int32_t polls, void* cuda_stream) {
+    if (!st || polls < 1 || polls > (1 << 20)) return OCTO_E_INVALID_ARG;
+    OCTO_CUDA(cudaSetDevice(st->cfg.device));
+    OCTO_CUDA(launch_kernel(wait_selftest_kernel, dim3(1), dim3(32), 0, static_cast<cudaStream_t>(cuda_stream), false,
+                            &st->d_ctr->status, (int)polls));
+    st->launches += 1;
     return OCTO_OK;
 }
 
@@ -292,11 +401,14 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
         da.conf = c.conf_thresh;
         da.key_stride = st->key_stride;
         da.d_keys = st->d_keys; da.d_cand_count = st->d_cand_count; da.d_status = &st->d_ctr->status;
+        da.pdl = n <= kPdlMaxBatch;
         OCTO_CUDA(launch_decode(da, stream));
     }
     st->launches += 1;
     NmsArgs a;
     a.frames = st->frames;
+    a.d_tab = st->tab_on_device ? st->d_tab : nullptr;
+    a.pdl = n <= kPdlMaxBatch;
     a.n = n;
     a.d_head = d_head;
     a.A = c.num_anchors;
@@ -350,6 +462,8 @@ extern "C" int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_i
     if (max_items > cap) max_items = (int32_t)cap;  // a branch can never hold more items
     CropArgs a;
     a.frames = st->frames;
+    a.d_tab = st->tab_on_device ? st->d_tab : nullptr;
+    a.pdl = st->n_frames <= kPdlMaxBatch;
     a.n = st->n_frames;
     a.max_det = c.max_det;
     a.first_item = first_item;
@@ -375,6 +489,7 @@ extern "C" int octo_crop_batch(octo_stage_t* st, int32_t branch, int32_t first_i
         OCTO_CUDA(launch_crop(a, stream));
     }
     st->launches += 1;
+    st->d_last_n_items[branch] = d_n_items;
     return OCTO_OK;
 }
 
@@ -472,6 +587,7 @@ extern "C" const char* octo_strerror(int code) {
         case OCTO_E_CUDA: return "CUDA runtime error";
         case OCTO_E_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
         case OCTO_E_NO_POSTPROCESS: return "the current batch has not been postprocessed";
+        case OCTO_E_NO_MEMORY: return "out of host or device memory";
         default: return "unknown status code";
     }
 }

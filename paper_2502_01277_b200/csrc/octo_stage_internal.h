@@ -18,13 +18,16 @@ struct octo_stage {
     int* d_bidx;    // [branches][max_batch][max_det]
     octo_item_t* d_items[OCTO_MAX_BRANCHES];
     octo::StageCounters* d_ctr;
+    octo::FrameDesc* d_tab;  // [max_batch] frame table of a batch adopted on the device (chained stage)
     int64_t workspace_bytes;
     // host state of the current batch
     octo::FrameDesc frames[OCTO_MAX_BATCH];
     int n_frames;
+    bool tab_on_device;  // the current batch's table is d_tab (octo_adopt_items_device), not `frames`
     int max_w;
     bool have_dets;
     const octo_det_t* d_dets;
+    const int32_t* d_last_n_items[OCTO_MAX_BRANCHES];  // {packed, total} of the last crop call per branch (caller's buffer)
     int64_t launches;
     // optional per-kernel timing
     bool timing;

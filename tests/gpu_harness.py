@@ -77,7 +77,15 @@ def run_stage_gpu(stage, frames: Sequence[np.ndarray], sizes, head: np.ndarray,
     return res
 
 
-def half_absdiff(a_bits: np.ndarray, b_bits: np.ndarray) -> float:
-    a = a_bits.view(np.float16).astype(np.float32)
-    b = b_bits.view(np.float16).astype(np.float32)
-    return float(np.max(np.abs(a - b))) if a.size else 0.0
+def half_absdiff(a_bits: np.ndarray, b_bits: np.ndarray, chunk: int = 1 << 24) -> float:
+    """Largest |a - b| over two arrays of binary16 bit patterns, taken in slices so that a
+    whole batch of crops (gigabytes) never exists as float32 at once."""
+    assert a_bits.shape == b_bits.shape
+    a = np.ascontiguousarray(a_bits).reshape(-1)
+    b = np.ascontiguousarray(b_bits).reshape(-1)
+    worst = 0.0
+    for lo in range(0, a.size, chunk):
+        x = a[lo:lo + chunk].view(np.float16).astype(np.float32)
+        y = b[lo:lo + chunk].view(np.float16).astype(np.float32)
+        worst = max(worst, float(np.max(np.abs(x - y))))
+    return worst

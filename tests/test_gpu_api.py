@@ -124,3 +124,107 @@ def test_repeated_passes_are_bit_identical():
     finally:
         for st in stages:
             st.close()
+
+
+def test_two_host_threads_drive_two_stages():
+    """Stage objects share no host state: two threads, each with a stage, a stream and a batch of
+    its own (different frame sizes, so a mixed-up frame table would move every box), run 200 passes
+    side by side on one GPU; every pass of both must give the oracle's detections, the last one
+    also its rectangles and crops."""
+    import threading
+    from dataclasses import replace
+
+    import oracle
+    import workloads
+    from gpu_harness import half_absdiff
+
+    passes = 200
+    dev = torch.device("cuda", 0)
+    specs = [(replace(workloads.WORKLOADS["traffic_1080p"], frame_sizes=((640, 360),), branches=((64, 64),)), 2, 71),
+             (replace(workloads.WORKLOADS["traffic_1080p"], frame_sizes=((1280, 720),), branches=((96, 32),)), 3, 72)]
+    jobs, errors = [], []
+    for wl, n, seed in specs:
+        b = workloads.make_batch(wl, batch=n, seed=seed)
+        ref = oracle.run_stage(b.frames, b.sizes, b.head, wl.net_size, wl.branches, max_det=wl.max_det,
+                               do_letterbox=False, threads=4)
+        st = octo.Stage(net_size=wl.net_size, max_batch=n, num_anchors=wl.num_anchors, num_classes=wl.num_classes,
+                        max_det=wl.max_det, branches=wl.branches)
+        stream = torch.cuda.Stream(dev)
+        with torch.cuda.stream(stream):
+            frames = [torch.from_numpy(f).to(dev) for f in b.frames]
+            head = torch.from_numpy(b.head).to(dev)
+            det_in = torch.empty((n, 3, wl.net_size, wl.net_size), dtype=torch.float16, device=dev)
+            dets = torch.zeros((passes, n, wl.max_det, 32), dtype=torch.uint8, device=dev)
+            counts = torch.full((passes, n), -1, dtype=torch.int32, device=dev)
+            cap = len(ref.items[0]) + 2
+            ow, oh = wl.branches[0]
+            crops = torch.zeros((cap, 3, oh, ow), dtype=torch.float16, device=dev)
+            offs = torch.zeros((n + 1,), dtype=torch.int32, device=dev)
+            ni = torch.zeros((2,), dtype=torch.int32, device=dev)
+        stream.synchronize()
+        jobs.append(dict(b=b, ref=ref, st=st, stream=stream, frames=frames, head=head, det_in=det_in, dets=dets,
+                         counts=counts, crops=crops, offs=offs, ni=ni, cap=cap))
+    start = threading.Barrier(len(jobs))
+
+    def work(j):
+        try:
+            torch.cuda.set_device(dev)
+            start.wait()
+            for k in range(passes):
+                j["st"].preprocess(j["frames"], j["b"].sizes, out=j["det_in"], stream=j["stream"])
+                j["st"].postprocess(j["head"], dets=j["dets"][k], counts=j["counts"][k], stream=j["stream"])
+                j["st"].crop(0, j["cap"], out=j["crops"], offsets=j["offs"], n_items=j["ni"], stream=j["stream"])
+            j["stream"].synchronize()
+        except Exception as e:  # pragma: no cover
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    try:
+        for t in threads:
+            t.start()
+        for t in threads:
+            t.join()
+        assert not errors, errors
+        for j in jobs:
+            ref, n = j["ref"], j["b"].n
+            counts = j["counts"].cpu().numpy()
+            dets = j["dets"].cpu().numpy().view(octo.DET_DTYPE).reshape(passes, n, -1)
+            assert np.all(counts == ref.counts[None, :])
+            for i, k in enumerate(ref.counts):
+                want = ref.dets[i, :k].tobytes()
+                for p in range(passes):
+                    assert dets[p, i, :k].tobytes() == want, f"pass {p}, frame {i}"
+            packed, total = (int(v) for v in j["ni"].cpu())
+            assert packed == total == len(ref.items[0])
+            it = j["st"].item_table(0, packed)
+            assert np.array_equal(np.stack([it["rx0"], it["ry0"], it["rx1"], it["ry1"]], 1), ref.rects[0])
+            got = j["crops"][:packed].view(torch.int16).cpu().numpy().view(np.uint16)
+            assert half_absdiff(got, ref.crops[0]) <= 2e-3
+            assert j["st"].status(j["stream"]) == 0
+    finally:
+        for j in jobs:
+            j["st"].close()
+
+
+def test_a_wait_that_runs_out_is_reported_and_cleared(stage):
+    """The time-out path of the bounded device waits, made to run out without any copy in flight:
+    the self-test kernel arms a barrier for bytes nobody sends and gives up after a few hundred
+    polls.  The status word carries the bit, octo_stage_status reports OCTO_E_DEVICE_TIMEOUT, the
+    context stays usable, and clearing the word brings the stage back to OCTO_OK."""
+    lib = octo.load_library()
+    import ctypes
+    w = ctypes.c_uint32(0)
+    assert lib.octo_stage_status(stage.handle, ctypes.byref(w), None) == B.OCTO_OK and w.value == 0
+    stage.selftest_wait(polls=300)
+    rc = lib.octo_stage_status(stage.handle, ctypes.byref(w), None)
+    assert rc == B.OCTO_E_DEVICE_TIMEOUT and w.value & B.OCTO_STATUS_COPY_TIMEOUT
+    assert octo.octo_stage_status(stage.handle) & B.OCTO_STATUS_COPY_TIMEOUT
+    stage.clear_status()
+    assert lib.octo_stage_status(stage.handle, ctypes.byref(w), None) == B.OCTO_OK and w.value == 0
+    # the stage still works
+    f = _frame()
+    out = stage.preprocess([f], [(40, 30)])
+    torch.cuda.synchronize()
+    assert stage.status() == 0 and out.shape == (1, 3, 64, 64)
+    assert lib.octo_stage_selftest_wait(stage.handle, 0, None) == B.OCTO_E_INVALID_ARG
+    assert lib.octo_stage_selftest_wait(None, 10, None) == B.OCTO_E_INVALID_ARG

@@ -96,6 +96,104 @@ def test_two_level_cascade_matches_oracle(layout2, opts2):
             st2.close()
 
 
+def test_device_hand_off_equals_the_host_hand_off_and_the_oracle():
+    """octo_adopt_items_device: the chained stage reads the upstream item table on the device, with
+    no synchronisation in between.  The level-2 batch is provisioned larger than the number of
+    upstream items: the surplus entries (fed with a head full of raised candidates) must yield no
+    detections.  A window that starts inside the item table is taken as well."""
+    wl = replace(workloads.WORKLOADS["traffic_1080p"], branches=((256, 256),))
+    b = workloads.make_batch(wl, batch=3, seed=33)
+    s2, c2, max_det2 = 256, 6, 12
+    a2 = workloads.num_anchors(s2)
+    ref1 = oracle.run_stage(b.frames, b.sizes, b.head, wl.net_size, wl.branches, max_det=wl.max_det,
+                            do_letterbox=False, do_crops=False)
+    n1 = len(ref1.items[0])
+    assert n1 > 20
+    bz = n1 + 5                      # downstream batch size: five surplus entries
+    head2 = workloads.make_heads(78, bz, s2, num_classes=c2, n_raised=14, n_groups=4)
+    st1 = octo.Stage(net_size=wl.net_size, max_batch=b.n, num_anchors=wl.num_anchors, num_classes=wl.num_classes,
+                     max_det=wl.max_det, branches=wl.branches)
+    st2 = octo.Stage(net_size=s2, max_batch=bz, num_anchors=a2, num_classes=c2, max_det=max_det2, branches=((64, 32),))
+    stream = torch.cuda.Stream()
+    try:
+        with torch.cuda.stream(stream):
+            frames = [torch.from_numpy(f).cuda() for f in b.frames]
+            d_head1, d_head2 = torch.from_numpy(b.head).cuda(), torch.from_numpy(head2).cuda()
+        stream.synchronize()
+        for first in (0, 7):
+            m = bz - first           # entries of this level-2 batch (n1 - first of them are real)
+            cap2 = m * max_det2
+            # both levels are enqueued back to back: nothing reads the device in between
+            st1.preprocess(frames, b.sizes, stream=stream)
+            st1.postprocess(d_head1, stream=stream)
+            crops1, off1, ni1 = st1.crop(0, 256, stream=stream)
+            st2.adopt_items_device(st1, 0, m, first=first, stream=stream)
+            dets2, counts2 = st2.postprocess(d_head2[first:], stream=stream)
+            with torch.cuda.stream(stream):
+                buf = torch.full((cap2, 3, 32, 64), 0x7BFF, dtype=torch.int16, device="cuda")
+            _, off2, ni2 = st2.crop(0, cap2, out=buf.view(torch.float16), stream=stream)
+            stream.synchronize()
+            assert int(ni1[0]) == n1
+            d2, c2n = octo.dets_to_numpy(dets2, counts2)
+            packed2, total2 = (int(v) for v in ni2.cpu())
+            items2 = st2.item_table(0, packed2)
+            got = buf.cpu().numpy().view(np.uint16)
+            assert st2.status(stream) == 0 and st1.status(stream) == 0
+            ref_d = np.zeros((m, max_det2), dtype=DET_DTYPE)
+            ref_c = np.zeros(m, dtype=np.int32)
+            for i in range(n1 - first):
+                r = ref1.rects[0][first + i]
+                d, _ = oracle.postprocess_region(head2[first + i], tuple(int(v) for v in r), s2, max_det=max_det2)
+                ref_d[i, : len(d)] = d
+                ref_c[i] = len(d)
+            assert np.array_equal(c2n, ref_c) and np.all(c2n[n1 - first:] == 0) and int(ref_c.sum()) > n1 - first
+            for i in range(m):
+                assert d2[i, : ref_c[i]].tobytes() == ref_d[i, : ref_c[i]].tobytes(), f"entry {i}: detections differ"
+            offs, its, (pk, tot) = oracle.assemble(ref_d, ref_c, max_det2)
+            assert (packed2, total2) == (pk, tot) and np.array_equal(off2.cpu().numpy(), offs)
+            assert np.array_equal(np.stack([items2["frame"], items2["det"]], 1), its)
+            for k, (i, j) in enumerate(its):
+                f = int(ref1.items[0][first + i][0])  # the ORIGINAL frame behind upstream item first + i
+                w, h = b.sizes[f]
+                rect = oracle.crop_rect(ref_d[i, j], w, h)
+                assert (int(items2["rx0"][k]), int(items2["ry0"][k]), int(items2["rx1"][k]),
+                        int(items2["ry1"][k])) == rect
+                assert half_absdiff(got[k], oracle.crop(b.frames[f], w, h, ref_d[i, j], 64, 32)) <= 2e-3
+            assert np.all(got[packed2:] == 0x7BFF)
+    finally:
+        st1.close()
+        st2.close()
+
+
+def test_adopt_items_device_argument_errors():
+    from paper_2502_01277_b200 import binding as B
+    lib = octo.load_library()
+    up = octo.Stage(net_size=64, max_batch=2, num_anchors=252, num_classes=4, max_det=10, branches=((32, 32), (16, 16)))
+    st = octo.Stage(net_size=32, max_batch=4, num_anchors=63, num_classes=4, max_det=5, branches=((8, 8),))
+    try:
+        call = lambda s, u, br, first, n: lib.octo_adopt_items_device(s, u, br, first, n, None)  # noqa: E731
+        assert call(st.handle, up.handle, 0, 0, 2) == B.OCTO_E_NO_PREPROCESS      # upstream has no batch yet
+        f = torch.zeros((30, 128), dtype=torch.uint8, device="cuda")
+        up.preprocess([f], [(40, 30)])
+        assert call(st.handle, up.handle, 0, 0, 2) == B.OCTO_E_NO_POSTPROCESS     # branch 0 never cropped
+        up.postprocess(torch.full((1, 252, 9), -9.0, device="cuda"))
+        up.crop(0, 4)
+        up.crop(1, 4)
+        assert call(st.handle, up.handle, 0, 0, 4) == B.OCTO_OK
+        assert call(st.handle, up.handle, 0, 0, 5) == B.OCTO_E_CAPACITY           # n > max_batch
+        assert call(st.handle, up.handle, 0, 19, 4) == B.OCTO_E_CAPACITY          # window past the item table
+        assert call(st.handle, up.handle, 1, 0, 2) == B.OCTO_E_INVALID_ARG        # branch is not net_size wide
+        assert call(st.handle, up.handle, 2, 0, 2) == B.OCTO_E_INVALID_ARG
+        assert call(st.handle, up.handle, 0, -1, 2) == B.OCTO_E_INVALID_ARG
+        assert call(st.handle, up.handle, 0, 0, 0) == B.OCTO_E_INVALID_ARG
+        assert call(st.handle, st.handle, 0, 0, 2) == B.OCTO_E_INVALID_ARG
+        assert call(None, up.handle, 0, 0, 2) == B.OCTO_E_INVALID_ARG
+        torch.cuda.synchronize()
+    finally:
+        st.close()
+        up.close()
+
+
 def test_adopt_regions_argument_errors():
     from paper_2502_01277_b200 import binding as B
     st = octo.Stage(net_size=64, max_batch=2, num_anchors=252, num_classes=4, max_det=10, branches=((16, 16),))

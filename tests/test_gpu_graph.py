@@ -78,3 +78,78 @@ def test_stage_pass_replayed_from_a_cuda_graph():
             assert st.status(stream) == 0
     finally:
         st.close()
+
+
+@pytest.mark.parametrize("bz,max_wait", [(16, 1), (48, 0)])
+def test_queue_calls_replayed_from_one_graph_per_batch_size(bz, max_wait):
+    """The serving loop of one downstream model at a fixed batch size bz, recorded once: detector
+    pass (letterbox, decode + NMS), octo_queue_push and octo_queue_pop_due in ONE graph, replayed
+    for three detector batches.  The scene stays in the same frame buffers (queued items refer to
+    their frames by pointer), the detector heads change from batch to batch.  Records, release
+    decisions and crops are compared with the queue oracle after every replay."""
+    ow, oh, capacity = 64, 48, 160
+    wl = replace(workloads.WORKLOADS["traffic_1080p"], frame_sizes=((640, 360),), branches=((ow, oh),),
+                 n_raised=90, n_groups=12)
+    n = 2
+    batches = [workloads.make_batch(wl, batch=n, seed=60 + k) for k in range(3)]
+    scene = batches[0]
+    dev = torch.device("cuda", 0)
+    st = make_stage(wl, n)
+    warm = octo.Queue(capacity, ow, oh, max_bz=bz)   # takes the first launch of every kernel
+    q = octo.Queue(capacity, ow, oh, max_bz=bz)
+    oq = oracle.OracleQueue(capacity)
+    stream = torch.cuda.Stream(dev)
+    try:
+        with torch.cuda.stream(stream):
+            frames = [torch.from_numpy(f).to(dev) for f in scene.frames]
+            head = torch.from_numpy(batches[0].head).to(dev)
+            det_in = torch.empty((n, 3, wl.net_size, wl.net_size), dtype=torch.float16, device=dev)
+            dets = torch.zeros((n, wl.max_det, 32), dtype=torch.uint8, device=dev)
+            counts = torch.zeros((n,), dtype=torch.int32, device=dev)
+            buf = torch.full((bz, 3, oh, ow), 0x7BFF, dtype=torch.int16, device=dev)
+            items = torch.zeros((bz, octo.QITEM_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+            info = torch.zeros((4,), dtype=torch.int32, device=dev)
+
+        def serve(queue):
+            st.preprocess(frames, scene.sizes, out=det_in, stream=stream)
+            st.postprocess(head, dets=dets, counts=counts, stream=stream)
+            queue.push(st, 0, stream=stream)
+            queue.pop(bz, out=buf.view(torch.float16), items=items, info=info, stream=stream, max_wait=max_wait)
+
+        serve(warm)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            serve(q)
+        payload = [(scene.frames[i], scene.sizes[i], frames[i].data_ptr(), frames[i].stride(0)) for i in range(n)]
+        popped_total = 0
+        for bt in batches:
+            with torch.cuda.stream(stream):
+                head.copy_(torch.from_numpy(bt.head))
+                buf.fill_(0x7BFF)
+                graph.replay()
+            stream.synchronize()
+            ref = oracle.run_stage(scene.frames, scene.sizes, bt.head, wl.net_size, wl.branches, max_det=wl.max_det,
+                                   do_letterbox=False, do_crops=False)
+            oq.push(ref.items[0], ref.rects[0], payload)
+            orecs, oinfo = oq.pop(bz, max_wait)
+            assert tuple(int(v) for v in info.cpu()) == oinfo
+            recs = items.cpu().numpy().view(octo.QITEM_DTYPE).reshape(-1)
+            crops = buf.cpu().numpy().view(np.uint16)
+            for i, (seq, f, j, rect, (pix, (w, h), ptr, pitch)) in enumerate(orecs):
+                r = recs[i]
+                assert (int(r["seq"]), int(r["frame"]), int(r["det"])) == (seq, f, j)
+                assert (int(r["rx0"]), int(r["ry0"]), int(r["rx1"]), int(r["ry1"])) == rect
+                assert (int(r["d_data"]), int(r["pitch_bytes"])) == (ptr, pitch)
+                box = np.zeros(1, dtype=oracle.DET_DTYPE)
+                box["x1"], box["y1"], box["x2"], box["y2"] = rect
+                assert half_absdiff(crops[i], oracle.crop(pix, w, h, box, ow, oh)) <= PIX_TOL
+            assert np.all(crops[len(orecs):] == 0x7BFF)
+            popped_total += len(orecs)
+        assert popped_total > 0
+        if bz == 16:
+            assert oinfo[1] > 0  # items of earlier batches are still pending: the queue spans replays
+    finally:
+        warm.close()
+        q.close()
+        st.close()

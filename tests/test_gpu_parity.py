@@ -57,25 +57,22 @@ def _oracle(b, **kw):
     return oracle.run_stage(b.frames, b.sizes, b.head, wl.net_size, wl.branches, **args)
 
 
-def _full_config(name, batch=None, letterbox_frames=None, max_crops=None):
+def _full_config(name, batch=None):
+    """The whole stage on a workload batch: every letterboxed frame and every crop is compared
+    with the oracle, beside the detections, the packing and the rectangles."""
     b = workloads.make_batch(name, batch=batch)
     wl = b.workload
     st = make_stage(wl, b.n)
     try:
-        ref = _oracle(b, do_letterbox=letterbox_frames is None, max_crops=max_crops)
+        ref = _oracle(b)
         cap = [int(len(ref.items[k])) + 3 for k in range(len(wl.branches))]
         res = run_stage_gpu(st, b.frames, b.sizes, b.head, max_items=cap)
         assert res.status & ~0x8 == 0
-        if letterbox_frames is None:
-            d = half_absdiff(res.det_in, ref.det_in)
-            assert d <= PIX_TOL, f"letterbox max-abs {d}"
-        else:
-            for i in letterbox_frames:
-                w, h = b.sizes[i]
-                want = oracle.letterbox(b.frames[i], w, h, wl.net_size)
-                assert half_absdiff(res.det_in[i], want) <= PIX_TOL
+        d = half_absdiff(res.det_in, ref.det_in)
+        assert d <= PIX_TOL, f"letterbox max-abs {d}"
         _check_dets(res, ref)
         for k in range(len(wl.branches)):
+            assert len(ref.crops[k]) == len(ref.items[k])  # the oracle rendered every crop
             packed = _check_branch(res, ref, k, max_items=cap[k])
             # slots beyond the packed ones are untouched
             assert np.all(res.crops[k][packed:] == 0x7BFF)
@@ -106,38 +103,19 @@ def test_config_two_branch():
 
 
 def test_config_dense_nms():
-    b, res, ref = _full_config("dense_nms", letterbox_frames=[0, 31])
+    b, res, ref = _full_config("dense_nms")
     assert int(ref.n_cand.min()) > 4000 and int(ref.counts.max()) <= 1000
 
 
-@pytest.mark.parametrize("batch", [1, 4, 16, 64])
+@pytest.mark.parametrize("batch", [1, 4, 16, 64, 256])
 def test_config_sweep(batch):
-    _full_config("sweep", batch=batch, letterbox_frames=[0, batch - 1] if batch > 8 else None)
-
-
-def test_config_sweep_256_sampled():
-    """Full-size sweep point: detections and packing checked on every frame, pixels on a
-    sample of frames and crops (the oracle renders those one by one)."""
-    b = workloads.make_batch("sweep", batch=256)
-    wl = b.workload
-    st = make_stage(wl, b.n)
-    try:
-        ref = _oracle(b, do_letterbox=False, do_crops=False)
-        total = len(ref.items[0])
-        res = run_stage_gpu(st, b.frames, b.sizes, b.head, max_items=[256 * wl.items_per_frame])
-        _check_dets(res, ref)
-        _check_branch(res, ref, 0, max_items=256 * wl.items_per_frame)
-        rng = np.random.default_rng(0)
-        for i in rng.choice(256, 6, replace=False):
-            w, h = b.sizes[i]
-            assert half_absdiff(res.det_in[i], oracle.letterbox(b.frames[i], w, h, wl.net_size)) <= PIX_TOL
-        for k in rng.choice(total, 96, replace=False):
-            f, j = ref.items[0][k]
-            w, h = b.sizes[f]
-            want = oracle.crop(b.frames[f], w, h, ref.dets[f, j], 224, 224)
-            assert half_absdiff(res.crops[0][k], want) <= PIX_TOL
-    finally:
-        st.close()
+    """Every point of the throughput sweep, the benchmarked B = 256 included, on the whole batch
+    (3:1 point sampling makes the letterbox bit-exact)."""
+    b, res, ref = _full_config("sweep", batch=batch)
+    assert np.array_equal(res.det_in, ref.det_in)
+    if batch == 256:
+        # the launch shape the benchmark times: whole crops as tiles, the last ones cut into bands
+        assert res.n_items[0][0] > 3 * 148 * 4
 
 
 # ---- letterbox geometry / resize cases --------------------------------------------------

@@ -4,9 +4,11 @@ octo_postprocess_frame_static exists for programs that cannot allocate GPU memor
 they run (a real-time loop with a fixed memory budget, a plug-in living in a host
 application's pool): it decodes one frame's head and runs NMS on a workspace compiled into
 the library instead of one obtained from cudaMalloc.  It must return exactly what
-octo_postprocess_batch returns for the same frame.  The workspace is shared by all calls and
-keeps old contents, so the check is made on two calls in a row, the second with far fewer
-candidates than the first, then on the first input again.
+octo_postprocess_batch returns for the same frame, which in turn is what the CPU oracle computes.
+The workspace is shared by all calls and keeps old contents, so the check is made on calls in a
+row whose candidate counts go up and down: a dense head, a head with more candidates than the
+NMS kernel holds on chip (the part of the workspace that only the global-memory path uses), a
+sparse head, and the first two again.  The status word of each call is read back as well.
 
 This file is named so that pytest collects it after every other test file.
 """
@@ -16,6 +18,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2502_01277_b200 as octo
 import workloads
 from paper_2502_01277_b200 import binding as B
@@ -29,7 +32,14 @@ def _heads():
     base = replace(workloads.WORKLOADS["traffic_1080p"], frame_sizes=((W, H),))
     dense = workloads.make_batch(replace(base, n_raised=3000, n_groups=200, max_det=300), batch=1, seed=21)
     sparse = workloads.make_batch(replace(base, n_raised=120, n_groups=15, max_det=300), batch=1, seed=22)
-    return dense, sparse
+    huge = workloads.make_batch(replace(base, n_raised=9500, n_groups=700, max_det=300), batch=1, seed=23)
+    return dense, sparse, huge
+
+
+def _via_oracle(batch, max_det=300):
+    wl = batch.workload
+    d, ncand = oracle.postprocess_image(batch.head[0], W, H, S, True, wl.conf_thresh, wl.iou_thresh, max_det)
+    return d, int(ncand)
 
 
 def _via_stage(stage, batch):
@@ -49,29 +59,52 @@ def _via_static(batch, max_det=300):
     octo.octo_postprocess_frame_static(0, head.data_ptr(), wl.num_anchors, wl.num_classes, True, wl.conf_thresh,
                                        wl.iou_thresh, max_det, S, W, H, dets.data_ptr(), count.data_ptr(),
                                        int(torch.cuda.current_stream().cuda_stream))
-    torch.cuda.synchronize()
+    status = octo.octo_static_status(0, int(torch.cuda.current_stream().cuda_stream))  # synchronises
     c = int(count.item())
     d = dets.cpu().numpy().view(B.DET_DTYPE).reshape(-1)
-    return d[:c].copy(), c
+    return d[:c].copy(), c, status
 
 
 def test_static_workspace_entry_matches_stage_entry_on_consecutive_calls():
-    dense, sparse = _heads()
+    dense, sparse, huge = _heads()
     wl = dense.workload
     stage = octo.Stage(net_size=S, max_batch=1, num_anchors=wl.num_anchors, num_classes=wl.num_classes,
                        max_det=300, branches=((64, 64),))
     try:
-        want_dense, n_dense = _via_stage(stage, dense)
-        want_sparse, n_sparse = _via_stage(stage, sparse)
+        via_stage = {id(b): _via_stage(stage, b) for b in (dense, sparse, huge)}
     finally:
         stage.close()
-    assert n_dense > n_sparse > 5
-    # two calls in a row on the shared workspace, then the first input once more
-    for batch, want, n in ((dense, want_dense, n_dense), (sparse, want_sparse, n_sparse),
-                           (dense, want_dense, n_dense)):
-        got, c = _via_static(batch)
+    via_oracle = {id(b): _via_oracle(b) for b in (dense, sparse, huge)}
+    assert via_oracle[id(huge)][1] > 8192 > via_oracle[id(dense)][1] > 256 > via_oracle[id(sparse)][1]
+    assert via_stage[id(dense)][1] > via_stage[id(sparse)][1] > 5
+    # calls in a row on the shared workspace; the candidate count goes up and down between them
+    for batch in (dense, huge, sparse, huge, dense, sparse):
+        got, c, status = _via_static(batch)
+        want, n = via_stage[id(batch)]
         assert c == n
         assert got.tobytes() == want.tobytes()  # same bit-exact bar as the other detection tests
+        ref, _ = via_oracle[id(batch)]
+        assert c == len(ref) and got.tobytes() == ref[:c].tobytes()  # and the oracle itself
+        # more candidates than fit on chip take the global-memory path and say so; nothing else is set
+        assert status == (B.OCTO_STATUS_BIG_NMS if batch is huge else 0)
+
+
+def test_static_workspace_entry_reports_dropped_rows():
+    """A head row with a non-finite value is dropped, as by a stage, and the status word of the call
+    says so; the next call starts from a clean word."""
+    _, sparse, _ = _heads()
+    bad = sparse.head[0].copy()
+    raised = np.nonzero(bad[:, 4] > 0)[0]
+    bad[raised[0], 0] = np.nan
+    bad[raised[1], 5 + 3] = np.inf
+    wl = sparse.workload
+    want, _ = oracle.postprocess_image(bad, W, H, S, True, wl.conf_thresh, wl.iou_thresh, 300)
+    broken = replace(sparse, head=bad[None])
+    got, c, status = _via_static(broken)
+    assert c == len(want) and got.tobytes() == want[:c].tobytes()
+    assert status == B.OCTO_STATUS_NONFINITE
+    _, _, status = _via_static(sparse)
+    assert status == 0
 
 
 def test_static_workspace_entry_rejects_sizes_beyond_its_limits():
