@@ -57,7 +57,8 @@ def parse_args():
     p.add_argument("--gpus", type=int, default=1)
     p.add_argument("--steps", type=int, default=30)
     p.add_argument("--warmup", type=int, default=5)
-    p.add_argument("--workload", default="sweep", choices=sorted(workloads.WORKLOADS) + ["two_level"])
+    p.add_argument("--workload", default="sweep", choices=sorted(workloads.WORKLOADS) + ["two_level", "queue"])
+    p.add_argument("--bz", type=int, default=64, help="downstream batch size of the queue workload")
     p.add_argument("--batch", type=int, default=None, help="frames per GPU per step")
     p.add_argument("--impl", default="octo", choices=["octo", "reference"])
     p.add_argument("--e2e-steps", type=int, default=None)
@@ -73,6 +74,8 @@ def parse_args():
 def default_batch(name: str) -> int:
     if name == "two_level":
         return 64
+    if name == "queue":
+        return 2  # the detector batch size the paper gives its baselines; about 44 items per step
     return 256 if name == "sweep" else workloads.WORKLOADS[name].batch
 
 
@@ -239,7 +242,7 @@ def run_reference(args):
     if rank != 0:
         return
     name = args.workload
-    if name == "two_level":
+    if name in ("two_level", "queue"):
         print(json.dumps({"impl": "reference", "unavailable": "the reference arm covers the single-stage workloads"}))
         return
     bsz = args.batch or default_batch(name)
@@ -807,10 +810,102 @@ def run_two_level(args):
     st2.close()
 
 
+def run_queue(args):
+    """Serving loop of one downstream model at a fixed batch size bz: per step one detector batch
+    (letterbox, decode + NMS), octo_queue_push of its items and octo_queue_pop_due of one batch of bz
+    crops (released when full, or when its first item has waited one push).  Timed with stream
+    launches and replayed from ONE CUDA graph per bz.  Single GPU."""
+    import torch
+
+    import paper_2502_01277_b200 as octo
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    n, bz = args.batch or default_batch("queue"), args.bz
+    wl = workloads.WORKLOADS["traffic_1080p"]
+    batch = workloads.make_batch(wl, batch=n)
+    ow, oh = wl.branches[0]
+    st = octo.Stage(net_size=wl.net_size, max_batch=n, num_anchors=wl.num_anchors, num_classes=wl.num_classes,
+                    max_det=wl.max_det, branches=wl.branches)
+    stream = torch.cuda.Stream(dev)
+    n_sets = 8  # rotating detector inputs and crop outputs, larger than L2 together
+    with torch.cuda.stream(stream):
+        frames = [torch.from_numpy(f).to(dev) for f in batch.frames]
+        heads = [torch.from_numpy(batch.head).to(dev) for _ in range(n_sets)]
+        det_in = [torch.empty((n, 3, wl.net_size, wl.net_size), dtype=torch.float16, device=dev) for _ in range(n_sets)]
+        dets = torch.zeros((n, wl.max_det, 32), dtype=torch.uint8, device=dev)
+        counts = torch.zeros((n,), dtype=torch.int32, device=dev)
+        crops = [torch.empty((bz, 3, oh, ow), dtype=torch.float16, device=dev) for _ in range(n_sets)]
+        items = torch.zeros((bz, octo.QITEM_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+        info = torch.zeros((4,), dtype=torch.int32, device=dev)
+    stream.synchronize()
+
+    def serve(q, k):
+        st.preprocess(frames, batch.sizes, out=det_in[k], stream=stream)
+        st.postprocess(heads[k], dets=dets, counts=counts, stream=stream)
+        q.push(st, 0, stream=stream)
+        q.pop(bz, out=crops[k], items=items, info=info, stream=stream, max_wait=1)
+
+    def measure(fn):
+        for i in range(max(args.warmup, 3)):
+            fn(i)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(args.steps):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / args.steps
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    q1 = octo.Queue(64 * bz, ow, oh, max_bz=bz)
+    ms_stream = measure(lambda i: serve(q1, i % n_sets))
+    q1.close()
+    q2 = octo.Queue(64 * bz, ow, oh, max_bz=bz)
+    serve(q2, 0)  # first launches outside the capture
+    stream.synchronize()
+    graphs = []
+    for k in range(n_sets):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            serve(q2, k)
+        graphs.append(g)
+
+    def replay(i):
+        with torch.cuda.stream(stream):
+            graphs[i % n_sets].replay()
+
+    ms_graph = measure(replay)
+    clocks = sampler.stop()
+    popped, pending, dropped, _ = (int(v) for v in info.cpu())
+    q2.close()
+    ms = ms_graph if args.graph else ms_stream
+    line = {
+        "metric": METRIC, "value": n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"queue B={n} bz={bz}", "frames": "1920x1080", "crops": [ow, oh],
+                   "launch": "CUDA graph replay (one graph per bz)" if args.graph else "stream launches",
+                   "last_pop": {"popped": popped, "pending": pending, "dropped": dropped},
+                   "l2": f"{n_sets} rotating input/output sets"},
+        "us_per_step": {"stream_launches": 1e3 * ms_stream, "graph_replay": 1e3 * ms_graph},
+        "e2e": None, "gpu_launches": 5 * args.steps, "clocks": clocks, "roofline": None, "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+    st.close()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "queue":
+        run_queue(args)
     elif args.workload == "two_level":
         run_two_level(args)
     else:

@@ -429,14 +429,14 @@ OCTO_API int octo_static_status(int32_t device, uint32_t* status_word, void* cud
  * several streams side by side; an execution occupies a portion of one stream, as long as its
  * run time and as wide as the share of the GPU's compute it needs; a stream repeats with a duty
  * cycle (half the pipeline's SLO).  Instances are placed one replica number at a time over all
- * pipelines and their models in order.  Each goes to the free portion with the least spare room
- * that (1) covers the window [start_us, end_us) it needs inside the cycle, (2) keeps the GPU
- * within memory (sum of weights + per-stream largest intermediate memory <= mem_bytes) and
- * utilisation (sum over streams of the widest resident <= util_max_permille) and (3) lies on a
- * stream whose duty cycle is not longer than the instance's.  The first instance on a stream
- * fixes the stream's duty cycle; the unused parts of the portion return to the free list.
- * Free portions are ordered by length, then GPU, stream and start; an empty stream offers one
- * unbounded portion.  All arrays are host memory; no CUDA call is made. */
+ * pipelines and their models in order.  Each goes to the stream whose free gap around the window
+ * [start_us, end_us) is the tightest (the least spare room), among the streams where (1) that
+ * window is free and inside the stream's cycle, (2) the GPU stays within memory (sum of weights +
+ * per-stream largest intermediate memory <= mem_bytes) and utilisation (sum over streams of the
+ * widest resident <= util_max_permille) and (3) the stream's duty cycle is not longer than the
+ * instance's.  Ties go to the lower GPU, then the lower stream.  The first instance on a stream
+ * fixes the stream's duty cycle; a stream without residents counts as an unbounded gap, so it is
+ * only taken when no bounded gap fits.  All arrays are host memory; no CUDA call is made. */
 typedef struct {
     int32_t pipeline, model, instance; /* pipeline index, position in its execution order, replica number */
     int32_t util_permille;             /* width: share of the GPU's compute, 0..1000            */

@@ -1,18 +1,22 @@
 """CPU oracle of the stream / portion placement (test infrastructure only).
 
-Follows the paper's co-location scheduler (Section III-C, Algorithm 2) in its own notation:
-FreePortions, pt, s = pt_stream, g = s_gpu, W_g / I_g / U_g, w_g / i_g / u_g, duty_cycle_r,
-duty_cycle_s, DividePortion, UpdateList.  Where the paper is silent this oracle takes these
-readings: FreePortions is ordered by portion length, then gpu, stream, start (so that the first
-feasible portion is the best fit, "minimal empty space"); a stream with no duty cycle yet offers
-one portion [0, infinity), cut to the duty cycle once the first instance fixes it; I_g is the sum
-over the GPU's streams of I_s, the largest intermediate memory among a stream's residents; times
-are integer microseconds.
+The paper's co-location scheduler (Section III-C, Algorithm 2) places model instances on the
+streams of GPUs: one replica number at a time over all pipelines and their models; each
+instance takes, among the free portions that cover its window, keep the GPU within memory and
+utilisation and lie on a stream whose duty cycle is not longer than the instance's, the one with
+the least empty space.  This oracle is that statement written as an exhaustive search: nothing is
+kept between instances except the list of placements made so far; every quantity (the free gap of
+a stream around the window, a GPU's memory and utilisation with the newcomer) is recomputed from
+that list for every stream of every GPU, and the feasible candidate with the smallest gap wins.
+Readings where the paper is silent: ties go to the lower GPU, then the lower stream; a stream
+without residents has no duty cycle and counts as an unbounded gap; a GPU's intermediate memory is
+the sum over its streams of the largest intermediate memory among the stream's residents, its
+utilisation the sum over its streams of the widest resident; times are integer microseconds.
 """
 from __future__ import annotations
 
 from dataclasses import dataclass
-from typing import Dict, List, Optional, Sequence, Tuple
+from typing import List, Optional, Sequence, Tuple
 
 INF = float("inf")
 
@@ -25,66 +29,63 @@ class Instance:
     start: int
     end: int
     duty_cycle: int
-    W: int        # weight memory W_m
-    I: int        # intermediate memory I_m
-    U: int        # utilisation U_r (permille)
+    W: int        # weight memory
+    I: int        # intermediate memory
+    U: int        # utilisation (permille)
 
 
 @dataclass
 class Gpu:
-    M: int        # memory M_g
-    U_max: int    # utilisation limit U_g^max (permille)
+    M: int        # memory
+    U_max: int    # utilisation limit (permille)
     streams: int
+
+
+def scheduling_order(instances: Sequence[Instance]) -> List[int]:
+    """Indices in the order the instances are placed: replica number, pipeline, model."""
+    return sorted(range(len(instances)), key=lambda i: (instances[i].instance, instances[i].pipeline,
+                                                        instances[i].model, i))
+
+
+def candidates(r: Instance, placed: Sequence[Tuple[Instance, int, int]], gpus: Sequence[Gpu]):
+    """Every (gap length, gpu, stream) where r could go, given the placements made so far
+    (`placed` = [(instance, gpu, stream)]), by exhaustive search."""
+    out = []
+    for g, gpu in enumerate(gpus):
+        on_gpu = [(q, s) for q, gg, s in placed if gg == g]
+        for s in range(gpu.streams):
+            res = [q for q, ss in on_gpu if ss == s]
+            duty = res[0].duty_cycle if res else 0  # the first resident fixed it (placements are in order)
+            if duty > r.duty_cycle:
+                continue
+            if any(q.start < r.end and r.start < q.end for q in res):
+                continue  # the window is not free
+            if res and r.end > duty:
+                continue  # the window does not lie inside the stream's cycle
+            lo = max([q.end for q in res if q.end <= r.start], default=0)
+            hi = min([q.start for q in res if q.start >= r.end], default=(duty if res else INF))
+            streams = {}
+            for q, ss in on_gpu + [(r, s)]:
+                streams.setdefault(ss, []).append(q)
+            mem = sum(q.W for q, _ in on_gpu) + r.W + sum(max(q.I for q in lst) for lst in streams.values())
+            util = sum(max(q.U for q in lst) for lst in streams.values())
+            if mem > gpu.M or util > gpu.U_max:
+                continue
+            out.append((hi - lo, g, s))
+    return out
 
 
 def schedule(instances: Sequence[Instance], gpus: Sequence[Gpu]) -> List[Optional[Tuple[int, int, int, int, int]]]:
     """Returns per instance (gpu, stream, start, end, duty cycle of the stream) or None."""
-    W = [0] * len(gpus)                                              # W_g
-    I_s: Dict[Tuple[int, int], int] = {}                             # per stream
-    U_s: Dict[Tuple[int, int], int] = {}                             # widest resident per stream
-    duty: Dict[Tuple[int, int], int] = {}                            # duty_cycle_s (0 = unset)
-    FreePortions: List[Tuple[int, int, float, float]] = []           # (gpu, stream, start, end)
-    for g, gpu in enumerate(gpus):
-        for s in range(gpu.streams):
-            I_s[(g, s)] = 0
-            U_s[(g, s)] = 0
-            duty[(g, s)] = 0
-            FreePortions.append((g, s, 0, INF))
-
-    def key(pt):
-        return (pt[3] - pt[2], pt[0], pt[1], pt[2])
-
+    placed: List[Tuple[Instance, int, int]] = []
     result: List[Optional[Tuple[int, int, int, int, int]]] = [None] * len(instances)
-    # Main: instanceNumber = 0, 1, ...; for p in scheduledPipelines; for m in p
-    numbers = sorted({r.instance for r in instances})
-    pipelines = sorted({r.pipeline for r in instances})
-    for instanceNumber in numbers:
-        for p in pipelines:
-            members = sorted((r.model, i) for i, r in enumerate(instances)
-                             if r.pipeline == p and r.instance == instanceNumber)
-            for _, i in members:
-                r = instances[i]
-                for pt in sorted(FreePortions, key=key):
-                    g, s, pt_start, pt_end = pt
-                    w_g = W[g] + r.W
-                    I_g = sum(I_s[(g, q)] for q in range(gpus[g].streams))
-                    i_g = I_g - I_s[(g, s)] + max(I_s[(g, s)], r.I)
-                    u_g = sum(max(U_s[(g, q)], r.U) if q == s else U_s[(g, q)] for q in range(gpus[g].streams))
-                    fully_available = pt_start <= r.start and pt_end >= r.end
-                    sufficient = w_g + i_g <= gpus[g].M and u_g <= gpus[g].U_max
-                    if fully_available and sufficient and r.duty_cycle >= duty[(g, s)]:
-                        if duty[(g, s)] == 0:
-                            duty[(g, s)] = r.duty_cycle
-                        W[g] = w_g
-                        I_s[(g, s)] = max(I_s[(g, s)], r.I)
-                        U_s[(g, s)] = max(U_s[(g, s)], r.U)
-                        # DividePortion / UpdateList
-                        FreePortions.remove(pt)
-                        cycle_end = min(pt_end, duty[(g, s)])
-                        if pt_start < r.start:
-                            FreePortions.append((g, s, pt_start, r.start))
-                        if r.end < cycle_end:
-                            FreePortions.append((g, s, r.end, cycle_end))
-                        result[i] = (g, s, r.start, r.end, duty[(g, s)])
-                        break
+    for i in scheduling_order(instances):
+        r = instances[i]
+        cands = candidates(r, placed, gpus)
+        if not cands:
+            continue
+        _, g, s = min(cands)
+        placed.append((r, g, s))
+        duty = next(q.duty_cycle for q, gg, ss in placed if (gg, ss) == (g, s))
+        result[i] = (g, s, r.start, r.end, duty)
     return result

@@ -341,74 +341,76 @@ void orc_scale_back(orc_det_t* d, int32_t w, int32_t h, int32_t S) {
     orc_scale_back_region(d, nw, nh, pl, pt, 0, 0, w, h);
 }
 
-/* R3..R6 for one image: head -> dets[<= max_det] in frame pixels.  Returns kept count;
- * *n_cand receives the candidate count before NMS. */
+/* R3..R6 for one detector input: decode, order, NMS, cap, then every kept box mapped into the
+ * source frame through the region map {nw, nh, pl, pt, ox, oy, rw, rh} of R6.  variants = 0 takes
+ * the plain row decode (orc_decode), 1 the decode with head layout and multi-label candidates
+ * (orc_decode_ex).  Returns the kept count; *n_cand receives the candidate count before NMS. */
+static int32_t postprocess_core(const float* head, int32_t A, int32_t C, int32_t logits, float conf, float iou_thr,
+                                int32_t max_det, int32_t agnostic, int32_t variants, int32_t layout,
+                                int32_t multi_label, const int32_t map[8], orc_det_t* dets, int32_t* n_cand) {
+    const size_t cap = (size_t)(A > 0 ? A : 1) * (size_t)(variants && multi_label ? (C > 0 ? C : 1) : 1);
+    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * cap);
+    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
+    int32_t n = variants ? orc_decode_ex(head, A, C, logits, conf, layout, multi_label, cand, (int32_t)cap)
+                         : orc_decode(head, A, C, logits, conf, cand);
+    orc_sort(cand, n);
+    int32_t k = orc_nms_ex(cand, n, iou_thr, max_det, agnostic, keep);
+    for (int32_t t = 0; t < k; ++t) {
+        dets[t] = cand[keep[t]];
+        orc_scale_back_region(&dets[t], map[0], map[1], map[2], map[3], map[4], map[5], map[6], map[7]);
+    }
+    if (n_cand) *n_cand = n;
+    free(cand);
+    free(keep);
+    return k;
+}
+
+/* First-level stage: the region is the whole w x h frame, letterboxed by R1. */
+static void frame_map(int32_t w, int32_t h, int32_t S, int32_t map[8]) {
+    orc_letterbox_geometry(w, h, S, &map[0], &map[1], &map[2], &map[3]);
+    map[4] = 0; map[5] = 0; map[6] = w; map[7] = h;
+}
+
+/* Chained (second-level) stage: the detector input is the upstream crop of the rectangle
+ * [ox, ox+rw) x [oy, oy+rh), stretched to S x S (no padding), so the head's boxes live on that
+ * S x S grid and map back into the rectangle of the ORIGINAL frame. */
+static void region_map(int32_t S, int32_t ox, int32_t oy, int32_t rw, int32_t rh, int32_t map[8]) {
+    map[0] = S; map[1] = S; map[2] = 0; map[3] = 0;
+    map[4] = ox; map[5] = oy; map[6] = rw; map[7] = rh;
+}
+
 int32_t orc_postprocess_image_ex(const float* head, int32_t A, int32_t C, int32_t logits,
                                  float conf, float iou_thr, int32_t max_det, int32_t w, int32_t h,
-                                 int32_t S, int32_t agnostic, orc_det_t* dets, int32_t* n_cand);
+                                 int32_t S, int32_t agnostic, orc_det_t* dets, int32_t* n_cand) {
+    int32_t map[8];
+    frame_map(w, h, S, map);
+    return postprocess_core(head, A, C, logits, conf, iou_thr, max_det, agnostic, 0, 0, 0, map, dets, n_cand);
+}
+
 int32_t orc_postprocess_image(const float* head, int32_t A, int32_t C, int32_t logits,
                               float conf, float iou_thr, int32_t max_det, int32_t w, int32_t h,
                               int32_t S, orc_det_t* dets, int32_t* n_cand) {
     return orc_postprocess_image_ex(head, A, C, logits, conf, iou_thr, max_det, w, h, S, 0, dets, n_cand);
 }
-int32_t orc_postprocess_image_ex(const float* head, int32_t A, int32_t C, int32_t logits,
-                                 float conf, float iou_thr, int32_t max_det, int32_t w, int32_t h,
-                                 int32_t S, int32_t agnostic, orc_det_t* dets, int32_t* n_cand) {
-    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * (size_t)(A > 0 ? A : 1));
-    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
-    int32_t n = orc_decode(head, A, C, logits, conf, cand);
-    orc_sort(cand, n);
-    int32_t k = orc_nms_ex(cand, n, iou_thr, max_det, agnostic, keep);
-    for (int32_t t = 0; t < k; ++t) {
-        dets[t] = cand[keep[t]];
-        orc_scale_back(&dets[t], w, h, S);
-    }
-    if (n_cand) *n_cand = n;
-    free(cand);
-    free(keep);
-    return k;
-}
 
-/* R3..R6 for one image with the decode variants of orc_decode_ex. */
+/* The same with the decode variants of orc_decode_ex. */
 int32_t orc_postprocess_image_v2(const float* head, int32_t A, int32_t C, int32_t logits, float conf,
                                  float iou_thr, int32_t max_det, int32_t w, int32_t h, int32_t S,
                                  int32_t agnostic, int32_t layout, int32_t multi_label, orc_det_t* dets,
                                  int32_t* n_cand) {
-    const size_t cap = (size_t)(A > 0 ? A : 1) * (size_t)(multi_label ? (C > 0 ? C : 1) : 1);
-    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * cap);
-    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
-    int32_t n = orc_decode_ex(head, A, C, logits, conf, layout, multi_label, cand, (int32_t)cap);
-    orc_sort(cand, n);
-    int32_t k = orc_nms_ex(cand, n, iou_thr, max_det, agnostic, keep);
-    for (int32_t t = 0; t < k; ++t) {
-        dets[t] = cand[keep[t]];
-        orc_scale_back(&dets[t], w, h, S);
-    }
-    if (n_cand) *n_cand = n;
-    free(cand);
-    free(keep);
-    return k;
+    int32_t map[8];
+    frame_map(w, h, S, map);
+    return postprocess_core(head, A, C, logits, conf, iou_thr, max_det, agnostic, 1, layout, multi_label, map, dets,
+                            n_cand);
 }
 
-/* R3..R6 for one item of a chained (second-level) stage.  Its detector input is the upstream
- * crop of the rectangle [ox, ox+rw) x [oy, oy+rh), stretched to S x S (no padding), so the
- * head's boxes live on that S x S grid and map back into the rectangle of the ORIGINAL frame. */
+/* R3..R6 for one item of a chained stage. */
 int32_t orc_postprocess_region(const float* head, int32_t A, int32_t C, int32_t logits, float conf,
                                float iou_thr, int32_t max_det, int32_t S, int32_t ox, int32_t oy,
                                int32_t rw, int32_t rh, orc_det_t* dets, int32_t* n_cand) {
-    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * (size_t)(A > 0 ? A : 1));
-    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
-    int32_t n = orc_decode(head, A, C, logits, conf, cand);
-    orc_sort(cand, n);
-    int32_t k = orc_nms(cand, n, iou_thr, max_det, keep);
-    for (int32_t t = 0; t < k; ++t) {
-        dets[t] = cand[keep[t]];
-        orc_scale_back_region(&dets[t], S, S, 0, 0, ox, oy, rw, rh);
-    }
-    if (n_cand) *n_cand = n;
-    free(cand);
-    free(keep);
-    return k;
+    int32_t map[8];
+    region_map(S, ox, oy, rw, rh, map);
+    return postprocess_core(head, A, C, logits, conf, iou_thr, max_det, 0, 0, 0, 0, map, dets, n_cand);
 }
 
 /* The same for the decode variants of orc_decode_ex (head layout, multi-label candidates). */
@@ -416,20 +418,9 @@ int32_t orc_postprocess_region_v2(const float* head, int32_t A, int32_t C, int32
                                   float iou_thr, int32_t max_det, int32_t S, int32_t ox, int32_t oy,
                                   int32_t rw, int32_t rh, int32_t layout, int32_t multi_label,
                                   orc_det_t* dets, int32_t* n_cand) {
-    const size_t cap = (size_t)(A > 0 ? A : 1) * (size_t)(multi_label ? (C > 0 ? C : 1) : 1);
-    orc_det_t* cand = (orc_det_t*)malloc(sizeof(orc_det_t) * cap);
-    int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_det > 0 ? max_det : 1));
-    int32_t n = orc_decode_ex(head, A, C, logits, conf, layout, multi_label, cand, (int32_t)cap);
-    orc_sort(cand, n);
-    int32_t k = orc_nms(cand, n, iou_thr, max_det, keep);
-    for (int32_t t = 0; t < k; ++t) {
-        dets[t] = cand[keep[t]];
-        orc_scale_back_region(&dets[t], S, S, 0, 0, ox, oy, rw, rh);
-    }
-    if (n_cand) *n_cand = n;
-    free(cand);
-    free(keep);
-    return k;
+    int32_t map[8];
+    region_map(S, ox, oy, rw, rh, map);
+    return postprocess_core(head, A, C, logits, conf, iou_thr, max_det, 0, 1, layout, multi_label, map, dets, n_cand);
 }
 
 /* R7: integer crop rectangle of a frame-space box: rx0 = clamp(floor(X1), 0, w-1),

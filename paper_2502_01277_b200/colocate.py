@@ -126,6 +126,7 @@ def demo(n_pipelines: int = 6, batch: int = 2, cycles: int = 200, streams: int =
 
     out = {"pass_us_alone": pass_us, "placed": placed, "streams_used": len(ex.streams),
            "passes_per_s_colocated": rate(ex), "passes_per_s_one_stream": rate(single), "batch": batch}
+    out["colocation_gain"] = out["passes_per_s_colocated"] / out["passes_per_s_one_stream"]  # > 1: co-location paid
     for st in stages:
         st.close()
     return out

@@ -1,52 +1,72 @@
-// Spatiotemporal placement of model instances on GPU inference streams (host code only).
+// Placement of model instances on GPU inference streams in space and time (host code only; the
+// paper's co-location scheduler, Section III-C, Algorithm 2).
 //
-// The paper's co-location scheduler (Section III-C, Algorithm 2) divides a GPU into concurrently
-// running streams; an execution occupies a portion of a stream (its length is the execution time,
-// its width the share of the GPU's compute it needs), and a stream repeats with a duty cycle.
-// Instances are taken one replica number at a time over all pipelines and their models (so that
-// every pipeline gets its first instance before any gets a second), and each goes to the
-// best-fitting free portion that (1) contains the window the instance needs, (2) leaves the GPU
-// within its memory and utilisation limits and (3) belongs to a stream whose duty cycle is not
-// longer than the pipeline's.  The chosen portion is split and what is left goes back to the
-// free list.
+// What is computed.  A GPU is divided into concurrently running streams; an execution occupies a
+// window of one stream's duty cycle and a share of the GPU's compute; a stream repeats with a duty
+// cycle.  Instances are placed one replica number at a time over all pipelines and their models.
+// Each goes to the stream whose free gap around the instance's window is the tightest, among the
+// streams where (1) the window is free, (2) the GPU stays within its memory (weights + per stream
+// the largest intermediate memory of its residents) and its utilisation limit (per stream the
+// widest resident) and (3) the stream's duty cycle is not longer than the instance's.  Ties go
+// to the lower GPU, then the lower stream.  The first resident of a stream fixes its duty cycle;
+// a stream without one counts as an unbounded gap, so it is taken only when no bounded gap fits.
 //
-// Readings where the paper is silent: the free list is kept ordered by length (then GPU, stream,
-// start), so the first feasible portion is the one with the least empty space; a stream without a
-// duty cycle offers one unbounded portion, which is cut to the duty cycle once the first instance
-// fixes it; all times are integer microseconds.
+// How.  Every stream keeps its busy windows in an ordered map (start -> end), so the free gap
+// around a window is found from the window's two neighbours in O(log residents); a window lies in
+// at most one gap of a stream, hence comparing one candidate per stream finds the tightest gap
+// overall.  A GPU's totals (weights, sum of the streams' intermediate maxima, sum of the streams'
+// widths) are kept up to date, so the limits are tested in O(1) per candidate.
 #include <algorithm>
 #include <cstdint>
+#include <iterator>
+#include <map>
+#include <numeric>
 #include <vector>
 
 #include "octo.h"
 
 namespace {
 
-constexpr int64_t kForever = INT64_MAX;
+constexpr int64_t kUnbounded = INT64_MAX;
 
-struct Portion {
-    int32_t gpu, stream;
-    int64_t start, end;
-    int64_t length() const { return end == kForever ? kForever : end - start; }
+class Stream {
+  public:
+    int64_t duty_cycle() const { return duty_; }
+    int64_t inter() const { return inter_; }
+    int32_t width() const { return width_; }
+
+    // Free gap [lo, hi) around the window [a, b), or false if the window touches a busy one.
+    bool gap_around(int64_t a, int64_t b, int64_t* lo, int64_t* hi) const {
+        auto next = busy_.lower_bound(a);  // first busy window starting at or after a
+        if (next != busy_.end() && next->first < b) return false;
+        *hi = next != busy_.end() ? next->first : (duty_ ? duty_ : kUnbounded);
+        *lo = 0;
+        if (next != busy_.begin()) {
+            auto prev = std::prev(next);
+            if (prev->second > a) return false;
+            *lo = prev->second;
+        }
+        return *hi == kUnbounded || b <= *hi;
+    }
+
+    void occupy(const octo_coral_instance_t& r) {
+        if (!duty_) duty_ = r.duty_cycle_us;
+        busy_.emplace(r.start_us, r.end_us);
+        inter_ = std::max(inter_, r.inter_bytes);
+        width_ = std::max(width_, r.util_permille);
+    }
+
+  private:
+    std::map<int64_t, int64_t> busy_;
+    int64_t duty_ = 0;  // 0: not fixed yet
+    int64_t inter_ = 0;
+    int32_t width_ = 0;
 };
 
-bool portion_less(const Portion& a, const Portion& b) {
-    if (a.length() != b.length()) return a.length() < b.length();
-    if (a.gpu != b.gpu) return a.gpu < b.gpu;
-    if (a.stream != b.stream) return a.stream < b.stream;
-    return a.start < b.start;
-}
-
-struct StreamState {
-    int64_t duty_cycle = 0;  // 0: not fixed yet
-    int64_t inter = 0;       // I_s: largest intermediate memory of its residents
-    int32_t util = 0;        // widest resident
-};
-
-struct GpuState {
-    int64_t weights = 0;  // W_g
-    int64_t inter = 0;    // I_g = sum of I_s
-    std::vector<StreamState> streams;
+struct Gpu {
+    std::vector<Stream> streams;
+    int64_t weights = 0, inter_sum = 0;
+    int32_t width_sum = 0;
 };
 
 }  // namespace
@@ -65,17 +85,12 @@ extern "C" int octo_coral_schedule(const octo_coral_instance_t* inst, int32_t n_
             return OCTO_E_INVALID_ARG;
     }
 
-    std::vector<GpuState> state((size_t)n_gpus);
-    std::vector<Portion> free_list;
-    for (int32_t g = 0; g < n_gpus; ++g) {
-        state[(size_t)g].streams.resize((size_t)gpus[g].num_streams);
-        for (int32_t s = 0; s < gpus[g].num_streams; ++s) free_list.push_back(Portion{g, s, 0, kForever});
-    }
-    std::sort(free_list.begin(), free_list.end(), portion_less);
+    std::vector<Gpu> state((size_t)n_gpus);
+    for (int32_t g = 0; g < n_gpus; ++g) state[(size_t)g].streams.resize((size_t)gpus[g].num_streams);
 
     // one replica number at a time, pipelines in order, models in their pipeline's order
     std::vector<int32_t> order((size_t)n_inst);
-    for (int32_t i = 0; i < n_inst; ++i) order[(size_t)i] = i;
+    std::iota(order.begin(), order.end(), 0);
     std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
         if (inst[a].instance != inst[b].instance) return inst[a].instance < inst[b].instance;
         if (inst[a].pipeline != inst[b].pipeline) return inst[a].pipeline < inst[b].pipeline;
@@ -84,45 +99,34 @@ extern "C" int octo_coral_schedule(const octo_coral_instance_t* inst, int32_t n_
 
     for (int32_t idx : order) {
         const octo_coral_instance_t& r = inst[idx];
-        octo_coral_placement_t& place = out[idx];
-        place.gpu = -1; place.stream = -1; place.start_us = 0; place.end_us = 0; place.duty_cycle_us = 0;
-        for (size_t k = 0; k < free_list.size(); ++k) {
-            const Portion pt = free_list[k];
-            GpuState& g = state[(size_t)pt.gpu];
-            StreamState& s = g.streams[(size_t)pt.stream];
-            // (1) the stream is free for the whole window
-            if (!(pt.start <= r.start_us && pt.end >= r.end_us)) continue;
-            // (2) memory and compute of the GPU with the instance on this stream
-            const int64_t w_g = g.weights + r.weight_bytes;
-            const int64_t i_g = g.inter - s.inter + std::max(s.inter, r.inter_bytes);
-            int64_t u_g = 0;
-            for (size_t q = 0; q < g.streams.size(); ++q)
-                u_g += (&g.streams[q] == &s) ? std::max(s.util, r.util_permille) : g.streams[q].util;
-            if (w_g + i_g > gpus[pt.gpu].mem_bytes || u_g > gpus[pt.gpu].util_max_permille) continue;
-            // (3) the instance may not stretch the stream's duty cycle
-            if (!(r.duty_cycle_us >= s.duty_cycle)) continue;
-
-            free_list.erase(free_list.begin() + (long)k);
-            if (s.duty_cycle == 0) {
-                s.duty_cycle = r.duty_cycle_us;
-                // the stream's unbounded portions now end with its duty cycle
-                for (Portion& f : free_list)
-                    if (f.gpu == pt.gpu && f.stream == pt.stream && f.end == kForever) f.end = s.duty_cycle;
+        int32_t best_g = -1, best_s = -1;
+        int64_t best_len = 0;
+        for (int32_t g = 0; g < n_gpus; ++g) {
+            const Gpu& gs = state[(size_t)g];
+            for (int32_t s = 0; s < (int32_t)gs.streams.size(); ++s) {
+                const Stream& st = gs.streams[(size_t)s];
+                if (st.duty_cycle() > r.duty_cycle_us) continue;  // the instance may not stretch the cycle
+                int64_t lo, hi;
+                if (!st.gap_around(r.start_us, r.end_us, &lo, &hi)) continue;
+                const int64_t mem = gs.weights + r.weight_bytes + gs.inter_sum - st.inter() + std::max(st.inter(), r.inter_bytes);
+                const int64_t width = (int64_t)gs.width_sum - st.width() + std::max(st.width(), r.util_permille);
+                if (mem > gpus[g].mem_bytes || width > gpus[g].util_max_permille) continue;
+                const int64_t len = hi == kUnbounded ? kUnbounded : hi - lo;
+                if (best_g < 0 || len < best_len) { best_g = g; best_s = s; best_len = len; }
             }
-            const int64_t pt_end = pt.end == kForever ? s.duty_cycle : pt.end;
-            place.gpu = pt.gpu; place.stream = pt.stream;
-            place.start_us = r.start_us; place.end_us = r.end_us;
-            place.duty_cycle_us = s.duty_cycle;
-            g.weights = w_g;
-            g.inter = i_g;
-            s.inter = std::max(s.inter, r.inter_bytes);
-            s.util = std::max(s.util, r.util_permille);
-            // what the instance does not use goes back to the list
-            if (pt.start < r.start_us) free_list.push_back(Portion{pt.gpu, pt.stream, pt.start, r.start_us});
-            if (r.end_us < pt_end) free_list.push_back(Portion{pt.gpu, pt.stream, r.end_us, pt_end});
-            std::sort(free_list.begin(), free_list.end(), portion_less);
-            break;
         }
+        octo_coral_placement_t& place = out[idx];
+        place.gpu = best_g; place.stream = best_s;
+        place.start_us = 0; place.end_us = 0; place.duty_cycle_us = 0;
+        if (best_g < 0) continue;
+        Gpu& gs = state[(size_t)best_g];
+        Stream& st = gs.streams[(size_t)best_s];
+        gs.weights += r.weight_bytes;
+        gs.inter_sum += std::max(st.inter(), r.inter_bytes) - st.inter();
+        gs.width_sum += std::max(st.width(), r.util_permille) - st.width();
+        st.occupy(r);
+        place.start_us = r.start_us; place.end_us = r.end_us;
+        place.duty_cycle_us = st.duty_cycle();
     }
     return OCTO_OK;
 }

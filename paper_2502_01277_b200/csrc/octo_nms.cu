@@ -87,7 +87,7 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
     pdl_enter(pdl);
     __shared__ int seg_start[128], seg_cnt[128], cursor[128], nkept[128];
     __shared__ int live[128];  // classes with survivors
-    __shared__ int s_total, s_live, s_big, s_nout;
+    __shared__ int s_total, s_live, s_big, s_nout, s_next;
     unsigned int* const status = &ctr->status;
     (void)status;  // referenced by the range checks of the checked build only
 
@@ -114,6 +114,7 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
         s_total = 0;
         s_live = 0;
         s_big = 0;
+        s_next = 0;
     }
 
     unsigned long long* const gk = gkeys + (size_t)img * key_stride;
@@ -308,8 +309,14 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
             }
         }
 
-        // ---- one warp per class: sort, gather boxes, greedy NMS ----
-        for (int cls = warp; cls < 128; cls += kNmsThreads / 32) {
+        // ---- one warp per class: sort, gather boxes, greedy NMS.  Classes are handed out by a
+        // counter, so a warp that drew small classes takes more of them (with a fixed share, 80
+        // classes on 32 warps leave half the warps with three classes and half with two). ----
+        for (;;) {
+            int cls = 0;
+            if (lane == 0) cls = atomicAdd(&s_next, 1);
+            cls = __shfl_sync(0xffffffffu, cls, 0);
+            if (cls >= 128) break;
             const int m = seg_cnt[cls];
             if (m == 0) continue;
             const int s = seg_start[cls], e = s + m;

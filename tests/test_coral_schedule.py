@@ -1,6 +1,11 @@
-"""Stream / portion placement (the paper's co-location scheduler, Algorithm 2): the oracle against
-hand-worked cases and a validity checker, and the library's host routine against the oracle on
-random problems.  No GPU is involved: the routine makes no CUDA call."""
+"""Stream / portion placement (the paper's co-location scheduler, Section III-C, Algorithm 2).  The
+oracle (an exhaustive search over every stream for every instance) is pinned by hand-worked
+placements and by properties that a replay with separate bookkeeping checks: windows on a stream
+never overlap, a stream has one duty cycle and no resident with a shorter one, no GPU exceeds its
+memory or utilisation at any point of the sequence, every placement took a gap no wider than any
+other feasible gap, and an instance left out had nowhere to go.  The library's routine (interval
+sets and running totals, a different construction) must agree with the oracle on random problems.
+No GPU is involved: the routine makes no CUDA call."""
 import numpy as np
 import pytest
 
@@ -23,15 +28,61 @@ def _lib(instances, gpus):
 
 
 def _check_valid(instances, gpus, placed):
-    """What any correct placement satisfies, whatever the search order."""
+    """Replays the placements in scheduling order with bookkeeping of its own (busy intervals per
+    stream, totals per GPU) and checks every property a correct schedule has."""
+    busy = {}      # (g, s) -> [(start, end)]
+    duty = {}      # (g, s) -> duty cycle
+    inter = {}     # (g, s) -> largest intermediate memory
+    width = {}     # (g, s) -> widest resident
+    weights = [0] * len(gpus)
+
+    def feasible_gaps(r):
+        gaps = []
+        for g, gpu in enumerate(gpus):
+            for s in range(gpu.streams):
+                k = (g, s)
+                if duty.get(k, 0) > r.duty_cycle:
+                    continue
+                if any(a < r.end and r.start < b for a, b in busy.get(k, [])):
+                    continue
+                if k in duty and r.end > duty[k]:
+                    continue
+                mem = weights[g] + r.W + sum(max(v, r.I) if kk == k else v for kk, v in inter.items() if kk[0] == g)
+                util = sum(max(v, r.U) if kk == k else v for kk, v in width.items() if kk[0] == g)
+                if k not in inter:
+                    mem, util = mem + r.I, util + r.U
+                if mem > gpu.M or util > gpu.U_max:
+                    continue
+                lo = max([b for a, b in busy.get(k, []) if b <= r.start], default=0)
+                hi = min([a for a, b in busy.get(k, []) if a >= r.end], default=duty.get(k, float("inf")))
+                gaps.append((hi - lo, g, s))
+        return gaps
+
+    for i in coral.scheduling_order(instances):
+        r, pl = instances[i], placed[i]
+        gaps = feasible_gaps(r)
+        if pl is None:
+            assert not gaps, f"instance {i} was left out although a portion fits: {gaps}"
+            continue
+        g, s, a, b, d = pl
+        assert (a, b) == (r.start, r.end)
+        mine = [t for t in gaps if t[1:] == (g, s)]
+        assert mine, f"instance {i} sits where it does not fit"
+        assert mine[0][0] == min(gaps)[0], "a tighter portion was free"       # best fit
+        assert mine[0] == min(gaps), "ties go to the lower GPU, then stream"  # the stated tie rule
+        k = (g, s)
+        duty.setdefault(k, r.duty_cycle)
+        assert d == duty[k] <= r.duty_cycle and b <= d
+        busy.setdefault(k, []).append((a, b))
+        inter[k] = max(inter.get(k, 0), r.I)
+        width[k] = max(width.get(k, 0), r.U)
+        weights[g] += r.W
+    # the final state once more, from the placements alone
     by_stream = {}
     for r, pl in zip(instances, placed):
-        if pl is None:
-            continue
-        g, s, a, b, duty = pl
-        assert (a, b) == (r.start, r.end) and duty <= r.duty_cycle and b <= duty
-        by_stream.setdefault((g, s), []).append((a, b, duty, r))
-    for (g, s), lst in by_stream.items():
+        if pl is not None:
+            by_stream.setdefault(pl[:2], []).append((pl[2], pl[3], pl[4], r))
+    for lst in by_stream.values():
         lst.sort(key=lambda t: t[0])
         assert len({d for _, _, d, _ in lst}) == 1                     # one duty cycle per stream
         for (a0, b0, _, _), (a1, b1, _, _) in zip(lst, lst[1:]):
@@ -41,6 +92,29 @@ def _check_valid(instances, gpus, placed):
         mem = sum(r.W for _, lst in res for *_, r in lst) + sum(max(r.I for *_, r in lst) for _, lst in res)
         util = sum(max(r.U for *_, r in lst) for _, lst in res)
         assert mem <= gpu.M and util <= gpu.U_max
+
+
+def test_the_checker_rejects_wrong_schedules():
+    """The replay is only worth something if it fails on mistakes: a placement moved to a wider
+    gap, a placement dropped, two overlapping windows."""
+    inst = [_inst(0, 0, 0, 0, 10_000, 50_000), _inst(0, 1, 0, 40_000, 50_000, 50_000),
+            _inst(1, 0, 0, 0, 18_000, 50_000), _inst(1, 1, 0, 30_000, 50_000, 50_000),
+            _inst(2, 0, 0, 19_000, 29_000, 50_000)]
+    gpus = [Gpu(8 << 30, 1000, 2)]
+    good = coral.schedule(inst, gpus)
+    _check_valid(inst, gpus, good)
+    worse = list(good)
+    worse[4] = (0, 0, 19_000, 29_000, 50_000)       # fits on stream 0 too, but in the wider gap
+    with pytest.raises(AssertionError):
+        _check_valid(inst, gpus, worse)
+    dropped = list(good)
+    dropped[4] = None
+    with pytest.raises(AssertionError):
+        _check_valid(inst, gpus, dropped)
+    clash = list(good)
+    clash[2] = (0, 0, 0, 18_000, 50_000)            # overlaps pipeline 0's first window
+    with pytest.raises(AssertionError):
+        _check_valid(inst, gpus, clash)
 
 
 def test_pipeline_models_follow_each_other_on_one_stream():
