@@ -42,14 +42,17 @@ NCU_TRAFFIC = {
     # kernel: (source files, sha256[:16] of their concatenation at capture time, bytes per unit, unit)
     # captured on the sweep workload at B = 64; decode_planes on the anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "a2adfd8f629814cc", 472654.6, "crop"),
+             "38ad77bc69baa998", 481030.0, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                  "ad30360af87ae8e6", 3695876.0, "frame"),
+                  "3ea6f467d75aad28", 3706404.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "2f5c19fd5c24faad", 1699900.0, "frame"),
+               "babeeaad110d66ce", 1745504.0, "frame"),
     "decode_planes": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                      "2f5c19fd5c24faad", 2811836.0, "frame"),
+                      "babeeaad110d66ce", 2816707.0, "frame"),
 }
+# Warp instructions the crop kernel executes per crop (ncu smsp__inst_executed.sum of the same capture):
+# the kernel is bound by instruction issue, so its issue rate is reported beside the byte rates.
+NCU_CROP_WARP_INST = 97447.0
 
 
 def parse_args():
@@ -536,6 +539,19 @@ def run_octo(args):
         "frac_dram": (traffic / (dom_ms * 1e-3) / 1e9 / hbm_peak) if traffic else None,
     }
     if dominant == "crop":
+        # What limits the kernel in practice: instruction issue (ncu: issue slots about 70 % busy, no
+        # memory pipe above 60 %).  Issue rate = executed warp instructions / time against one
+        # instruction per scheduler and clock (4 schedulers per SM) at the clock seen during the run.
+        sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+        mhz = clocks.get("sm_mhz") or peaks.get("sm_max_mhz") or 1965.0
+        inst = NCU_CROP_WARP_INST * units if traffic else None
+        roofline["issue"] = {
+            "limits_the_kernel": True, "warp_inst_per_launch": inst,
+            "achieved_ginst_s": inst / (dom_ms * 1e-3) / 1e9 if inst else None,
+            "peak_ginst_s": sm_count * 4 * mhz * 1e6 / 1e9,
+            "frac": (inst / (dom_ms * 1e-3)) / (sm_count * 4 * mhz * 1e6) if inst else None,
+            "peak_source": f"{sm_count} SMs x 4 schedulers x {mhz:.0f} MHz (clock sampled during the run)",
+        }
         comp = sum(crop_compulsory_bytes(items[b], batch.sizes, *wl.branches[b]) for b in range(len(wl.branches))) \
             / len(wl.branches)
         roofline["compulsory_bytes"] = comp  # output + every covered source byte once per frame
