@@ -603,6 +603,7 @@ def run_octo(args):
         # frames of one shape travel as one pinned block per sub-batch (one copy instead of one per frame)
         h_block = torch.stack(h_frames).pin_memory() if same_shape else None
         d2h = [0]
+        read_crops = [True]  # False: the downstream batches stay on the device, where their model runs
 
         def enqueue(ci):
             lo, hi = chunks[ci]
@@ -637,7 +638,8 @@ def run_octo(args):
             with torch.cuda.stream(ln.stream):
                 for b in range(len(wl.branches)):
                     packed = min(int(ln.h_ni[b][0]), ccap, h_crops[b].shape[0] - cursor[b])
-                    h_crops[b][cursor[b]:cursor[b] + packed].copy_(ln.crops[b][:packed], non_blocking=True)
+                    if read_crops[0]:
+                        h_crops[b][cursor[b]:cursor[b] + packed].copy_(ln.crops[b][:packed], non_blocking=True)
                     cursor[b] += packed
 
         def e2e_step(_i):
@@ -650,15 +652,23 @@ def run_octo(args):
             for ln in lanes:
                 ln.stream.synchronize()
             d2h[0] = (h_dets.numel() + h_counts.numel() * 4 +
-                      sum(cursor[b] * h_crops[b][0].numel() * 2 + (n + len(chunks)) * 4 + 8 * len(chunks)
-                          for b in range(len(wl.branches))))
+                      sum((cursor[b] * h_crops[b][0].numel() * 2 if read_crops[0] else 0) + (n + len(chunks)) * 4 +
+                          8 * len(chunks) for b in range(len(wl.branches))))
 
         for i in range(3):
             e2e_step(i)
         ms_e2e = timed(e2e_steps, e2e_step) / e2e_steps
         e2e = {"value": world * n / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
                "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(d2h[0]),
-               "mode": f"{len(chunks)} sub-batches of <= {c} frames over {len(lanes)} streams"}
+               "mode": f"{len(chunks)} sub-batches of <= {c} frames over {len(lanes)} streams; every result read back, "
+                       "the packed crops included"}
+        # the same with the downstream batches left on the device (where the downstream model would
+        # consume them): inputs in, detections / counts / offsets / item counts out
+        read_crops[0] = False
+        e2e_step(0)
+        ms_keep = timed(e2e_steps, e2e_step) / e2e_steps
+        e2e["crops_stay_on_device"] = {"value": world * n / (ms_keep * 1e-3), "unit": UNIT, "ms_per_step": ms_keep,
+                                       "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(d2h[0])}
         for ln in lanes:
             ln.stage.close()
 
