@@ -5,18 +5,25 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "octo.h"
 #include "octo_kernels.h"
 #include "octo_stage_internal.h"
 
 using namespace octo;
 
-// Records an event pair around one kernel launch while timing is enabled.
+static const char* const kKernelRangeNames[OCTO_K_COUNT] = {"octo::letterbox", "octo::decode", "octo::nms",
+                                                            "octo::assemble", "octo::crop"};
+
+// Brackets one kernel launch: an NVTX range on the host side (a few nanoseconds when no tool
+// listens; profilers show it over the launch) and, while timing is enabled, a CUDA event pair.
 struct ScopedKernelTimer {
     octo_stage* st;
     cudaStream_t stream;
     int slot;
     ScopedKernelTimer(octo_stage* s, int kernel, cudaStream_t str) : st(s), stream(str), slot(-1) {
+        nvtxRangePushA(kKernelRangeNames[kernel]);
         if (!st->timing) return;
         if (st->ev_used >= kEventPairs) { st->ev_dropped += 1; return; }
         slot = st->ev_used++;
@@ -25,6 +32,7 @@ struct ScopedKernelTimer {
     }
     ~ScopedKernelTimer() {
         if (slot >= 0) cudaEventRecord(st->ev[2 * slot + 1], stream);
+        nvtxRangePop();
     }
 };
 

@@ -165,6 +165,79 @@ def test_device_hand_off_equals_the_host_hand_off_and_the_oracle():
         st2.close()
 
 
+def test_three_levels_chained_on_the_device():
+    """frames -> detector -> 128x128 crops -> chained detector -> 64x64 crops -> chained detector:
+    the third stage adopts items of a stage whose own frame table already lives on the device.
+    Boxes of every level are in ORIGINAL-frame pixels and clamped to the rectangle above them."""
+    wl = replace(workloads.WORKLOADS["traffic_1080p"], frame_sizes=((1280, 720),), branches=((128, 128),),
+                 n_raised=40, n_groups=6)
+    b = workloads.make_batch(wl, batch=2, seed=35)
+    s2, s3, c, md2, md3 = 128, 64, 5, 6, 4
+    a2, a3 = workloads.num_anchors(s2), workloads.num_anchors(s3)
+    ref1 = oracle.run_stage(b.frames, b.sizes, b.head, wl.net_size, wl.branches, max_det=wl.max_det,
+                            do_letterbox=False, do_crops=False)
+    n1 = len(ref1.items[0])
+    assert n1 > 8
+    head2 = workloads.make_heads(80, n1, s2, num_classes=c, n_raised=10, n_groups=3)
+    # level 2 in the oracle: detections per upstream item, then its item list
+    d2 = np.zeros((n1, md2), dtype=DET_DTYPE)
+    c2 = np.zeros(n1, dtype=np.int32)
+    for i in range(n1):
+        d, _ = oracle.postprocess_region(head2[i], tuple(int(v) for v in ref1.rects[0][i]), s2, max_det=md2)
+        d2[i, : len(d)] = d
+        c2[i] = len(d)
+    _, its2, (n2, _) = oracle.assemble(d2, c2, md2)
+    assert n2 > n1
+    rects2 = [oracle.crop_rect(d2[i, j], *b.sizes[int(ref1.items[0][i][0])]) for i, j in its2]
+    head3 = workloads.make_heads(81, n2, s3, num_classes=c, n_raised=8, n_groups=2)
+    st1 = octo.Stage(net_size=wl.net_size, max_batch=b.n, num_anchors=wl.num_anchors, num_classes=wl.num_classes,
+                     max_det=wl.max_det, branches=wl.branches)
+    st2 = octo.Stage(net_size=s2, max_batch=n1, num_anchors=a2, num_classes=c, max_det=md2, branches=((s3, s3),))
+    st3 = octo.Stage(net_size=s3, max_batch=n2, num_anchors=a3, num_classes=c, max_det=md3, branches=((32, 32),))
+    try:
+        frames = [torch.from_numpy(f).cuda() for f in b.frames]
+        st1.preprocess(frames, b.sizes)
+        st1.postprocess(torch.from_numpy(b.head).cuda())
+        st1.crop(0, n1 + 4)
+        st2.adopt_items_device(st1, 0, n1)
+        st2.postprocess(torch.from_numpy(head2).cuda())
+        _, _, ni2 = st2.crop(0, n1 * md2)
+        st3.adopt_items_device(st2, 0, n2)
+        dets3, counts3 = st3.postprocess(torch.from_numpy(head3).cuda())
+        buf = torch.full((n2 * md3, 3, 32, 32), 0x7BFF, dtype=torch.int16, device="cuda")
+        _, off3, ni3 = st3.crop(0, n2 * md3, out=buf.view(torch.float16))
+        torch.cuda.synchronize()
+        assert int(ni2[0]) == n2
+        d3, c3 = octo.dets_to_numpy(dets3, counts3)
+        ref_d = np.zeros((n2, md3), dtype=DET_DTYPE)
+        ref_c = np.zeros(n2, dtype=np.int32)
+        for k in range(n2):
+            d, _ = oracle.postprocess_region(head3[k], rects2[k], s3, max_det=md3)
+            ref_d[k, : len(d)] = d
+            ref_c[k] = len(d)
+            rx0, ry0, rx1, ry1 = rects2[k]
+            assert np.all((d["x1"] >= rx0) & (d["x2"] <= rx1) & (d["y1"] >= ry0) & (d["y2"] <= ry1))
+        assert np.array_equal(c3, ref_c) and int(ref_c.sum()) > 0
+        for k in range(n2):
+            assert d3[k, : ref_c[k]].tobytes() == ref_d[k, : ref_c[k]].tobytes(), f"level-2 item {k}"
+        offs, its3, (pk, tot) = oracle.assemble(ref_d, ref_c, md3)
+        assert tuple(int(v) for v in ni3.cpu()) == (pk, tot) and np.array_equal(off3.cpu().numpy(), offs)
+        items3 = st3.item_table(0, pk)
+        got = buf.cpu().numpy().view(np.uint16)
+        for q, (k, j) in enumerate(its3):
+            f = int(ref1.items[0][its2[k][0]][0])  # the original frame two levels up
+            w, h = b.sizes[f]
+            assert (int(items3["rx0"][q]), int(items3["ry0"][q]), int(items3["rx1"][q]),
+                    int(items3["ry1"][q])) == oracle.crop_rect(ref_d[k, j], w, h)
+            assert half_absdiff(got[q], oracle.crop(b.frames[f], w, h, ref_d[k, j], 32, 32)) <= 2e-3
+        for st in (st1, st2, st3):
+            assert st.status() == 0
+    finally:
+        st1.close()
+        st2.close()
+        st3.close()
+
+
 def test_adopt_items_device_argument_errors():
     from paper_2502_01277_b200 import binding as B
     lib = octo.load_library()

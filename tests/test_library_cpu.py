@@ -78,6 +78,14 @@ def test_null_arguments_are_rejected():
     assert lib.octo_postprocess_batch(None, None, 1, None, None, None) == binding.OCTO_E_INVALID_ARG
     assert lib.octo_crop_batch(None, 0, 0, 0, None, None, None, None) == binding.OCTO_E_INVALID_ARG
     assert lib.octo_stage_workspace_bytes(None) == 0
+    assert lib.octo_adopt_regions(None, None, 1, None) == binding.OCTO_E_INVALID_ARG
+    assert lib.octo_adopt_items_device(None, None, 0, 0, 1, None) == binding.OCTO_E_INVALID_ARG
+    assert lib.octo_stage_selftest_wait(None, 10, None) == binding.OCTO_E_INVALID_ARG
+    assert lib.octo_static_status(0, None, None) == binding.OCTO_E_INVALID_ARG
+    assert lib.octo_static_status(-1, None, None) == binding.OCTO_E_INVALID_ARG
+    assert lib.octo_queue_push(None, None, 0, None) == binding.OCTO_E_INVALID_ARG
+    assert lib.octo_queue_pop_due(None, 1, 0, None, None, None, None) == binding.OCTO_E_INVALID_ARG
+    assert lib.octo_strerror(binding.OCTO_E_NO_MEMORY) == b"out of host or device memory"
 
 
 def test_missing_library_fails_loudly(tmp_path):
