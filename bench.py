@@ -46,9 +46,9 @@ NCU_TRAFFIC = {
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
                   "3ea6f467d75aad28", 3706404.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "babeeaad110d66ce", 1745504.0, "frame"),
+               "270f693d995aa1ce", 1741824.0, "frame"),
     "decode_planes": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                      "babeeaad110d66ce", 2816707.0, "frame"),
+                      "270f693d995aa1ce", 2812296.0, "frame"),
 }
 # Warp instructions the crop kernel executes per crop (ncu smsp__inst_executed.sum of the same capture):
 # the kernel is bound by instruction issue, so its issue rate is reported beside the byte rates.

@@ -2,9 +2,9 @@
 //
 // HBM-bound scan.  For logit heads sigma <= 1 makes sigma(obj) > conf a necessary condition
 // for score = fl(sigma(obj) * sigma(cls)) > conf, so the scan reads only the obj value of
-// each 340-byte row (one DRAM sector) and fetches the whole row, coalesced across the warp,
-// for the few anchors that pass.  Probability heads are read densely.  A passing row is
-// reduced by the warp (finite check, first-maximum class), scored in the fixed binary32
+// each 340-byte row (one DRAM sector) and fetches the whole row, 32 bytes at a time by a group
+// of eight lanes (four passing rows per warp in flight together), for the few anchors that pass.  Probability heads are read densely.  A passing row is
+// reduced by eight lanes (finite check, first-maximum class), scored in the fixed binary32
 // sequence and appended to the image's key list with one atomic; the key carries class,
 // inverted score bits and anchor, so later steps need nothing else from this kernel and the
 // nondeterministic append order is erased by the sort.
@@ -58,6 +58,8 @@ decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf
     const float* __restrict__ hbase = head + (size_t)img * (size_t)A * (size_t)row_len;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
+    const int grp = lane >> 3, gl = lane & 7, gbase = lane & 24;  // group of eight lanes, lane in it, its first lane
+    const unsigned gmask = 0xffu << gbase;
     // each warp owns kDecPerThread consecutive groups of 32 anchors
     const int a_warp = blockIdx.x * (kDecThreads * kDecPerThread) + warp * (32 * kDecPerThread);
 
@@ -77,42 +79,60 @@ decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf
             nonfinite_seen |= !fin;
             pass = fin && sigmoid_fixed(obj[u]) > conf;
         }
+        // Passing rows are reduced four at a time, one per group of eight lanes (a row is read in
+        // 32-byte pieces, lane g of a group holds elements g, g + 8, ...): the four row fetches are in
+        // flight together and a row costs a quarter of the warp's instructions.
         unsigned todo = __ballot_sync(0xffffffffu, pass);
         while (todo) {
-            const int src = __ffs(todo) - 1;
-            todo &= todo - 1;
+            unsigned mine = todo;  // this group's row: the grp-th lowest set bit
+            for (int i = 0; i < grp; ++i) mine &= mine - 1;
+            const bool have = mine != 0u;
+            const int src = have ? __ffs(mine) - 1 : 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) todo &= todo - 1;  // the four lowest rows are taken
             const int ra = a_warp + u * 32 + src;
             const float* __restrict__ row = hbase + (size_t)ra * row_len;
-            // the warp reads the row; lane l holds elements l, l+32, l+64, ...
-            constexpr int kRowRegs = (5 + 128 + 31) / 32;
             bool fin = true;
             float best = -INFINITY;
             int best_k = 0x7fffffff;
             float e0 = 0.0f;
+            if (have) {
+                // the row is requested in batches of kPieces 32-byte pieces (48 values per group), so
+                // a row of 85 values takes two round trips and the kernel stays at 32-40 registers
+                // (the obj scan of large batches lives on occupancy)
+                constexpr int kPieces = 6;
+                for (int e00 = 0; e00 < row_len; e00 += 8 * kPieces) {
+                    float v[kPieces];
 #pragma unroll
-            for (int j = 0; j < kRowRegs; ++j) {
-                const int e = lane + 32 * j;
-                if (e < row_len) {
-                    const float v = __ldg(row + e);
-                    if (j == 0) e0 = v;
-                    fin &= finite_f(v);
-                    if (e >= 5 && v > best) { best = v; best_k = e - 5; }
+                    for (int j = 0; j < kPieces; ++j) {
+                        const int e = e00 + gl + 8 * j;
+                        v[j] = e < row_len ? __ldg(row + e) : 0.0f;
+                    }
+                    if (e00 == 0) e0 = v[0];
+#pragma unroll
+                    for (int j = 0; j < kPieces; ++j) {
+                        const int e = e00 + gl + 8 * j;
+                        if (e < row_len) {
+                            fin &= finite_f(v[j]);
+                            if (e >= 5 && v[j] > best) { best = v[j]; best_k = e - 5; }
+                        }
+                    }
                 }
             }
-            fin = __all_sync(0xffffffffu, fin);
-            const float bw = __shfl_sync(0xffffffffu, e0, 2);
-            const float bh = __shfl_sync(0xffffffffu, e0, 3);
-            const float ob = __shfl_sync(0xffffffffu, e0, 4);
-            if (!fin) { nonfinite_seen = true; continue; }
-            if (!(bw > 0.0f && bh > 0.0f)) continue;
+            const unsigned bad = __ballot_sync(0xffffffffu, !fin) & gmask;
+            const float bw = __shfl_sync(0xffffffffu, e0, gbase + 2);
+            const float bh = __shfl_sync(0xffffffffu, e0, gbase + 3);
+            const float ob = __shfl_sync(0xffffffffu, e0, gbase + 4);
+            if (bad) nonfinite_seen = true;
+            const bool ok = have && !bad && bw > 0.0f && bh > 0.0f;
             if (!multi) {
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) {
+                for (int off = 4; off > 0; off >>= 1) {  // first maximum over the group's eight lanes
                     const float ov = __shfl_xor_sync(0xffffffffu, best, off);
-                    const int ok = __shfl_xor_sync(0xffffffffu, best_k, off);
-                    if (ov > best || (ov == best && ok < best_k)) { best = ov; best_k = ok; }
+                    const int ok2 = __shfl_xor_sync(0xffffffffu, best_k, off);
+                    if (ov > best || (ov == best && ok2 < best_k)) { best = ov; best_k = ok2; }
                 }
-                if (lane == 0) {
+                if (ok && gl == 0) {
                     const float score = logits ? __fmul_rn(sigmoid_fixed(ob), sigmoid_fixed(best))
                                                : __fmul_rn(ob, best);
                     if (score > conf) {
@@ -125,23 +145,21 @@ decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf
                 }
             } else {
                 // one candidate per class whose own score passes; the keys of a row go out in
-                // groups of up to 32 with one counter update per group
+                // groups of up to eight with one counter update per group
                 const float so = logits ? sigmoid_fixed(ob) : ob;
-#pragma unroll
-                for (int j = 0; j < kRowRegs; ++j) {
-                    const int e = lane + 32 * j;
+                for (int e0i = 0; e0i < row_len; e0i += 8) {  // the same trip count in every group
+                    const int e = e0i + gl;
                     float score = 0.0f;
                     bool hit = false;
-                    if (e >= 5 && e < row_len) {
+                    if (ok && e >= 5 && e < row_len) {
                         const float v = __ldg(row + e);  // second pass over the row: an L1 hit
                         score = __fmul_rn(so, logits ? sigmoid_fixed(v) : v);
                         hit = score > conf;
                     }
-                    const unsigned hits = __ballot_sync(0xffffffffu, hit);
-                    if (hits == 0u) continue;
+                    const unsigned hits = __ballot_sync(0xffffffffu, hit) & gmask;
                     int base = 0;
-                    if (lane == 0) base = atomicAdd(cand_count + img, __popc(hits));
-                    base = __shfl_sync(0xffffffffu, base, 0);
+                    if (hits != 0u && gl == 0) base = atomicAdd(cand_count + img, __popc(hits));
+                    base = __shfl_sync(0xffffffffu, base, gbase);
                     if (hit) {
                         const int slot = base + __popc(hits & ((1u << lane) - 1u));
                         if (slot < key_stride) keys[(size_t)img * key_stride + slot] = make_key(e - 5, score, ra);
