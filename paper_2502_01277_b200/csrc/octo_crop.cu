@@ -19,9 +19,11 @@
 // vertical scale is below 2) point at the same staged copy, so a pass covers as many output
 // rows as its distinct source rows fit the buffer.
 //
-// Consumers own columns.  A consumer thread keeps one pair of neighbouring output columns
-// (its two tap-table entries live in registers) and walks a run of consecutive output rows of
-// the pass.  The horizontal integer lerp of a staged row (an exact two-way dot product per
+// Consumers own columns.  A consumer thread keeps two pairs of neighbouring output columns, half
+// a tile apart (its four tap-table entries live in registers), and walks a run of consecutive
+// output rows of the pass: the per-row work that does not depend on the column (row record,
+// reuse decision, weights, addresses) is paid once for four pixels, and because the lanes of a
+// warp hold neighbouring pairs in both halves, a warp's taps still fall on neighbouring bytes.  The horizontal integer lerp of a staged row (an exact two-way dot product per
 // channel) is kept in registers and reused by the next output row whenever that row taps the
 // same source row: per output row only the NEW source rows cost a horizontal pass, i.e. about
 // min(2, vertical scale) instead of 2.  The vertical lerp and all scaling are two packed fp32
@@ -44,7 +46,7 @@ constexpr int kCropMaxStride = kCropRowBudget / 2;
 constexpr int kCropTilePx = 5300;
 constexpr int kCropMaxPassRows = 32;   // one producer lane per output row of a pass
 constexpr int kCropCtasPerSm = 3;
-constexpr int kCropConsumerWarps = 8;
+constexpr int kCropConsumerWarps = 7;   // with the producer warp 8 warps: 80 registers a thread at 3 CTAs per SM
 constexpr int kCropConsumers = 32 * kCropConsumerWarps;
 constexpr int kCropTailBands = 4;     // finer tiles for the last crops of a launch
 constexpr int kCropTilesPerCta = 4;  // measured: 4 > 8 > 16 > 1 for small batches; a tile switch costs about 1 us
@@ -57,9 +59,9 @@ struct __align__(16) CropPass {
     int32_t valid;  // 0: no more passes
     int32_t table;  // which tap table the pass uses
     int32_t slot, r0, nr, c0, ncols;
-    uint32_t magic;  // floor(2^32 / pairs) + 1: unit index -> row run by one multiplication
+    uint32_t magic;  // floor(2^32 / units per run) + 1: unit index -> row run by one multiplication
     int32_t run_rows;  // the pass is cut into runs of this many consecutive rows ...
-    int32_t units;     // ... and (run, column pair) units are dealt to the consumer threads
+    int32_t units;     // ... and (run, two column pairs) units are dealt to the consumer threads
     int32_t _pad[2];
 };
 
@@ -197,7 +199,7 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
         int w_c0 = 0, w_ncols = 0, w_r0 = 0;
         int w_seg_lo = 0, w_seg = 0, w_stride = 16, w_cap_slots = 2;
         int w_runs = 1;           // row runs that fit the consumer threads side by side
-        uint32_t w_run_magic = 0, w_pair_magic = 0;  // divisions by w_runs / by the pair count, as multiplications
+        uint32_t w_run_magic = 0, w_unit_magic = 0;  // divisions by w_runs / by the units of a run, as multiplications
         bool w_valid = false, w_new = false;
         // size and offset of the resized rectangle inside the slot: the whole slot unless the
         // branch keeps the aspect ratio
@@ -227,13 +229,13 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
             w_seg = hi - lo;
             w_stride = w_seg + 16;
             w_cap_slots = kCropRowBudget / w_stride;  // >= 2
-            // Work units of a pass: (run of consecutive rows, column pair).  A pass is cut into as
-            // many runs as fit the consumer threads side by side (224 columns: 2 runs x 112
-            // pairs), so that a warp works on one run and its reuse decisions are uniform.
-            const uint32_t pairs = (uint32_t)max(w_ncols >> 1, 1);
-            w_runs = max(1, min(kCropConsumers / (int)pairs, kCropMaxPassRows));
+            // Work units of a pass: (run of consecutive rows, two column pairs half a tile apart).
+            // A pass is cut into as many runs as fit the consumer threads side by side (224
+            // columns: 4 runs x 56 units = the 224 consumer threads).
+            const uint32_t quads = (uint32_t)max(w_ncols >> 2, 1);
+            w_runs = max(1, min(kCropConsumers / (int)quads, kCropMaxPassRows));
             w_run_magic = w_runs > 1 ? 0xffffffffu / (uint32_t)w_runs + 1u : 0u;
-            w_pair_magic = pairs > 1u ? 0xffffffffu / pairs + 1u : 0u;
+            w_unit_magic = quads > 1u ? 0xffffffffu / quads + 1u : 0u;
         };
         // first pass of the next tile, if there is one; every lane resolves the same item
         auto open_tile = [&]() {
@@ -317,7 +319,7 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
             }
             const int full_seg = ((3 * rx1 + 15) & ~15) - ((3 * rx0) & ~15);
             w_tile_cols =
-                (full_seg + 16 > kCropMaxStride) ? max(2, (int)((long long)kCropTilePx * w_nw / w_cw) & ~1) : ow;
+                (full_seg + 16 > kCropMaxStride) ? max(4, (int)((long long)kCropTilePx * w_nw / w_cw) & ~3) : ow;
             w_c0 = 0;
             set_tile();
             w_row_lo = w_band * w_band_rows;
@@ -413,10 +415,10 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
             p.valid = w_valid ? 1 : 0;
             p.table = tb;
             p.slot = w_slot; p.r0 = w_r0; p.nr = nr; p.c0 = w_c0; p.ncols = w_ncols;
-            p.magic = w_pair_magic;
+            p.magic = w_unit_magic;
             // rows per run = ceil(nr / runs); runs that start past the last row stay empty
             p.run_rows = w_runs > 1 ? (int)__umulhi((uint32_t)(nr + w_runs - 1), w_run_magic) : nr;
-            p.units = (w_ncols >> 1) * w_runs;
+            p.units = (w_ncols >> 2) * w_runs;
             p._pad[0] = 0; p._pad[1] = 0;
             // ---- ring slot b: wait until the consumers have finished the pass that used it ----
             if (k >= kCropStages) {
@@ -485,30 +487,45 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
             __half* const t0 = out0 + tile_off;
             __half* const t1 = out1 + tile_off;
             __half* const t2 = out2 + tile_off;
-            // Work units (run of rows, column pair), laid out by the producer.  The warp that takes the
-            // first units rotates from pass to pass: at 224 columns the units fill seven of the eight
-            // warps, and a fixed assignment would leave the same warp, hence the same scheduler of the
-            // SM (a warp's scheduler follows from its index), idle in every pass of every CTA
-            // (0.862 -> 0.815 ms at 7356 crops).  Padding the runs to whole warps instead, so that no
-            // warp holds lanes of two runs, costs more instructions than it saves waiting (0.919).
-            const int pairs = cur.ncols >> 1;
+            // Work units (run of rows, two column pairs), laid out by the producer.  The warp that takes
+            // the first units rotates from pass to pass: when the units do not fill every warp, a fixed
+            // assignment would leave the same warp, hence the same scheduler of the SM (a warp's
+            // scheduler follows from its index), idle in every pass of every CTA.  Padding the runs to
+            // whole warps instead, so that no warp holds lanes of two runs, costs more (shorter runs
+            // reuse fewer rows) than it saves waiting.
+            const int quads = cur.ncols >> 2;
             for (int u = (int)((threadIdx.x + 32u * (uint32_t)k) % (uint32_t)kCropConsumers); u < cur.units;
                  u += kCropConsumers) {
-                const int run = pairs > 1 ? (int)__umulhi((uint32_t)u, cur.magic) : u;
-                const int pair = u - run * pairs;
+                const int run = quads > 1 ? (int)__umulhi((uint32_t)u, cur.magic) : u;
+                const int quad = u - run * quads;
                 const int ra = run * cur.run_rows, rb = min(ra + cur.run_rows, cur.nr);
-                const uint4 ee = lds128(xt + 16u * (uint32_t)pair);  // two XEntry: {off, wts} x 2
-                const uint32_t basea = rows + (ee.x & ~3u), sha = ee.x << 3;
-                const uint32_t baseb = rows + (ee.z & ~3u), shb = ee.z << 3;
-                // horizontal lerps of the current top (T) and bottom (B) tap rows, three channels x two pixels
-                unsigned long long T0 = 0ull, T1 = 0ull, T2 = 0ull, B0 = 0ull, B1 = 0ull, B2 = 0ull;
-                uint32_t o = (uint32_t)(ra * ow + 2 * pair);
+                // the unit's two column pairs lie half a tile apart, so that the lanes of a warp tap
+                // neighbouring source bytes in both (four neighbouring columns per thread would double
+                // the byte span of every load of the warp, and with it its shared-memory wavefronts)
+                const uint4 ea = lds128(xt + 16u * (uint32_t)quad);            // XEntry {off, wts} x 2, first pair
+                const uint4 eb = lds128(xt + 16u * (uint32_t)(quad + quads));  // ... second pair
+                const uint32_t base0 = rows + (ea.x & ~3u), sh0 = ea.x << 3;
+                const uint32_t base1 = rows + (ea.z & ~3u), sh1 = ea.z << 3;
+                const uint32_t base2 = rows + (eb.x & ~3u), sh2 = eb.x << 3;
+                const uint32_t base3 = rows + (eb.z & ~3u), sh3 = eb.z << 3;
+                // horizontal lerps of the current top (T) and bottom (B) tap rows: three channels x
+                // (columns 0, 1), then three channels x (columns 2, 3)
+                unsigned long long T0 = 0ull, T1 = 0ull, T2 = 0ull, T3 = 0ull, T4 = 0ull, T5 = 0ull;
+                unsigned long long B0 = 0ull, B1 = 0ull, B2 = 0ull, B3 = 0ull, B4 = 0ull, B5 = 0ull;
+                uint32_t o = (uint32_t)(ra * ow + 2 * quad);
+                const uint32_t oh2 = 2u * (uint32_t)quads;  // distance to the second pair
                 for (int r = ra; r < rb; ++r, o += (uint32_t)ow) {
                     const uint4 rw = lds128(rinfo + 16u * (uint32_t)r);
                     if (GENERAL && (int)rw.y < 0) {  // canvas row
-                        *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(opts.fill[0], opts.fill[0]);
-                        *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(opts.fill[1], opts.fill[1]);
-                        *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(opts.fill[2], opts.fill[2]);
+                        const uint32_t f0 = pack_half2(opts.fill[0], opts.fill[0]);
+                        const uint32_t f1 = pack_half2(opts.fill[1], opts.fill[1]);
+                        const uint32_t f2 = pack_half2(opts.fill[2], opts.fill[2]);
+                        *reinterpret_cast<uint32_t*>(t0 + o) = f0;
+                        *reinterpret_cast<uint32_t*>(t1 + o) = f1;
+                        *reinterpret_cast<uint32_t*>(t2 + o) = f2;
+                        *reinterpret_cast<uint32_t*>(t0 + o + oh2) = f0;
+                        *reinterpret_cast<uint32_t*>(t1 + o + oh2) = f1;
+                        *reinterpret_cast<uint32_t*>(t2 + o + oh2) = f2;
                         continue;
                     }
                     const uint32_t code = r == ra ? 2u : (rw.y >> 16) & 3u;
@@ -516,43 +533,62 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
 #ifdef OCTO_BOUNDS_CHECK
                     {
                         // every tap reads 12 bytes from its aligned word: both rows must lie in the buffer
-                        const long long lo = (long long)(int)rw.x + (long long)min(ee.x & ~3u, ee.z & ~3u);
-                        const long long hi = (long long)(int)rw.x + (long long)max(ee.x & ~3u, ee.z & ~3u) + step + 12;
+                        const uint32_t omin = min(min(ea.x & ~3u, ea.z & ~3u), min(eb.x & ~3u, eb.z & ~3u));
+                        const uint32_t omax = max(max(ea.x & ~3u, ea.z & ~3u), max(eb.x & ~3u, eb.z & ~3u));
+                        const long long lo = (long long)(int)rw.x + (long long)omin;
+                        const long long hi = (long long)(int)rw.x + (long long)omax + step + 12;
                         if (!OCTO_IN_RANGE(lo >= 0 && hi <= kCropRowBudget && r < kCropMaxPassRows &&
                                            cur.slot >= 0 && cur.slot < max_items && cur.r0 + r < oh &&
-                                           cur.c0 + 2 * pair + 1 < ow, status))
+                                           cur.c0 + 2 * (quad + quads) + 1 < ow, status))
                             continue;
                     }
 #endif
-                    if (code == 2u) hpair(basea + rw.x, sha, ee.y, baseb + rw.x, shb, ee.w, T0, T1, T2);
-                    else if (code == 1u) { T0 = B0; T1 = B1; T2 = B2; }
-                    if (code != 0u && step != 0u)
-                        hpair(basea + rw.x + step, sha, ee.y, baseb + rw.x + step, shb, ee.w, B0, B1, B2);
+                    if (code == 2u) {
+                        hpair(base0 + rw.x, sh0, ea.y, base1 + rw.x, sh1, ea.w, T0, T1, T2);
+                        hpair(base2 + rw.x, sh2, eb.y, base3 + rw.x, sh3, eb.w, T3, T4, T5);
+                    } else if (code == 1u) {
+                        T0 = B0; T1 = B1; T2 = B2; T3 = B3; T4 = B4; T5 = B5;
+                    }
+                    if (code != 0u && step != 0u) {
+                        const uint32_t rb1 = rw.x + step;
+                        hpair(base0 + rb1, sh0, ea.y, base1 + rb1, sh1, ea.w, B0, B1, B2);
+                        hpair(base2 + rb1, sh2, eb.y, base3 + rb1, sh3, eb.w, B3, B4, B5);
+                    }
                     const float wx = __uint_as_float(rw.z), wy = __uint_as_float(rw.w);
                     const unsigned long long wx2 = f32x2(wx, wx), wy2 = f32x2(wy, wy);
                     // fl(fl(v0 * wx) + v1 * wy) per element (B is finite and wy = 0 when the row has one tap row)
                     const unsigned long long p0 = fma_f32x2(B0, wy2, mul_f32x2(T0, wx2));
                     const unsigned long long p1 = fma_f32x2(B1, wy2, mul_f32x2(T1, wx2));
                     const unsigned long long p2 = fma_f32x2(B2, wy2, mul_f32x2(T2, wx2));
+                    const unsigned long long p3 = fma_f32x2(B3, wy2, mul_f32x2(T3, wx2));
+                    const unsigned long long p4 = fma_f32x2(B4, wy2, mul_f32x2(T4, wx2));
+                    const unsigned long long p5 = fma_f32x2(B5, wy2, mul_f32x2(T5, wx2));
                     if (!GENERAL) {
                         *reinterpret_cast<uint32_t*>(t0 + o) = half2_of_f32x2(p0);
                         *reinterpret_cast<uint32_t*>(t1 + o) = half2_of_f32x2(p1);
                         *reinterpret_cast<uint32_t*>(t2 + o) = half2_of_f32x2(p2);
+                        *reinterpret_cast<uint32_t*>(t0 + o + oh2) = half2_of_f32x2(p3);
+                        *reinterpret_cast<uint32_t*>(t1 + o + oh2) = half2_of_f32x2(p4);
+                        *reinterpret_cast<uint32_t*>(t2 + o + oh2) = half2_of_f32x2(p5);
                     } else {
-                        float a0, a1, a2, b0, b1, b2;
-                        unpack_f32x2(p0, a0, b0);
-                        unpack_f32x2(p1, a1, b1);
-                        unpack_f32x2(p2, a2, b2);
-                        // zero weights mark a canvas column
-                        a0 = ee.y ? fmaf(a0, opts.sc[0], opts.of[0]) : opts.fill[0];
-                        a1 = ee.y ? fmaf(a1, opts.sc[1], opts.of[1]) : opts.fill[1];
-                        a2 = ee.y ? fmaf(a2, opts.sc[2], opts.of[2]) : opts.fill[2];
-                        b0 = ee.w ? fmaf(b0, opts.sc[0], opts.of[0]) : opts.fill[0];
-                        b1 = ee.w ? fmaf(b1, opts.sc[1], opts.of[1]) : opts.fill[1];
-                        b2 = ee.w ? fmaf(b2, opts.sc[2], opts.of[2]) : opts.fill[2];
-                        *reinterpret_cast<uint32_t*>(t0 + o) = pack_half2(a0, b0);
-                        *reinterpret_cast<uint32_t*>(t1 + o) = pack_half2(a1, b1);
-                        *reinterpret_cast<uint32_t*>(t2 + o) = pack_half2(a2, b2);
+                        // per-plane scale and offset; zero weights mark a canvas column
+                        auto finish = [&](unsigned long long lo01, unsigned long long hi23, int c) {
+                            float v0, v1, v2, v3;
+                            unpack_f32x2(lo01, v0, v1);
+                            unpack_f32x2(hi23, v2, v3);
+                            v0 = ea.y ? fmaf(v0, opts.sc[c], opts.of[c]) : opts.fill[c];
+                            v1 = ea.w ? fmaf(v1, opts.sc[c], opts.of[c]) : opts.fill[c];
+                            v2 = eb.y ? fmaf(v2, opts.sc[c], opts.of[c]) : opts.fill[c];
+                            v3 = eb.w ? fmaf(v3, opts.sc[c], opts.of[c]) : opts.fill[c];
+                            return make_uint2(pack_half2(v0, v1), pack_half2(v2, v3));
+                        };
+                        const uint2 h0 = finish(p0, p3, 0), h1 = finish(p1, p4, 1), h2 = finish(p2, p5, 2);
+                        *reinterpret_cast<uint32_t*>(t0 + o) = h0.x;
+                        *reinterpret_cast<uint32_t*>(t1 + o) = h1.x;
+                        *reinterpret_cast<uint32_t*>(t2 + o) = h2.x;
+                        *reinterpret_cast<uint32_t*>(t0 + o + oh2) = h0.y;
+                        *reinterpret_cast<uint32_t*>(t1 + o + oh2) = h1.y;
+                        *reinterpret_cast<uint32_t*>(t2 + o + oh2) = h2.y;
                     }
                 }
             }
