@@ -49,6 +49,7 @@ constexpr int kCropCtasPerSm = 3;
 constexpr int kCropConsumerWarps = 7;   // with the producer warp 8 warps: 80 registers a thread at 3 CTAs per SM
 constexpr int kCropConsumers = 32 * kCropConsumerWarps;
 constexpr int kCropTailBands = 4;     // finer tiles for the last crops of a launch
+constexpr int kCropTilesAhead = 2;   // tiles of a CTA that are fixed in advance and resolved side by side
 constexpr int kCropTilesPerCta = 4;  // measured: 4 > 8 > 16 > 1 for small batches; a tile switch costs about 1 us
 constexpr unsigned kCropProducerSleepNs = 200;  // between the producer's polls of an "empty" barrier
 constexpr int kCropKernelThreads = kCropConsumers + 32;  // + one producer warp
@@ -186,11 +187,11 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
         const float inv_dx = 1.0f / (float)(2 * ow), inv_dy = 1.0f / (float)(2 * oh);
         // every scale factor folded into the vertical weights: 1 / (255 * den_x * den_y)
         const float inv_all = 1.0f / (255.0f * (float)(2 * ow) * (float)(2 * oh));
-        // Tiles (index = slot * bands + band) are handed out dynamically: the first tile of a CTA
-        // is blockIdx.x, every further one comes from an atomic counter, so CTAs that drew cheap
-        // crops (small source rectangles) take more of them and the grid finishes together.  The
-        // round trips of a tile's resolution (counter -> detection index -> detection) are hidden
-        // behind the passes that are already staged in the ring.
+        // Tiles (index = slot * bands + band) are handed out dynamically: the first tiles of a CTA
+        // are fixed, every further one comes from an atomic counter, so CTAs that drew cheap crops
+        // (small source rectangles) take more of them and the grid finishes together.  The round
+        // trips of a tile's resolution (counter -> detection index -> detection) are hidden behind
+        // the passes that are already staged in the ring.
         int w_tiles = 0;  // tiles opened so far
         int w_slot = 0, w_band = 0, w_band_rows = band_rows;
         int w_pitch = 0, w_rx0 = 0, w_ry0 = 0, w_cw = 1, w_ch = 1;
@@ -237,69 +238,103 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
             w_run_magic = w_runs > 1 ? 0xffffffffu / (uint32_t)w_runs + 1u : 0u;
             w_unit_magic = quads > 1u ? 0xffffffffu / quads + 1u : 0u;
         };
-        // first pass of the next tile, if there is one; every lane resolves the same item
-        auto open_tile = [&]() {
-            long long tile = blockIdx.x;
-            if (w_tiles > 0) {
-                int t = 0;
-                if (lane == 0) t = atomicAdd(sched, 1);
-                tile = (long long)gridDim.x + (long long)__shfl_sync(0xffffffffu, t, 0);
-            }
-            w_tiles += 1;
-            w_valid = tile < all_tiles;
-            if (!w_valid) return;
+        // A tile resolved: (slot, band) -> item -> detection -> outward-rounded rectangle in its frame.
+        // Three dependent global round trips when the tile number comes from the counter; no warp
+        // collectives inside, so that the lanes may resolve different tiles side by side.
+        struct Tile {
+            int ok, slot, band, band_rows, f, det, rx0, ry0, rx1, ry1, pitch, fh;
+            const uint8_t* data;
+        };
+        auto resolve = [&](long long tile) {
+            Tile t;
+            t.ok = tile < all_tiles ? 1 : 0;
+            t.slot = 0; t.band = 0; t.band_rows = band_rows; t.f = 0; t.det = 0;
+            t.rx0 = 0; t.ry0 = 0; t.rx1 = 1; t.ry1 = 1; t.pitch = 0; t.fh = 1; t.data = nullptr;
+            if (!t.ok) return t;
             if (tile < coarse_tiles) {
-                w_slot = (int)(tile / bands);
-                w_band = (int)(tile - (long long)w_slot * bands);
-                w_band_rows = band_rows;
+                t.slot = (int)(tile / bands);
+                t.band = (int)(tile - (long long)t.slot * bands);
             } else {
                 const long long u = tile - coarse_tiles;
-                w_slot = (packed - tail_crops) + (int)(u / tail_bands);
-                w_band = (int)(u % tail_bands);
-                w_band_rows = tail_rows;
+                t.slot = (packed - tail_crops) + (int)(u / tail_bands);
+                t.band = (int)(u % tail_bands);
+                t.band_rows = tail_rows;
             }
-            int rx0, ry0, rx1, ry1;
             if (QUEUE) {
-                const QRecord rec = qrec[w_slot];
-                w_data = rec.data; w_pitch = rec.pitch;
-                rx0 = rec.rx0; ry0 = rec.ry0; rx1 = rec.rx1; ry1 = rec.ry1;
-#ifdef OCTO_BOUNDS_CHECK
-                w_fh = rec.h;
-#endif
+                const QRecord rec = qrec[t.slot];
+                t.data = rec.data; t.pitch = rec.pitch; t.fh = rec.h;
+                t.rx0 = rec.rx0; t.ry0 = rec.ry0; t.rx1 = rec.rx1; t.ry1 = rec.ry1;
             } else {
-                const int item = first_item + w_slot;
+                const int item = first_item + t.slot;
                 int lo = 0, hi = n;  // largest f with s_off[f] <= item (frames without items are skipped)
                 while (hi - lo > 1) {
                     const int mid = (lo + hi) >> 1;
                     if (s_off[mid] <= item) lo = mid; else hi = mid;
                 }
-                const int f = lo;
-                int det = 0;
-                if (OCTO_IN_RANGE(item - s_off[f] >= 0 && item - s_off[f] < max_det, status))
-                    det = bidx[(size_t)f * max_det + (item - s_off[f])];
-                if (!OCTO_IN_RANGE(det >= 0 && det < max_det, status)) det = 0;
-                const octo_det_t d = dets[(size_t)f * max_det + det];
-                const FrameDesc fd = gtab ? gtab[f] : tab.f[f];
+                t.f = lo;
+                if (OCTO_IN_RANGE(item - s_off[t.f] >= 0 && item - s_off[t.f] < max_det, status))
+                    t.det = bidx[(size_t)t.f * max_det + (item - s_off[t.f])];
+                if (!OCTO_IN_RANGE(t.det >= 0 && t.det < max_det, status)) t.det = 0;
+                const octo_det_t d = dets[(size_t)t.f * max_det + t.det];
+                const FrameDesc fd = gtab ? gtab[t.f] : tab.f[t.f];
                 // outward-rounded rectangle, clamped so that it is never empty
-                rx0 = (int)floorf(d.x1); ry0 = (int)floorf(d.y1);
-                rx1 = (int)ceilf(d.x2); ry1 = (int)ceilf(d.y2);
-                rx0 = min(max(rx0, 0), fd.w - 1);
-                ry0 = min(max(ry0, 0), fd.h - 1);
-                rx1 = min(max(rx1, rx0 + 1), fd.w);
-                ry1 = min(max(ry1, ry0 + 1), fd.h);
-                if (w_band == 0 && lane == 0 && OCTO_IN_RANGE(w_slot >= 0 && w_slot < max_items, status)) {
-                    // the tile of a slot's first band records the item
-                    octo_item_t it;
-                    it.frame = f; it.det = det;
-                    it.rx0 = rx0; it.ry0 = ry0; it.rx1 = rx1; it.ry1 = ry1;
-                    it._pad[0] = 0; it._pad[1] = 0;
-                    items[w_slot] = it;
-                }
-                w_data = fd.data; w_pitch = fd.pitch;
-#ifdef OCTO_BOUNDS_CHECK
-                w_fh = fd.h;
-#endif
+                t.rx0 = (int)floorf(d.x1); t.ry0 = (int)floorf(d.y1);
+                t.rx1 = (int)ceilf(d.x2); t.ry1 = (int)ceilf(d.y2);
+                t.rx0 = min(max(t.rx0, 0), fd.w - 1);
+                t.ry0 = min(max(t.ry0, 0), fd.h - 1);
+                t.rx1 = min(max(t.rx1, t.rx0 + 1), fd.w);
+                t.ry1 = min(max(t.ry1, t.ry0 + 1), fd.h);
+                t.data = fd.data; t.pitch = fd.pitch; t.fh = fd.h;
             }
+            return t;
+        };
+        // The first kCropTilesAhead tiles of a CTA are fixed (block index + j * grid size) and
+        // resolved up front, lane j resolving tile j, so that their round trips overlap: with few
+        // tiles per CTA (small batches) the chain is paid once, not once per tile.
+        const Tile ahead = resolve(lane < kCropTilesAhead ? (long long)blockIdx.x + (long long)lane * (long long)gridDim.x
+                                                          : all_tiles);
+        // first pass of the next tile, if there is one
+        auto open_tile = [&]() {
+            Tile t;
+            if (w_tiles < kCropTilesAhead) {
+                const int src = w_tiles;
+                t.ok = __shfl_sync(0xffffffffu, ahead.ok, src);
+                t.slot = __shfl_sync(0xffffffffu, ahead.slot, src);
+                t.band = __shfl_sync(0xffffffffu, ahead.band, src);
+                t.band_rows = __shfl_sync(0xffffffffu, ahead.band_rows, src);
+                t.f = __shfl_sync(0xffffffffu, ahead.f, src);
+                t.det = __shfl_sync(0xffffffffu, ahead.det, src);
+                t.rx0 = __shfl_sync(0xffffffffu, ahead.rx0, src);
+                t.ry0 = __shfl_sync(0xffffffffu, ahead.ry0, src);
+                t.rx1 = __shfl_sync(0xffffffffu, ahead.rx1, src);
+                t.ry1 = __shfl_sync(0xffffffffu, ahead.ry1, src);
+                t.pitch = __shfl_sync(0xffffffffu, ahead.pitch, src);
+                t.fh = __shfl_sync(0xffffffffu, ahead.fh, src);
+                t.data = reinterpret_cast<const uint8_t*>(
+                    __shfl_sync(0xffffffffu, (unsigned long long)reinterpret_cast<uintptr_t>(ahead.data), src));
+            } else {
+                int c = 0;
+                if (lane == 0) c = atomicAdd(sched, 1);
+                t = resolve((long long)kCropTilesAhead * (long long)gridDim.x +
+                            (long long)__shfl_sync(0xffffffffu, c, 0));
+            }
+            w_tiles += 1;
+            w_valid = t.ok != 0;
+            if (!w_valid) return;
+            w_slot = t.slot; w_band = t.band; w_band_rows = t.band_rows;
+            const int rx0 = t.rx0, ry0 = t.ry0, rx1 = t.rx1, ry1 = t.ry1;
+            if (!QUEUE && w_band == 0 && lane == 0 && OCTO_IN_RANGE(w_slot >= 0 && w_slot < max_items, status)) {
+                // the tile of a slot's first band records the item
+                octo_item_t it;
+                it.frame = t.f; it.det = t.det;
+                it.rx0 = rx0; it.ry0 = ry0; it.rx1 = rx1; it.ry1 = ry1;
+                it._pad[0] = 0; it._pad[1] = 0;
+                items[w_slot] = it;
+            }
+            w_data = t.data; w_pitch = t.pitch;
+#ifdef OCTO_BOUNDS_CHECK
+            w_fh = t.fh;
+#endif
             w_rx0 = rx0; w_ry0 = ry0; w_cw = rx1 - rx0; w_ch = ry1 - ry0;
             if (GENERAL && opts.keep_aspect) {
                 // the side with the larger ratio fills the slot, the other is the exact quotient
