@@ -122,3 +122,11 @@ def test_very_wide_rectangles_under_the_checked_build(checked):
         _compare(res, ref, ((224, 16),))
     finally:
         st.close()
+
+
+@pytest.mark.parametrize("ow,oh", [(24, 40), (136, 40), (456, 40), (904, 20), (2048, 9)])
+def test_output_widths_around_the_unit_layout_under_the_checked_build(checked, ow, oh):
+    """Crop work layouts with an odd number of column units, fewer and more units than consumer
+    threads: the same cases as in the parity module, with every index range-checked."""
+    from test_gpu_parity import test_crop_output_widths_around_the_unit_layout as case
+    case(ow, oh)  # asserts parity and a clean status word (OCTO_STATUS_BOUNDS included)

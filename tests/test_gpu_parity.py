@@ -347,6 +347,37 @@ def test_crop_shapes_and_degenerate_boxes():
             st.close()
 
 
+@pytest.mark.parametrize("ow,oh", [(24, 40), (40, 33), (72, 40), (120, 37), (136, 40), (448, 24), (456, 40),
+                                   (896, 12), (904, 20), (2048, 9)])
+def test_crop_output_widths_around_the_unit_layout(ow, oh):
+    """Output widths at which the crop kernel's work layout changes: an odd number of column units per
+    row, fewer / exactly as many / more units than consumer threads, rows of one pass dealt to 1 .. 32
+    runs; heights that leave a ragged last pass."""
+    import paper_2502_01277_b200 as octo
+    rng = np.random.default_rng(100 + ow)
+    w, h, s = 416, 240, 320
+    img = rng.integers(0, 256, size=(h, (3 * w + 15) // 16 * 16), dtype=np.uint8)
+    C, A = 4, 64
+    head = np.full((1, A, 5 + C), -9.0, dtype=np.float32)
+    nw, nh, pl, pt = oracle.letterbox_geometry(w, h, s)
+    g = w / nw
+    boxes = [(208, 120, 416, 240), (100, 60, 37, 21), (300, 200, 150, 60), (50.3, 40.7, 9, 130), (400, 30, 30, 55)]
+    for k, (cx, cy, bw, bh) in enumerate(boxes):
+        head[0, k, :4] = [cx / g + pl, cy / g + pt, bw / g, bh / g]
+        head[0, k, 4] = 4.0 - 0.1 * k
+        head[0, k, 5 + (k % C)] = 5.0
+    st = octo.Stage(net_size=s, max_batch=1, num_anchors=A, num_classes=C, branches=((ow, oh),))
+    try:
+        res = run_stage_gpu(st, [img], [(w, h)], head)
+        ref = oracle.run_stage([img], [(w, h)], head, s, ((ow, oh),))
+        assert ref.counts[0] == len(boxes)
+        _check_dets(res, ref)
+        _check_branch(res, ref, 0)
+        assert res.status == 0
+    finally:
+        st.close()
+
+
 def test_crop_of_very_wide_rectangles_is_tiled_by_columns():
     """Rectangles wider than one staging buffer (about 4000 source pixels) are processed in
     column tiles; results must not show the seams."""
