@@ -172,12 +172,13 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
     const int bands_req = min(max(bands_want, 1), (oh + 7) >> 3);
     const int band_rows = min(((oh + bands_req - 1) / bands_req + 7) & ~7, oh);
     const int bands = (oh + band_rows - 1) / band_rows;
-    // With whole crops as tiles the grid would end up to one crop apart, so the last crops (one
-    // per CTA) are cut into up to kCropTailBands finer tiles that even the end out.
-    const int tail_req = min(kCropTailBands, (oh + 7) >> 3);
+    // The CTAs would end up to one tile apart, so the last crops (about one tile of the coarse cut
+    // per CTA) are cut finer and even the end out: into kCropTailBands bands where a whole crop is a
+    // tile, into twice as many bands as the others where crops are cut already.
+    const int tail_req = min(bands == 1 ? kCropTailBands : 2 * bands, (oh + 7) >> 3);
     const int tail_rows = min(((oh + tail_req - 1) / tail_req + 7) & ~7, oh);
     const int tail_bands = (oh + tail_rows - 1) / tail_rows;
-    const int tail_crops = (bands == 1 && tail_bands > 1) ? min(packed, (int)gridDim.x) : 0;
+    const int tail_crops = tail_bands > bands ? min(packed, max((int)gridDim.x / bands, 1)) : 0;
     const long long coarse_tiles = (long long)(packed - tail_crops) * bands;
     const long long all_tiles = coarse_tiles + (long long)tail_crops * tail_bands;
     const size_t plane = (size_t)ow * (size_t)oh;
