@@ -425,12 +425,11 @@ crop_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __rest
                 else if (y0 == p_max) { newrows = need2; back = 1; code = p_need2 ? 1u : (need2 ? 3u : 0u); }
                 else { back = 2; code = 0u; }  // y0 == p_max - 1: both rows are staged
             }
-            int incl = newrows;  // inclusive scan: staged rows up to and including this output row
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += t;
-            }
+            // inclusive scan (staged rows up to and including this output row) from two votes: a row
+            // brings 0, 1 or 2 new rows
+            const unsigned upto = 0xffffffffu >> (31 - lane);
+            const int incl = __popc(__ballot_sync(0xffffffffu, newrows & 1) & upto) +
+                             2 * __popc(__ballot_sync(0xffffffffu, newrows >> 1) & upto);
             const int nr = __popc(__ballot_sync(0xffffffffu, cand && incl <= w_cap_slots));  // >= 1 when valid
             const bool in_pass = lane < nr;
             const int slot_top = incl - newrows - back;
