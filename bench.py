@@ -62,6 +62,8 @@ def parse_args():
     p.add_argument("--warmup", type=int, default=5)
     p.add_argument("--workload", default="sweep", choices=sorted(workloads.WORKLOADS) + ["two_level", "queue"])
     p.add_argument("--bz", type=int, default=64, help="downstream batch size of the queue workload")
+    p.add_argument("--nms-cluster", type=int, default=0, choices=[0, 1, 2, 4, 8],
+                   help="CTAs per image of the NMS launches (0: the stage chooses)")
     p.add_argument("--batch", type=int, default=None, help="frames per GPU per step")
     p.add_argument("--impl", default="octo", choices=["octo", "reference"])
     p.add_argument("--e2e-steps", type=int, default=None)
@@ -309,6 +311,7 @@ def run_octo(args):
                        num_classes=wl.num_classes, head_is_logits=wl.logits, conf_thresh=wl.conf_thresh,
                        iou_thresh=wl.iou_thresh, max_det=wl.max_det, branches=wl.branches,
                        head_layout=wl.head_layout, multi_label=wl.multi_label)
+    stage.set_nms_cluster(args.nms_cluster)
     stream = torch.cuda.Stream(dev)
     cap = n * wl.items_per_frame
 
@@ -699,6 +702,7 @@ def run_octo(args):
                 "crops": [list(b) for b in wl.branches], "items_per_step": [t[1] for t in totals],
                 "candidates_per_step": cand_per_step, "parallelism": f"replicas x{world}",
                 "launch": "CUDA graph replay" if args.graph else "stream launches",
+                "nms_ctas_per_image": stage.last_nms_cluster(),
                 "l2": (f"{n_sets} rotating input/output sets, {n_sets * (in_bytes + out_bytes) / 2**20:.0f} MiB working set"
                        if n_sets > 1 else f"one set of {(in_bytes + out_bytes) / 2**20:.0f} MiB per step, larger than L2"),
             },

@@ -377,6 +377,19 @@ OCTO_API int octo_stage_set_timing(octo_stage_t* st, int32_t enable);
  * *times and release them. */
 OCTO_API int octo_stage_kernel_times(octo_stage_t* st, octo_kernel_times_t* times, void* cuda_stream);
 
+/* CTAs per image of the NMS launches (paper Section III-C: a stage is scheduled by its latency,
+ * and a crowded scene served at a small batch leaves most of the GPU idle with one CTA per image).
+ * cluster = 0 (the default): automatic.  The stage gives every image a thread-block cluster of 2,
+ * 4 or 8 CTAs while the batch has at most a half, a quarter or an eighth as many images as the GPU
+ * has SMs and the NMS kernel's latest launches saw an image with more than 1024 candidates (the
+ * kernel reports that through mapped host memory; nothing is copied or synchronised).  cluster =
+ * 1, 2, 4, 8: that size for every launch (clamped to what the device can co-schedule).  Results do
+ * not depend on the size.  OCTO_E_INVALID_ARG for any other value. */
+OCTO_API int octo_stage_set_nms_cluster(octo_stage_t* st, int32_t cluster);
+
+/* Cluster size of the stage's latest NMS launch (0 before the first one, or for a null stage). */
+OCTO_API int32_t octo_stage_last_nms_cluster(const octo_stage_t* st);
+
 /* Bytes of device memory the stage holds. */
 OCTO_API int64_t octo_stage_workspace_bytes(const octo_stage_t* st);
 

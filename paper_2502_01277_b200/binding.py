@@ -51,6 +51,7 @@ EXPORTS = (
     "octo_adopt_regions", "octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop",
     "octo_queue_pop_due", "octo_coral_schedule", "octo_queue_set_options",
     "octo_adopt_items_device", "octo_stage_selftest_wait", "octo_static_status",
+    "octo_stage_set_nms_cluster", "octo_stage_last_nms_cluster",
 )
 
 
@@ -170,6 +171,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_stage_copy_items.restype = ctypes.c_int
     lib.octo_stage_set_timing.argtypes = [vp, i32]
     lib.octo_stage_set_timing.restype = ctypes.c_int
+    lib.octo_stage_set_nms_cluster.argtypes = [vp, i32]
+    lib.octo_stage_set_nms_cluster.restype = ctypes.c_int
+    lib.octo_stage_last_nms_cluster.argtypes = [vp]
+    lib.octo_stage_last_nms_cluster.restype = i32
     lib.octo_stage_kernel_times.argtypes = [vp, ctypes.POINTER(KernelTimes), vp]
     lib.octo_stage_kernel_times.restype = ctypes.c_int
     lib.octo_postprocess_frame_static.argtypes = [i32, vp, i32, i32, i32, ctypes.c_float, ctypes.c_float,
@@ -455,6 +460,15 @@ class Stage:
 
     def stats(self, stream=None) -> dict:
         return octo_stage_get_stats(self.handle, self._stream(stream))
+
+    def set_nms_cluster(self, cluster: int) -> None:
+        """CTAs per image of the NMS launches: 0 automatic, 1 / 2 / 4 / 8 fixed."""
+        rc = load_library().octo_stage_set_nms_cluster(self.handle, int(cluster))
+        if rc != OCTO_OK:
+            raise OctoError(rc, "octo_stage_set_nms_cluster")
+
+    def last_nms_cluster(self) -> int:
+        return int(load_library().octo_stage_last_nms_cluster(self.handle))
 
     def set_timing(self, enable: bool) -> None:
         rc = load_library().octo_stage_set_timing(self.handle, 1 if enable else 0)

@@ -50,6 +50,13 @@ struct NmsArgs {
     int* d_bidx;
     int max_batch;
     StageCounters* d_ctr;
+    // CTAs per image (a thread-block cluster; 1, 2, 4 or 8).  More than one pays off when few
+    // images carry many candidates each.  d_dense_seen (device pointer to two integers the host
+    // can read, or null): the kernel stores launch_seq in [1] and, when an image had many
+    // candidates, in [0]; the caller picks the cluster size of later launches from the two.
+    int cluster;
+    int* d_dense_seen;
+    int launch_seq;
 };
 
 // Branch options of the crop kernel, per INPUT channel c (output plane swap_rb ? 2 - c : c):
@@ -87,7 +94,9 @@ int report_cuda_error(cudaError_t e, const char* what);
 
 // Opt the kernels of every table capacity into the shared memory they need (current device).
 cudaError_t prepare_letterbox();
-cudaError_t prepare_nms();
+// max_cluster (optional): the largest cluster of the NMS kernel (8, 4, 2 or 1) that the current
+// device can co-schedule.
+cudaError_t prepare_nms(int* max_cluster = nullptr);
 cudaError_t prepare_crop();
 
 cudaError_t launch_letterbox(const FrameDesc* frames, int n, void* d_out, int S, int max_w, int pad_value,
@@ -120,6 +129,34 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1u : 0u;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// The same with a thread-block cluster of `cluster` CTAs along x (grid.x is a multiple of it).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                         cudaStream_t stream, bool pdl, int cluster, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    unsigned na = 0;
+    if (cluster > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)cluster;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 

@@ -17,13 +17,23 @@
 // Images with more candidates than fit in shared memory take the same code path with the
 // arrays in a global-memory workspace; classes with more than kWarpSortMax candidates are
 // sorted by the whole CTA.
+//
+// Few images with many candidates each (a crowded scene served at a small batch) leave most SMs
+// idle with one CTA per image, so the kernel can be launched with a thread-block cluster per
+// image: every CTA of the cluster buckets the image's keys for itself, the classes are handed out
+// by one counter in the first CTA's shared memory to the warps of all CTAs, and every finished
+// class is written into the first CTA's arrays through distributed shared memory.  The first CTA
+// alone merges the classes and writes the image's results.
 #include "octo_common.cuh"
 #include <cmath>
+#include <cooperative_groups.h>
 #include <cstring>
 
 #include "octo_kernels.h"
 
 namespace octo {
+
+namespace cg = cooperative_groups;
 
 constexpr int kNmsThreads = 1024;
 constexpr int kNmsSmemCap = 8192;   // candidates handled on chip: 8 B key + 16 B box each
@@ -31,6 +41,8 @@ constexpr int kWarpSortMax = 2048;  // largest class segment a single warp sorts
 constexpr int kRankSortMax = 512;   // up to here the warp sorts by counting instead of a network
 constexpr int kSmallMax = 256;      // images with at most this many candidates take the short path
 constexpr int kSmallWords = kSmallMax / 32;
+constexpr long long kMergeBySortMin = 8192;  // survivors x live classes above which the merge is a sort
+constexpr int kClusterMinCand = 1024;  // an image with more candidates than this makes clusters worth while
 
 __device__ __forceinline__ void cmp_swap(unsigned long long* __restrict__ k, int i, int j) {
     const unsigned long long a = k[i], b = k[j];
@@ -82,7 +94,7 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
            int* __restrict__ counts, int num_branches, int class_agnostic,
            const __grid_constant__ BranchMasks masks,
            int* __restrict__ bcount, int* __restrict__ bidx, int max_batch, StageCounters* __restrict__ ctr,
-           int pdl) {
+           int* __restrict__ dense_seen, int launch_seq, int pdl) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     pdl_enter(pdl);
     __shared__ int seg_start[128], seg_cnt[128], cursor[128], nkept[128];
@@ -91,7 +103,10 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
     unsigned int* const status = &ctr->status;
     (void)status;  // referenced by the range checks of the checked build only
 
-    const int img = blockIdx.x;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned csize = cluster.num_blocks();  // 1 unless the launch gave every image a cluster
+    const unsigned crank = cluster.block_rank();
+    const int img = (int)(blockIdx.x / csize);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // rows layout [A][5 + C] or planes layout [4 + C][A]
     const int nbox = layout == OCTO_HEAD_PLANES ? 4 : 5;
@@ -106,15 +121,23 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
     cnt = min(cnt, key_stride);
     if (gtab && fd.data == nullptr) cnt = 0;
     if (threadIdx.x < 128) { seg_cnt[threadIdx.x] = 0; nkept[threadIdx.x] = 0; }
-    __syncthreads();
     if (threadIdx.x == 0) {
-        cand_count[img] = 0;  // ready for the next batch's decode
-        atomicAdd(&ctr->candidates, (unsigned long long)cnt);
-        atomicMax(&ctr->max_cand, cnt);
         s_total = 0;
         s_live = 0;
         s_big = 0;
         s_next = 0;
+    }
+    // every CTA of the image has read the count, and the first CTA's counters are set, before the
+    // count is cleared and before any CTA touches those counters
+    if (csize > 1) cluster.sync(); else __syncthreads();
+    if (threadIdx.x == 0 && crank == 0) {
+        cand_count[img] = 0;  // ready for the next batch's decode
+        atomicAdd(&ctr->candidates, (unsigned long long)cnt);
+        atomicMax(&ctr->max_cand, cnt);
+        if (dense_seen) {
+            if (img == 0) dense_seen[1] = launch_seq;
+            if (cnt > kClusterMinCand) dense_seen[0] = launch_seq;
+        }
     }
 
     unsigned long long* const gk = gkeys + (size_t)img * key_stride;
@@ -127,8 +150,19 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
     } else {
         boxes = gboxes + (size_t)img * key_stride;
         keys = gk;
-        if (threadIdx.x == 0) atomicOr(&ctr->status, 0x8u);
+        if (threadIdx.x == 0 && crank == 0) atomicOr(&ctr->status, 0x8u);
     }
+    // the short path and the global-memory path are the first CTA's alone (same count, hence the
+    // same decision, in every CTA of the cluster; no cluster barrier follows on those paths)
+    if (crank != 0 && (cnt <= kSmallMax || !on_chip)) return;
+    // where the other CTAs of the cluster put their finished classes: the first CTA's arrays
+    unsigned long long* const keys0 = csize > 1 && on_chip ? cluster.map_shared_rank(keys, 0) : keys;
+    int* const nkept0 = csize > 1 ? cluster.map_shared_rank(nkept, 0) : nkept;
+    int* const live0 = csize > 1 ? cluster.map_shared_rank(live, 0) : live;
+    int* const total0 = csize > 1 ? cluster.map_shared_rank(&s_total, 0) : &s_total;
+    int* const nlive0 = csize > 1 ? cluster.map_shared_rank(&s_live, 0) : &s_live;
+    int* const next0 = csize > 1 ? cluster.map_shared_rank(&s_next, 0) : &s_next;
+    const bool shared_work = csize > 1 && on_chip && cnt > kSmallMax;
 
     // boxes are dead once NMS is done: their memory holds the ordered survivors (and the ranks)
     unsigned long long* const ordered = reinterpret_cast<unsigned long long*>(boxes);
@@ -309,12 +343,16 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
             }
         }
 
+        // The first CTA's bucketing and block-wide sorts are finished before another CTA of the
+        // cluster writes a finished class into its arrays.
+        if (shared_work) cluster.sync();
+
         // ---- one warp per class: sort, gather boxes, greedy NMS.  Classes are handed out by a
         // counter, so a warp that drew small classes takes more of them (with a fixed share, 80
         // classes on 32 warps leave half the warps with three classes and half with two). ----
         for (;;) {
             int cls = 0;
-            if (lane == 0) cls = atomicAdd(&s_next, 1);
+            if (lane == 0) cls = atomicAdd(next0, 1);
             cls = __shfl_sync(0xffffffffu, cls, 0);
             if (cls >= 128) break;
             const int m = seg_cnt[cls];
@@ -359,10 +397,17 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
                 unsigned long long k = kKeySentinel;
                 if (valid) { b = boxes[p]; k = keys[p]; }
                 bool alive = valid;
-                for (int t = 0; t < nk; ++t) {
+                // four survivors per round: the tests of a round are independent of one another, so
+                // their latencies overlap (a lone warp is bound by the dependent chain, not by issue)
+                for (int t = 0; t < nk; t += 4) {
                     if (!__any_sync(0xffffffffu, alive)) break;
-                    const float4 kb = boxes[s + t];
-                    if (alive && iou_above(kb, b, iou_test)) alive = false;
+                    const float4 k0 = boxes[s + t];
+                    const float4 k1 = boxes[s + min(t + 1, nk - 1)];
+                    const float4 k2 = boxes[s + min(t + 2, nk - 1)];
+                    const float4 k3 = boxes[s + min(t + 3, nk - 1)];
+                    const bool hit = iou_above(k0, b, iou_test) | iou_above(k1, b, iou_test) |
+                                     iou_above(k2, b, iou_test) | iou_above(k3, b, iou_test);
+                    if (hit) alive = false;
                 }
                 unsigned rem = __ballot_sync(0xffffffffu, alive);
                 unsigned keptmask = 0;
@@ -391,80 +436,121 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
                 nk += allowed;
             }
             for (int p = s + nk + lane; p < e; p += 32) keys[p] = kKeySentinel;
+            if (crank != 0) {  // hand the finished class to the first CTA
+                __syncwarp();
+                for (int p = s + lane; p < e; p += 32) keys0[p] = keys[p];
+            }
             if (lane == 0 && nk > 0) {
-                nkept[cls] = nk;
-                atomicAdd(&s_total, nk);
-                live[atomicAdd(&s_live, 1)] = cls;
+                nkept0[cls] = nk;
+                atomicAdd(total0, nk);
+                const int q = atomicAdd(nlive0, 1);
+                if (OCTO_IN_RANGE(q >= 0 && q < 128, status)) live0[q] = cls;
             }
         }
-        __syncthreads();
+        if (shared_work) {
+            cluster.sync();  // every class has arrived in the first CTA's arrays
+            if (crank != 0) return;
+        } else {
+            __syncthreads();
+        }
 
         // ---- global score order: merge of the per-class survivor lists by rank ----
         const int nlive = s_live;
-        if (warp == 0) {
-            // exclusive scan of the survivor counts over the live classes -> cursor[q]
-            int run = 0;
-            for (int base = 0; base < nlive; base += 32) {
-                const int q = base + lane;
-                const int v = q < nlive ? nkept[live[q]] : 0;
-                int inc = v;
-    #pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const int t = __shfl_up_sync(0xffffffffu, inc, off);
-                    if (lane >= off) inc += t;
+        if ((long long)s_total * nlive > kMergeBySortMin) {
+            // Many survivors in many classes: the rank merge below costs survivors x classes binary
+            // searches, a sort of the survivors by the whole CTA far less.  Every survivor carries
+            // its global-order key (inverted score | anchor | class); the lists are packed into the
+            // memory of the (dead) boxes and sorted there.
+            if (warp == 0) {
+                // exclusive scan of the survivor counts over the classes -> cursor[cls]
+                int run = 0;
+#pragma unroll
+                for (int base = 0; base < 128; base += 32) {
+                    const int v = nkept[base + lane];
+                    int inc = v;
+#pragma unroll
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const int u = __shfl_up_sync(0xffffffffu, inc, off);
+                        if (lane >= off) inc += u;
+                    }
+                    cursor[base + lane] = run + inc - v;
+                    run += __shfl_sync(0xffffffffu, inc, 31);
                 }
-                if (q < nlive) cursor[q] = run + inc - v;
-                run += __shfl_sync(0xffffffffu, inc, 31);
             }
+            __syncthreads();
+            const int total = s_total;
+            for (int cls = warp; cls < 128; cls += kNmsThreads / 32) {
+                const int m = nkept[cls], from = seg_start[cls], to = cursor[cls];
+                for (int i = lane; i < m; i += 32)
+                    if (OCTO_IN_RANGE(to + i >= 0 && to + i < total && total <= cnt, status)) ordered[to + i] = keys[from + i];
+            }
+            bitonic_range<true>(ordered, total, threadIdx.x, kNmsThreads);
+        } else {
+            if (warp == 0) {
+                // exclusive scan of the survivor counts over the live classes -> cursor[q]
+                int run = 0;
+                for (int base = 0; base < nlive; base += 32) {
+                    const int q = base + lane;
+                    const int v = q < nlive ? nkept[live[q]] : 0;
+                    int inc = v;
+        #pragma unroll
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const int t = __shfl_up_sync(0xffffffffu, inc, off);
+                        if (lane >= off) inc += t;
+                    }
+                    if (q < nlive) cursor[q] = run + inc - v;
+                    run += __shfl_sync(0xffffffffu, inc, 31);
+                }
+            }
+            __syncthreads();
+            // boxes are no longer needed: their memory holds the ordered survivors and the ranks
+            int* const rank = reinterpret_cast<int*>(ordered + min(max_det, cnt));
+            const int total = s_total;
+            // survivor e (dense numbering over the live classes): rank starts as the index in its own list
+            for (int e = threadIdx.x; e < total; e += kNmsThreads) {
+                int lo = 0, hi = nlive;  // live class q with cursor[q] <= e < cursor[q + 1]
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (cursor[mid] <= e) lo = mid; else hi = mid;
+                }
+                rank[e] = e - cursor[lo];
+            }
+            __syncthreads();
+            // every (survivor, other live class) pair adds the number of that class's survivors that
+            // precede the survivor; pairs are independent, so the searches run in parallel
+            // (neighbouring threads take neighbouring survivors against the same class, so the list reads
+            // broadcast and the rank updates hit different addresses)
+            for (int i = threadIdx.x; i < total * nlive; i += kNmsThreads) {
+                const int q = i / total, e = i - q * total;
+                int lo = 0, hi = nlive;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (cursor[mid] <= e) lo = mid; else hi = mid;
+                }
+                if (lo == q) continue;
+                const unsigned long long g = keys[seg_start[live[lo]] + (e - cursor[lo])];
+                const unsigned long long* const list = keys + seg_start[live[q]];
+                int l2 = 0, h2 = nkept[live[q]];
+                while (l2 < h2) {
+                    const int mid = (l2 + h2) >> 1;
+                    if (list[mid] < g) l2 = mid + 1; else h2 = mid;
+                }
+                if (l2 && OCTO_IN_RANGE(e >= 0 && e < total, status)) atomicAdd(&rank[e], l2);
+            }
+            __syncthreads();
+            for (int e = threadIdx.x; e < total; e += kNmsThreads) {
+                const int r = rank[e];
+                if (r >= max_det) continue;
+                int lo = 0, hi = nlive;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (cursor[mid] <= e) lo = mid; else hi = mid;
+                }
+                if (OCTO_IN_RANGE(r >= 0 && r < min(max_det, cnt), status))
+                    ordered[r] = keys[seg_start[live[lo]] + (e - cursor[lo])];
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        // boxes are no longer needed: their memory holds the ordered survivors and the ranks
-        int* const rank = reinterpret_cast<int*>(ordered + min(max_det, cnt));
-        const int total = s_total;
-        // survivor e (dense numbering over the live classes): rank starts as the index in its own list
-        for (int e = threadIdx.x; e < total; e += kNmsThreads) {
-            int lo = 0, hi = nlive;  // live class q with cursor[q] <= e < cursor[q + 1]
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (cursor[mid] <= e) lo = mid; else hi = mid;
-            }
-            rank[e] = e - cursor[lo];
-        }
-        __syncthreads();
-        // every (survivor, other live class) pair adds the number of that class's survivors that
-        // precede the survivor; pairs are independent, so the searches run in parallel
-        // (neighbouring threads take neighbouring survivors against the same class, so the list reads
-        // broadcast and the rank updates hit different addresses)
-        for (int i = threadIdx.x; i < total * nlive; i += kNmsThreads) {
-            const int q = i / total, e = i - q * total;
-            int lo = 0, hi = nlive;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (cursor[mid] <= e) lo = mid; else hi = mid;
-            }
-            if (lo == q) continue;
-            const unsigned long long g = keys[seg_start[live[lo]] + (e - cursor[lo])];
-            const unsigned long long* const list = keys + seg_start[live[q]];
-            int l2 = 0, h2 = nkept[live[q]];
-            while (l2 < h2) {
-                const int mid = (l2 + h2) >> 1;
-                if (list[mid] < g) l2 = mid + 1; else h2 = mid;
-            }
-            if (l2 && OCTO_IN_RANGE(e >= 0 && e < total, status)) atomicAdd(&rank[e], l2);
-        }
-        __syncthreads();
-        for (int e = threadIdx.x; e < total; e += kNmsThreads) {
-            const int r = rank[e];
-            if (r >= max_det) continue;
-            int lo = 0, hi = nlive;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (cursor[mid] <= e) lo = mid; else hi = mid;
-            }
-            if (OCTO_IN_RANGE(r >= 0 && r < min(max_det, cnt), status))
-                ordered[r] = keys[seg_start[live[lo]] + (e - cursor[lo])];
-        }
-        __syncthreads();
         nout = min(s_total, max_det);
     }
 
@@ -528,13 +614,39 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
 
 constexpr size_t kNmsSmemBytes = (size_t)kNmsSmemCap * (sizeof(float4) + sizeof(unsigned long long));
 
-cudaError_t prepare_nms() {
+cudaError_t prepare_nms(int* max_cluster) {
     cudaError_t e;
     e = cudaFuncSetAttribute(nms_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(nms_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(nms_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
+    e = cudaFuncSetAttribute(nms_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
+    if (e != cudaSuccess) return e;
+    if (max_cluster) {
+        // the largest cluster (one CTA per SM: the kernel takes nearly all shared memory of an SM)
+        // of which the device can hold at least one
+        *max_cluster = 1;
+        for (int c = 8; c > 1; c >>= 1) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)c);
+            cfg.blockDim = dim3(kNmsThreads);
+            cfg.dynamicSmemBytes = kNmsSmemBytes;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)c;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int active = 0;
+            if (cudaOccupancyMaxActiveClusters(&active, nms_kernel<8>, &cfg) == cudaSuccess && active > 0) {
+                *max_cluster = c;
+                break;
+            }
+            (void)cudaGetLastError();
+        }
+    }
+    return cudaSuccess;
 }
 
 template <int CAP>
@@ -550,10 +662,12 @@ static cudaError_t launch_cap(const NmsArgs& a, cudaStream_t stream) {
     unsigned int up_bits;
     memcpy(&up_bits, &up, sizeof(up_bits));
     iou_test.tie_up = (up_bits & 1u) == 0u ? 1 : 0;
-    return launch_kernel(nms_kernel<CAP>, dim3(a.n), dim3(kNmsThreads), smem, stream, a.pdl, tab, a.d_tab, a.d_head, a.A,
-                         a.C, a.layout, iou_test, a.max_det, a.key_stride, a.d_keys, a.d_boxes, a.d_cand_count,
-                         reinterpret_cast<octo_det_rec*>(a.d_dets), a.d_counts, a.num_branches, a.class_agnostic,
-                         a.masks, a.d_bcount, a.d_bidx, a.max_batch, a.d_ctr, a.pdl ? 1 : 0);
+    const int cluster = a.cluster == 2 || a.cluster == 4 || a.cluster == 8 ? a.cluster : 1;
+    return launch_kernel_cluster(nms_kernel<CAP>, dim3((unsigned)(a.n * cluster)), dim3(kNmsThreads), smem, stream, a.pdl,
+                                 cluster, tab, a.d_tab, a.d_head, a.A, a.C, a.layout, iou_test, a.max_det, a.key_stride,
+                                 a.d_keys, a.d_boxes, a.d_cand_count, reinterpret_cast<octo_det_rec*>(a.d_dets),
+                                 a.d_counts, a.num_branches, a.class_agnostic, a.masks, a.d_bcount, a.d_bidx,
+                                 a.max_batch, a.d_ctr, a.d_dense_seen, a.launch_seq, a.pdl ? 1 : 0);
 }
 
 cudaError_t launch_nms(const NmsArgs& a, cudaStream_t stream) {

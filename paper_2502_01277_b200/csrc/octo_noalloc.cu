@@ -53,7 +53,7 @@ cudaError_t setup_device(int device, unsigned char** out) {
         cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_scratch);
         if (e != cudaSuccess) return e;
         if (p == nullptr) return cudaErrorInvalidSymbol;
-        e = prepare_nms();
+        e = prepare_nms(nullptr);
         if (e != cudaSuccess) return e;
         g_dev_ptr[device] = p;
         g_ready[device] = true;
@@ -174,6 +174,9 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
     a.d_bidx = d_bidx;
     a.max_batch = 1;
     a.d_ctr = d_ctr;
+    a.cluster = 1;
+    a.d_dense_seen = nullptr;
+    a.launch_seq = 0;
     e = launch_nms(a, stream);
     if (e != cudaSuccess) return report_cuda_error(e, "nms_kernel");
     return OCTO_OK;

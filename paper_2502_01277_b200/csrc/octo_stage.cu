@@ -126,6 +126,7 @@ static void free_all(octo_stage* st) {
     for (int b = 0; b < OCTO_MAX_BRANCHES; ++b) cudaFree(st->d_items[b]);
     cudaFree(st->d_ctr);
     cudaFree(st->d_tab);
+    if (st->h_dense_seen) cudaFreeHost(st->h_dense_seen);
     for (int i = 0; i < 2 * kEventPairs; ++i)
         if (st->ev[i]) cudaEventDestroy(st->ev[i]);
 }
@@ -167,7 +168,16 @@ extern "C" int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** 
     if (e == cudaSuccess) e = dev_alloc(&st->d_ctr, 1, &st->workspace_bytes);
     if (e == cudaSuccess) e = dev_alloc(&st->d_tab, mb, &st->workspace_bytes);
     if (e == cudaSuccess) e = prepare_letterbox();
-    if (e == cudaSuccess) e = prepare_nms();
+    if (e == cudaSuccess) e = prepare_nms(&st->nms_max_cluster);
+    if (e == cudaSuccess) {
+        // two integers the NMS kernel writes and the host reads without a copy
+        e = cudaHostAlloc(reinterpret_cast<void**>(&st->h_dense_seen), 2 * sizeof(int), cudaHostAllocMapped);
+        if (e == cudaSuccess) {
+            st->h_dense_seen[0] = -(1 << 30);  // no image with many candidates seen yet
+            st->h_dense_seen[1] = 0;
+            e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&st->d_dense_seen), st->h_dense_seen, 0);
+        }
+    }
     if (e == cudaSuccess) e = prepare_crop();
     if (e != cudaSuccess) {
         free_all(st);
@@ -438,6 +448,23 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     a.d_bidx = st->d_bidx;
     a.max_batch = c.max_batch;
     a.d_ctr = st->d_ctr;
+    // A cluster of CTAs per image while images with many candidates were seen in the kernel's latest
+    // launches and the batch is too small to fill the GPU with one CTA per image.
+    st->nms_seq += 1;
+    a.cluster = 1;
+    a.d_dense_seen = st->d_dense_seen;
+    a.launch_seq = st->nms_seq;
+    if (st->nms_cluster_mode > 0) {
+        a.cluster = st->nms_cluster_mode < st->nms_max_cluster ? st->nms_cluster_mode : st->nms_max_cluster;
+    } else if (st->h_dense_seen) {
+        const volatile int* seen = st->h_dense_seen;
+        const int last_dense = seen[0], last_run = seen[1];
+        if (last_run - last_dense <= 4) {
+            const int want = n * 8 <= st->sm_count ? 8 : n * 4 <= st->sm_count ? 4 : n * 2 <= st->sm_count ? 2 : 1;
+            a.cluster = want < st->nms_max_cluster ? want : st->nms_max_cluster;
+        }
+    }
+    st->nms_cluster_last = a.cluster;
     cudaError_t e;
     {
         ScopedKernelTimer t(st, OCTO_K_NMS, stream);
@@ -554,6 +581,15 @@ extern "C" int octo_stage_copy_items(octo_stage_t* st, int32_t branch, octo_item
                              cudaMemcpyDeviceToHost));
     return OCTO_OK;
 }
+
+extern "C" int octo_stage_set_nms_cluster(octo_stage_t* st, int32_t cluster) {
+    if (!st) return OCTO_E_INVALID_ARG;
+    if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8) return OCTO_E_INVALID_ARG;
+    st->nms_cluster_mode = cluster;
+    return OCTO_OK;
+}
+
+extern "C" int32_t octo_stage_last_nms_cluster(const octo_stage_t* st) { return st ? st->nms_cluster_last : 0; }
 
 extern "C" int octo_stage_set_timing(octo_stage_t* st, int32_t enable) {
     if (!st) return OCTO_E_INVALID_ARG;
