@@ -381,8 +381,9 @@ OCTO_API int octo_stage_kernel_times(octo_stage_t* st, octo_kernel_times_t* time
  * and a crowded scene served at a small batch leaves most of the GPU idle with one CTA per image).
  * cluster = 0 (the default): automatic.  The stage gives every image a thread-block cluster of 2,
  * 4 or 8 CTAs while the batch has at most a half, a quarter or an eighth as many images as the GPU
- * has SMs and the NMS kernel's latest launches saw an image with more than 1024 candidates (the
- * kernel reports that through mapped host memory; nothing is copied or synchronised).  cluster =
+ * has SMs and one of the stage's latest 64 NMS launches is known to have seen an image with more
+ * than 1024 candidates (the kernel reports that through mapped host memory; nothing is copied or
+ * synchronised, so the report of a launch may arrive a few calls late).  cluster =
  * 1, 2, 4, 8: that size for every launch (clamped to what the device can co-schedule).  Results do
  * not depend on the size.  OCTO_E_INVALID_ARG for any other value. */
 OCTO_API int octo_stage_set_nms_cluster(octo_stage_t* st, int32_t cluster);

@@ -51,9 +51,9 @@ struct NmsArgs {
     int max_batch;
     StageCounters* d_ctr;
     // CTAs per image (a thread-block cluster; 1, 2, 4 or 8).  More than one pays off when few
-    // images carry many candidates each.  d_dense_seen (device pointer to two integers the host
-    // can read, or null): the kernel stores launch_seq in [1] and, when an image had many
-    // candidates, in [0]; the caller picks the cluster size of later launches from the two.
+    // images carry many candidates each.  d_dense_seen (device pointer to an integer the host can
+    // read, or null): the kernel stores launch_seq there when an image had many candidates; the
+    // caller picks the cluster size of later launches from it.
     int cluster;
     int* d_dense_seen;
     int launch_seq;

@@ -134,10 +134,9 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
         cand_count[img] = 0;  // ready for the next batch's decode
         atomicAdd(&ctr->candidates, (unsigned long long)cnt);
         atomicMax(&ctr->max_cand, cnt);
-        if (dense_seen) {
-            if (img == 0) dense_seen[1] = launch_seq;
-            if (cnt > kClusterMinCand) dense_seen[0] = launch_seq;
-        }
+        // (only crowded images write: a store to host memory delays the end of the kernel by a PCIe
+        // round trip, which a sparse launch of ten microseconds would feel)
+        if (dense_seen && cnt > kClusterMinCand) *dense_seen = launch_seq;
     }
 
     unsigned long long* const gk = gkeys + (size_t)img * key_stride;

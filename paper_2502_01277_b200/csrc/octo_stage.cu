@@ -170,11 +170,10 @@ extern "C" int octo_stage_create(const octo_stage_config_t* cfg, octo_stage_t** 
     if (e == cudaSuccess) e = prepare_letterbox();
     if (e == cudaSuccess) e = prepare_nms(&st->nms_max_cluster);
     if (e == cudaSuccess) {
-        // two integers the NMS kernel writes and the host reads without a copy
-        e = cudaHostAlloc(reinterpret_cast<void**>(&st->h_dense_seen), 2 * sizeof(int), cudaHostAllocMapped);
+        // an integer the NMS kernel writes and the host reads without a copy
+        e = cudaHostAlloc(reinterpret_cast<void**>(&st->h_dense_seen), sizeof(int), cudaHostAllocMapped);
         if (e == cudaSuccess) {
             st->h_dense_seen[0] = -(1 << 30);  // no image with many candidates seen yet
-            st->h_dense_seen[1] = 0;
             e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&st->d_dense_seen), st->h_dense_seen, 0);
         }
     }
@@ -457,9 +456,8 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     if (st->nms_cluster_mode > 0) {
         a.cluster = st->nms_cluster_mode < st->nms_max_cluster ? st->nms_cluster_mode : st->nms_max_cluster;
     } else if (st->h_dense_seen) {
-        const volatile int* seen = st->h_dense_seen;
-        const int last_dense = seen[0], last_run = seen[1];
-        if (last_run - last_dense <= 4) {
+        const int last_dense = *static_cast<const volatile int*>(st->h_dense_seen);
+        if (st->nms_seq - last_dense <= kNmsClusterWindow) {
             const int want = n * 8 <= st->sm_count ? 8 : n * 4 <= st->sm_count ? 4 : n * 2 <= st->sm_count ? 2 : 1;
             a.cluster = want < st->nms_max_cluster ? want : st->nms_max_cluster;
         }

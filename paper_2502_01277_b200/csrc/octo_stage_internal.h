@@ -5,6 +5,7 @@
 #include "octo_kernels.h"
 
 constexpr int kEventPairs = 2048;
+constexpr int kNmsClusterWindow = 64;  // NMS launches that keep forming clusters after a crowded image was reported
 
 struct octo_stage {
     octo_stage_config_t cfg;
@@ -29,16 +30,16 @@ struct octo_stage {
     const octo_det_t* d_dets;
     const int32_t* d_last_n_items[OCTO_MAX_BRANCHES];  // {packed, total} of the last crop call per branch (caller's buffer)
     int64_t launches;
-    // Cluster size of the NMS launches.  The kernel reports through two integers in mapped host
-    // memory (no copy, no synchronisation) the number of its latest launch [1] and of the latest
-    // launch that saw an image with many candidates [0]; while the two are close, launches with few
-    // images give every image a cluster of CTAs.
+    // Cluster size of the NMS launches.  The kernel reports through an integer in mapped host memory
+    // (no copy, no synchronisation) the number of the latest launch that saw an image with many
+    // candidates; for kNmsClusterWindow launches after it (the host may have enqueued many launches
+    // that the GPU has not run yet), launches with few images give every image a cluster of CTAs.
     int nms_max_cluster;
     int nms_cluster_mode;  // 0 automatic, else the caller's size
     int nms_cluster_last;  // size of the latest launch
     int nms_seq;
     int* h_dense_seen;  // host view (volatile reads)
-    int* d_dense_seen;  // device view of the same two integers
+    int* d_dense_seen;  // device view of the same integer
     // optional per-kernel timing
     bool timing;
     cudaEvent_t ev[2 * kEventPairs];
