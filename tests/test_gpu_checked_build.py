@@ -130,3 +130,23 @@ def test_output_widths_around_the_unit_layout_under_the_checked_build(checked, o
     threads: the same cases as in the parity module, with every index range-checked."""
     from test_gpu_parity import test_crop_output_widths_around_the_unit_layout as case
     case(ow, oh)  # asserts parity and a clean status word (OCTO_STATUS_BOUNDS included)
+
+
+@pytest.mark.parametrize("cluster", [1, 4])
+def test_crowded_image_under_the_checked_build(checked, cluster):
+    """General NMS path with the sorted merge, alone and on a cluster of CTAs (finished classes written
+    into the first CTA's shared memory), with every index range-checked."""
+    from test_gpu_nms_cluster import _batch, _oracle_dets
+    from test_gpu_parity import _check_dets
+    from gpu_harness import make_stage, run_stage_gpu
+    b = _batch(5000, 250, 2, max_det=1000)
+    st = make_stage(b.workload, b.n)
+    try:
+        st.set_nms_cluster(cluster)
+        ref = _oracle_dets(b)
+        res = run_stage_gpu(st, b.frames, b.sizes, b.head, max_items=[8])
+        assert st.last_nms_cluster() == cluster
+        assert res.status & B.OCTO_STATUS_BOUNDS == 0, "an index left its range"
+        _check_dets(res, ref)
+    finally:
+        st.close()
