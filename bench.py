@@ -15,6 +15,7 @@ from __future__ import annotations
 
 import argparse
 import hashlib
+import re
 import json
 import os
 import statistics
@@ -39,16 +40,16 @@ UNIT = "frames/s"
 # source the capture was taken from.  An entry whose hash no longer matches the source is
 # reported as null.
 NCU_TRAFFIC = {
-    # kernel: (source files, sha256[:16] of their concatenation at capture time, bytes per unit, unit)
+    # kernel: (source files, sha256[:16] of their code (comments and layout stripped) at capture time, bytes per unit, unit)
     # captured on the sweep workload at B = 64; decode_planes on the anchor_free workload at B = 64
     "crop": (("paper_2502_01277_b200/csrc/octo_crop.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-             "70db07fbfcff14fd", 487791.2, "crop"),
+             "cb3b58cf225f647f", 487791.2, "crop"),
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                  "3ea6f467d75aad28", 3706404.0, "frame"),
+                  "82ba43ca31895b9a", 3706404.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "270f693d995aa1ce", 1741824.0, "frame"),
+               "47f0eeeadf72fd19", 1741824.0, "frame"),
     "decode_planes": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                      "270f693d995aa1ce", 2812296.0, "frame"),
+                      "47f0eeeadf72fd19", 2812296.0, "frame"),
 }
 # Warp instructions the crop kernel executes per crop (ncu smsp__inst_executed.sum of the same capture):
 # the kernel is bound by instruction issue, so its issue rate is reported beside the byte rates.
@@ -143,10 +144,20 @@ def decode_bytes(n: int, a: int, c: int, candidates: int, logits: bool, layout: 
     return int(scan + candidates * (row + 8))
 
 
+def code_only(text: str) -> str:
+    """A CUDA source without its comments and without whitespace: what the compiler sees of it, up to
+    tokens.  (String literals of these sources contain neither comment markers nor blanks that matter.)"""
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"//[^\n]*", "", text)
+    return re.sub(r"\s+", "", text)
+
+
 def files_hash(paths) -> str:
+    """Hash of the code of the given sources (comments and layout do not count: editing a comment does
+    not invalidate counters that were taken from the same kernel)."""
     h = hashlib.sha256()
     for p in paths:
-        h.update(open(os.path.join(ROOT, p), "rb").read())
+        h.update(code_only(open(os.path.join(ROOT, p), "r", encoding="utf-8").read()).encode())
     return h.hexdigest()[:16]
 
 

@@ -9,9 +9,9 @@
 //
 // Crop-resize: bound by instruction issue and shared-memory wavefronts, then HBM (the fp16
 // output is as large as the source rectangles).  A persistent grid works through (slot, row
-// band) tiles that an atomic counter hands out (whole crops, except that the last crops of a
-// launch are cut into bands so that the grid ends together), so no host synchronisation sits
-// between NMS and cropping.  Inside a CTA one producer warp walks its tiles: it resolves the
+// band) tiles (whole crops where there are many; the last crops of a launch are cut finer so
+// that the grid ends together).  A CTA's first two tiles are fixed, the others come from an
+// atomic counter, so no host synchronisation sits between NMS and cropping.  Inside a CTA one producer warp walks its tiles: it resolves the
 // item, builds the table of horizontal taps (byte offset + exact integer weights per output
 // column) and has the bulk-copy engine stage the source rows a pass taps into one of two
 // shared-memory buffers (mbarrier "full" / "empty" ring, every wait bounded).  Every tapped
@@ -23,12 +23,13 @@
 // a tile apart (its four tap-table entries live in registers), and walks a run of consecutive
 // output rows of the pass: the per-row work that does not depend on the column (row record,
 // reuse decision, weights, addresses) is paid once for four pixels, and because the lanes of a
-// warp hold neighbouring pairs in both halves, a warp's taps still fall on neighbouring bytes.  The horizontal integer lerp of a staged row (an exact two-way dot product per
-// channel) is kept in registers and reused by the next output row whenever that row taps the
-// same source row: per output row only the NEW source rows cost a horizontal pass, i.e. about
-// min(2, vertical scale) instead of 2.  The vertical lerp and all scaling are two packed fp32
-// operations per channel, and a warp writes 128 contiguous bytes per plane and row straight
-// into the downstream slot.
+// warp hold neighbouring pairs in both halves, a warp's taps still fall on neighbouring bytes.
+// The horizontal integer lerp of a staged row (an exact two-way dot product per channel) is
+// kept in registers and reused by the next output row whenever that row taps the same source
+// row: per output row only the NEW source rows cost a horizontal pass, i.e. about min(2,
+// vertical scale) instead of 2.  The vertical lerp and all scaling are two packed fp32
+// operations per channel, and a warp writes 128 contiguous bytes per plane, row and pair
+// straight into the downstream slot.
 #include "octo_common.cuh"
 #include <cstring>
 
