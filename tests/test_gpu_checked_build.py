@@ -78,11 +78,11 @@ def test_global_memory_nms_path_under_the_checked_build(checked):
         st.close()
 
 
-@pytest.mark.parametrize("seed", range(0, 64, 4))
-def test_random_configurations_under_the_checked_build(checked, seed):
+@pytest.mark.parametrize("seed,large", [(s, False) for s in range(0, 64, 4)] + [(s, True) for s in (1, 5, 7)])
+def test_random_configurations_under_the_checked_build(checked, seed, large):
     from test_gpu_fuzz import _case
     from gpu_harness import make_stage, run_stage_gpu
-    b, frames, sizes, cfg = _case(seed)
+    b, frames, sizes, cfg = _case(seed, large=large)
     wl = b.workload
     st = make_stage(wl, b.n, **cfg)
     try:

@@ -15,10 +15,12 @@ from test_gpu_parity import PIX_TOL, _check_dets
 pytestmark = pytest.mark.gpu
 
 
-def _case(seed):
-    rng = np.random.default_rng(1000 + seed)
-    s = int(rng.choice([64, 96, 160, 320, 640]))
-    n = int(rng.integers(1, 5))
+def _case(seed, large=False):
+    """large: frames up to 4K, crops up to 512 x 512 and hundreds of detections, so that the crop
+    kernel runs many passes per crop, cuts crops into row bands and ends on its finer tail tiles."""
+    rng = np.random.default_rng((5000 if large else 1000) + seed)
+    s = int(rng.choice([320, 640])) if large else int(rng.choice([64, 96, 160, 320, 640]))
+    n = int(rng.integers(1, 7)) if large else int(rng.integers(1, 5))
     layout = "planes" if rng.random() < 0.4 else "rows"
     logits = bool(rng.random() < 0.7)
     multi = bool(rng.random() < 0.3)
@@ -26,7 +28,10 @@ def _case(seed):
     nb = int(rng.integers(1, 4))
     branches, opts, masks = [], [], []
     for _ in range(nb):
-        branches.append((8 * int(rng.integers(1, 9)), int(rng.integers(1, 70))))
+        if large:
+            branches.append((8 * int(rng.integers(8, 65)), int(rng.integers(32, 513))))
+        else:
+            branches.append((8 * int(rng.integers(1, 9)), int(rng.integers(1, 70))))
         o = {}
         if rng.random() < 0.4:
             o["keep_aspect"] = True
@@ -39,14 +44,17 @@ def _case(seed):
     sizes = []
     for _ in range(n):
         kind = rng.random()
-        if kind < 0.2:
+        if large:
+            sizes.append((int(rng.integers(640, 3841)), int(rng.integers(360, 2161))))
+        elif kind < 0.2:
             sizes.append((int(rng.integers(1, 8)), int(rng.integers(40, 300))))      # sliver
         elif kind < 0.4:
             sizes.append((int(rng.integers(300, 900)), int(rng.integers(1, 12))))    # strip
         else:
             sizes.append((int(rng.integers(8, 700)), int(rng.integers(8, 500))))
     wl = replace(workloads.WORKLOADS["anchor_free" if layout == "planes" else "traffic_1080p"], net_size=s,
-                 n_raised=int(rng.integers(0, 60)), n_groups=int(rng.integers(1, 12)), size_range=(0.05 * s, 0.5 * s),
+                 n_raised=int(rng.integers(100, 400)) if large else int(rng.integers(0, 60)),
+                 n_groups=int(rng.integers(10, 60)) if large else int(rng.integers(1, 12)), size_range=(0.05 * s, 0.5 * s),
                  box_rows=(0.0, float(s)), logits=logits, multi_label=multi, max_det=int(rng.choice([3, 20, 300])),
                  branches=tuple(branches), conf_thresh=float(rng.choice([0.25, 0.5])),
                  iou_thresh=float(rng.choice([0.3, 0.45, 0.6])))
@@ -64,7 +72,15 @@ def _case(seed):
 
 @pytest.mark.parametrize("seed", range(64))
 def test_random_configuration(seed):
-    b, frames, sizes, cfg = _case(seed)
+    _run_case(*_case(seed))
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_configuration_with_large_frames_and_crops(seed):
+    _run_case(*_case(seed, large=True))
+
+
+def _run_case(b, frames, sizes, cfg):
     wl = b.workload
     st = make_stage(wl, b.n, **cfg)
     try:
