@@ -228,3 +228,35 @@ def test_a_wait_that_runs_out_is_reported_and_cleared(stage):
     assert stage.status() == 0 and out.shape == (1, 3, 64, 64)
     assert lib.octo_stage_selftest_wait(stage.handle, 0, None) == B.OCTO_E_INVALID_ARG
     assert lib.octo_stage_selftest_wait(None, 10, None) == B.OCTO_E_INVALID_ARG
+
+
+def test_kernel_timing_counts_every_launch_and_resets(stage):
+    """octo_stage_set_timing / octo_stage_kernel_times: with timing on, every kernel launch of the
+    batch calls is bracketed by an event pair; the getter sums them per kernel, synchronises, and
+    starts from zero again.  With timing off nothing is recorded."""
+    f = _frame()
+    head = torch.zeros((1, 252, 9), dtype=torch.float32, device="cuda")
+
+    def one_pass():
+        stage.preprocess([f], [(40, 30)])
+        stage.postprocess(head)
+        stage.crop(0, 4)
+
+    one_pass()  # untimed
+    t = stage.kernel_times()
+    assert all(t[k] == (0.0, 0) for k in B.KERNEL_NAMES) and t["dropped"] == 0
+    stage.set_timing(True)
+    before = stage.launch_count
+    for _ in range(3):
+        one_pass()
+    t = stage.kernel_times()
+    launched = {k: v[1] for k, v in t.items() if k != "dropped" and v[1]}
+    assert launched == {"letterbox": 3, "decode": 3, "nms": 3, "crop": 3}
+    assert sum(launched.values()) == stage.launch_count - before
+    assert all(0.0 < t[k][0] < 50.0 for k in launched) and t["dropped"] == 0
+    t = stage.kernel_times()  # the getter reset the record
+    assert all(t[k] == (0.0, 0) for k in B.KERNEL_NAMES)
+    stage.set_timing(False)
+    one_pass()
+    t = stage.kernel_times()
+    assert all(t[k] == (0.0, 0) for k in B.KERNEL_NAMES)
