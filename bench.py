@@ -72,6 +72,9 @@ def parse_args():
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--interleave", action="store_true",
                    help="also time two stage instances interleaved on two streams (extra JSON field)")
+    p.add_argument("--fork-preprocess", action="store_true",
+                   help="enqueue the letterbox of a step on a second stream, beside decode / NMS / crop of the "
+                        "same batch (they share no data); joins the main stream at the end of the step")
     p.add_argument("--graph", action="store_true",
                    help="replay each step from a captured CUDA graph (small batches are launch-bound)")
     return p.parse_args()
@@ -353,11 +356,25 @@ def run_octo(args):
             sets.append(z)
     stream.synchronize()
 
+    side = torch.cuda.Stream(device=dev) if args.fork_preprocess else None
+    ev_fork = torch.cuda.Event() if side is not None else None
+    ev_join = torch.cuda.Event() if side is not None else None
+
     def step(z):
-        stage.preprocess_array(z.desc, n, z.det_in, stream=stream, keepalive=z.frames)
+        if side is not None:
+            # the letterbox reads the frames and writes the detector batch; decode, NMS and crop read the
+            # head and the frames: nothing of one is an input of the other within a batch
+            ev_fork.record(stream)
+            side.wait_event(ev_fork)
+            stage.preprocess_array(z.desc, n, z.det_in, stream=side, keepalive=z.frames)
+        else:
+            stage.preprocess_array(z.desc, n, z.det_in, stream=stream, keepalive=z.frames)
         stage.postprocess(z.head, dets=z.dets, counts=z.counts, stream=stream)
         for b in range(len(wl.branches)):
             stage.crop(b, cap, out=z.crops[b], offsets=z.offsets[b], n_items=z.n_items[b], stream=stream)
+        if side is not None:
+            ev_join.record(side)
+            stream.wait_event(ev_join)
 
     def barrier():
         if world > 1:
@@ -712,7 +729,8 @@ def run_octo(args):
                 "net_size": s, "head": list(batch.head.shape),
                 "crops": [list(b) for b in wl.branches], "items_per_step": [t[1] for t in totals],
                 "candidates_per_step": cand_per_step, "parallelism": f"replicas x{world}",
-                "launch": "CUDA graph replay" if args.graph else "stream launches",
+                "launch": ("CUDA graph replay" if args.graph else "stream launches")
+                + (", letterbox on a second stream" if args.fork_preprocess else ""),
                 "nms_ctas_per_image": stage.last_nms_cluster(),
                 "l2": (f"{n_sets} rotating input/output sets, {n_sets * (in_bytes + out_bytes) / 2**20:.0f} MiB working set"
                        if n_sets > 1 else f"one set of {(in_bytes + out_bytes) / 2**20:.0f} MiB per step, larger than L2"),

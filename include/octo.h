@@ -25,7 +25,12 @@
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).  The three
  *     batch calls only enqueue work on it and return; they never synchronise.
  *   - A stage (or queue) object is not re-entrant: use it from one host thread and one stream
- *     at a time.  Different objects are independent: the library keeps no state outside them
+ *     at a time.  One exception: the kernel of octo_preprocess_batch shares no device data with
+ *     the kernels of octo_postprocess_batch and octo_crop_batch of the same batch (it reads the
+ *     frames and writes the detector input; they read the head and the frames; the status word
+ *     is updated atomically), so the call may be given a second stream and its kernel runs beside
+ *     theirs.  The host calls still come from one thread in the usual order, and the next
+ *     batch's calls wait for both streams.  Different objects are independent: the library keeps no state outside them
  *     (apart from the fixed workspace of octo_postprocess_frame_static), so several host
  *     threads may each drive their own stage, on one GPU or on several.
  *   - Every function returns OCTO_OK (0) or a negative octo_status_t.  No exception

@@ -39,9 +39,11 @@ def make_stage(wl, max_batch: int, **over) -> "octo.Stage":
 
 def run_stage_gpu(stage, frames: Sequence[np.ndarray], sizes, head: np.ndarray,
                   max_items: Optional[Sequence[int]] = None, first_item: int = 0,
-                  stream: Optional[torch.cuda.Stream] = None, sentinel: int = 0x7BFF) -> GpuResult:
+                  stream: Optional[torch.cuda.Stream] = None, sentinel: int = 0x7BFF,
+                  preprocess_stream: Optional[torch.cuda.Stream] = None) -> GpuResult:
     """One pass of the whole stage.  Output buffers are pre-filled with a sentinel so that
-    untouched slots can be recognised."""
+    untouched slots can be recognised.  With preprocess_stream the letterbox is enqueued there,
+    beside the other kernels of the pass, and joined before the results are read."""
     dev = stage.device
     n = len(frames)
     d_frames = upload_frames(frames, dev)
@@ -51,7 +53,12 @@ def run_stage_gpu(stage, frames: Sequence[np.ndarray], sizes, head: np.ndarray,
     with ctx:
         det_in = torch.full((n, 3, s, s), 0, dtype=torch.int16, device=dev)
         det_in.fill_(sentinel)
-        stage.preprocess(d_frames, sizes, out=det_in.view(torch.float16))
+        if preprocess_stream is not None:
+            main = torch.cuda.current_stream(dev)
+            preprocess_stream.wait_stream(main)  # the sentinel fill above
+            stage.preprocess(d_frames, sizes, out=det_in.view(torch.float16), stream=preprocess_stream)
+        else:
+            stage.preprocess(d_frames, sizes, out=det_in.view(torch.float16))
         dets = torch.zeros((n, stage.cfg.max_det, 32), dtype=torch.uint8, device=dev)
         counts = torch.full((n,), -1, dtype=torch.int32, device=dev)
         stage.postprocess(d_head, dets=dets, counts=counts)

@@ -318,6 +318,27 @@ def test_stage_reuse_across_batches_and_streams():
         st.close()
 
 
+def test_letterbox_on_a_second_stream_beside_the_rest_of_the_pass():
+    """The letterbox kernel shares no device data with decode, NMS and crop of the same batch (it
+    reads the frames and writes the detector input; they read the head and the frames), so a caller
+    may enqueue it on a second stream.  Alternating batches, every pass against the oracle."""
+    wl = workloads.WORKLOADS["traffic_1080p"]
+    batches = [workloads.make_batch("traffic_1080p", batch=3), workloads.make_batch("traffic_1080p", batch=2, first_frame=50)]
+    refs = [_oracle(b) for b in batches]
+    st = make_stage(wl, 4)
+    side = torch.cuda.Stream()
+    try:
+        for i in range(8):
+            b, ref = batches[i % 2], refs[i % 2]
+            r = run_stage_gpu(st, b.frames, b.sizes, b.head, max_items=[200], preprocess_stream=side)
+            assert r.status == 0
+            assert half_absdiff(r.det_in, ref.det_in) <= PIX_TOL
+            _check_dets(r, ref)
+            _check_branch(r, ref, 0, max_items=200)
+    finally:
+        st.close()
+
+
 def test_crop_shapes_and_degenerate_boxes():
     """Crops of hand-placed boxes: tiny, frame-sized, clipped at the border, 1-pixel."""
     import paper_2502_01277_b200 as octo
