@@ -396,6 +396,13 @@ OCTO_API int octo_stage_set_nms_cluster(octo_stage_t* st, int32_t cluster);
 /* Cluster size of the stage's latest NMS launch (0 before the first one, or for a null stage). */
 OCTO_API int32_t octo_stage_last_nms_cluster(const octo_stage_t* st);
 
+/* 1 when the stage's latest NMS launch ran two half-sized CTAs per SM, else 0.  In automatic mode a
+ * batch of more images than the GPU has SMs is launched that way (one wave of CTAs instead of
+ * two) unless one of the stage's latest 64 NMS launches is known to have seen an image with more
+ * than 1024 candidates; a half-sized CTA holds 4096 candidates on chip instead of 8192 and sends
+ * a larger image through the global-memory path.  Results do not depend on the form. */
+OCTO_API int32_t octo_stage_last_nms_half_ctas(const octo_stage_t* st);
+
 /* Bytes of device memory the stage holds. */
 OCTO_API int64_t octo_stage_workspace_bytes(const octo_stage_t* st);
 

@@ -51,7 +51,7 @@ EXPORTS = (
     "octo_adopt_regions", "octo_queue_create", "octo_queue_destroy", "octo_queue_push", "octo_queue_pop",
     "octo_queue_pop_due", "octo_coral_schedule", "octo_queue_set_options",
     "octo_adopt_items_device", "octo_stage_selftest_wait", "octo_static_status",
-    "octo_stage_set_nms_cluster", "octo_stage_last_nms_cluster",
+    "octo_stage_set_nms_cluster", "octo_stage_last_nms_cluster", "octo_stage_last_nms_half_ctas",
 )
 
 
@@ -175,6 +175,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.octo_stage_set_nms_cluster.restype = ctypes.c_int
     lib.octo_stage_last_nms_cluster.argtypes = [vp]
     lib.octo_stage_last_nms_cluster.restype = i32
+    lib.octo_stage_last_nms_half_ctas.argtypes = [vp]
+    lib.octo_stage_last_nms_half_ctas.restype = i32
     lib.octo_stage_kernel_times.argtypes = [vp, ctypes.POINTER(KernelTimes), vp]
     lib.octo_stage_kernel_times.restype = ctypes.c_int
     lib.octo_postprocess_frame_static.argtypes = [i32, vp, i32, i32, i32, ctypes.c_float, ctypes.c_float,
@@ -469,6 +471,9 @@ class Stage:
 
     def last_nms_cluster(self) -> int:
         return int(load_library().octo_stage_last_nms_cluster(self.handle))
+
+    def last_nms_half_ctas(self) -> bool:
+        return bool(load_library().octo_stage_last_nms_half_ctas(self.handle))
 
     def set_timing(self, enable: bool) -> None:
         rc = load_library().octo_stage_set_timing(self.handle, 1 if enable else 0)

@@ -57,6 +57,9 @@ struct NmsArgs {
     int cluster;
     int* d_dense_seen;
     int launch_seq;
+    // two half-sized CTAs per SM (half the threads and half the on-chip capacity each) instead of
+    // one: for batches of more images than SMs whose images are sparse
+    bool half_ctas;
 };
 
 // Branch options of the crop kernel, per INPUT channel c (output plane swap_rb ? 2 - c : c):

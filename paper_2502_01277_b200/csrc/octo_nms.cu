@@ -35,8 +35,14 @@ namespace octo {
 
 namespace cg = cooperative_groups;
 
-constexpr int kNmsThreads = 1024;
+constexpr int kNmsThreadsFull = 1024;
 constexpr int kNmsSmemCap = 8192;   // candidates handled on chip: 8 B key + 16 B box each
+// Batches of more images than the GPU has SMs that have held only sparse images lately run two
+// smaller CTAs per SM (half the threads, half the on-chip capacity), so that the launch is one
+// wave of CTAs instead of two; an image that exceeds the smaller capacity takes the global-memory
+// path, and the launches after it are full-sized again.
+constexpr int kNmsThreadsHalf = 512;
+constexpr int kNmsSmemCapHalf = 4096;
 constexpr int kWarpSortMax = 2048;  // largest class segment a single warp sorts
 constexpr int kRankSortMax = 512;   // up to here the warp sorts by counting instead of a network
 constexpr int kSmallMax = 256;      // images with at most this many candidates take the short path
@@ -85,8 +91,8 @@ __device__ __forceinline__ float4 gather_box(const float* __restrict__ p, size_t
     return box_corners(__ldg(p), __ldg(p + es), __ldg(p + 2 * es), __ldg(p + 3 * es));
 }
 
-template <int CAP>
-__global__ void __launch_bounds__(kNmsThreads, 1)
+template <int CAP, int kNmsThreads>
+__global__ void __launch_bounds__(kNmsThreads, kNmsThreadsFull / kNmsThreads)
 nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restrict__ gtab,
            const float* __restrict__ head, int A, int C, int layout,
            const IouTest iou_test, int max_det, int key_stride, unsigned long long* __restrict__ gkeys,
@@ -140,16 +146,18 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
     }
 
     unsigned long long* const gk = gkeys + (size_t)img * key_stride;
-    const bool on_chip = cnt <= kNmsSmemCap;
+    // candidates the launch's shared memory holds
+    constexpr int smem_cap = kNmsThreads == kNmsThreadsFull ? kNmsSmemCap : kNmsSmemCapHalf;
+    const bool on_chip = cnt <= smem_cap;
     unsigned long long* keys;
     float4* boxes;
     if (on_chip) {
         boxes = reinterpret_cast<float4*>(smem_raw);
-        keys = reinterpret_cast<unsigned long long*>(smem_raw + (size_t)kNmsSmemCap * sizeof(float4));
+        keys = reinterpret_cast<unsigned long long*>(smem_raw + (size_t)smem_cap * sizeof(float4));
     } else {
         boxes = gboxes + (size_t)img * key_stride;
         keys = gk;
-        if (threadIdx.x == 0 && crank == 0) atomicOr(&ctr->status, 0x8u);
+        if (threadIdx.x == 0 && crank == 0 && cnt > kNmsSmemCap) atomicOr(&ctr->status, 0x8u);
     }
     // the short path and the global-memory path are the first CTA's alone (same count, hence the
     // same decision, in every CTA of the cluster; no cluster barrier follows on those paths)
@@ -612,14 +620,17 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
 }
 
 constexpr size_t kNmsSmemBytes = (size_t)kNmsSmemCap * (sizeof(float4) + sizeof(unsigned long long));
+constexpr size_t kNmsSmemBytesHalf = (size_t)kNmsSmemCapHalf * (sizeof(float4) + sizeof(unsigned long long));
 
 cudaError_t prepare_nms(int* max_cluster) {
     cudaError_t e;
-    e = cudaFuncSetAttribute(nms_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
+    e = cudaFuncSetAttribute(nms_kernel<8, kNmsThreadsFull>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(nms_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
+    e = cudaFuncSetAttribute(nms_kernel<64, kNmsThreadsFull>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(nms_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
+    e = cudaFuncSetAttribute(nms_kernel<512, kNmsThreadsFull>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(nms_kernel<512, kNmsThreadsHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kNmsSmemBytesHalf);
     if (e != cudaSuccess) return e;
     if (max_cluster) {
         // the largest cluster (one CTA per SM: the kernel takes nearly all shared memory of an SM)
@@ -628,7 +639,7 @@ cudaError_t prepare_nms(int* max_cluster) {
         for (int c = 8; c > 1; c >>= 1) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3((unsigned)c);
-            cfg.blockDim = dim3(kNmsThreads);
+            cfg.blockDim = dim3(kNmsThreadsFull);
             cfg.dynamicSmemBytes = kNmsSmemBytes;
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -638,7 +649,7 @@ cudaError_t prepare_nms(int* max_cluster) {
             cfg.attrs = attr;
             cfg.numAttrs = 1;
             int active = 0;
-            if (cudaOccupancyMaxActiveClusters(&active, nms_kernel<8>, &cfg) == cudaSuccess && active > 0) {
+            if (cudaOccupancyMaxActiveClusters(&active, nms_kernel<8, kNmsThreadsFull>, &cfg) == cudaSuccess && active > 0) {
                 *max_cluster = c;
                 break;
             }
@@ -653,7 +664,6 @@ static cudaError_t launch_cap(const NmsArgs& a, cudaStream_t stream) {
     FrameTable<CAP> tab;  // built per call (copied into kernel parameter space by the launch)
     if (!a.d_tab)
         for (int i = 0; i < a.n; ++i) tab.f[i] = a.frames[i];
-    const size_t smem = kNmsSmemBytes;
     // rounding boundary of the IoU test (see iou_above)
     const float up = nextafterf(a.iou_thr, INFINITY);
     IouTest iou_test;
@@ -662,7 +672,14 @@ static cudaError_t launch_cap(const NmsArgs& a, cudaStream_t stream) {
     memcpy(&up_bits, &up, sizeof(up_bits));
     iou_test.tie_up = (up_bits & 1u) == 0u ? 1 : 0;
     const int cluster = a.cluster == 2 || a.cluster == 4 || a.cluster == 8 ? a.cluster : 1;
-    return launch_kernel_cluster(nms_kernel<CAP>, dim3((unsigned)(a.n * cluster)), dim3(kNmsThreads), smem, stream, a.pdl,
+    // two half-sized CTAs per SM: only the largest table size has that form (more images than SMs)
+    const bool half = CAP == 512 && a.half_ctas && cluster == 1;
+    auto kernel = nms_kernel<CAP, kNmsThreadsFull>;
+    if constexpr (CAP == 512) {
+        if (half) kernel = nms_kernel<512, kNmsThreadsHalf>;
+    }
+    return launch_kernel_cluster(kernel, dim3((unsigned)(a.n * cluster)), dim3(half ? kNmsThreadsHalf : kNmsThreadsFull),
+                                 half ? kNmsSmemBytesHalf : kNmsSmemBytes, stream, a.pdl,
                                  cluster, tab, a.d_tab, a.d_head, a.A, a.C, a.layout, iou_test, a.max_det, a.key_stride,
                                  a.d_keys, a.d_boxes, a.d_cand_count, reinterpret_cast<octo_det_rec*>(a.d_dets),
                                  a.d_counts, a.num_branches, a.class_agnostic, a.masks, a.d_bcount, a.d_bidx,

@@ -173,6 +173,7 @@ extern "C" int octo_postprocess_frame_static(int32_t device, const float* d_head
     a.d_bcount = d_bcount;
     a.d_bidx = d_bidx;
     a.max_batch = 1;
+    a.half_ctas = false;
     a.d_ctr = d_ctr;
     a.cluster = 1;
     a.d_dense_seen = nullptr;

@@ -463,6 +463,10 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
         }
     }
     st->nms_cluster_last = a.cluster;
+    // More images than SMs and no crowded image lately: two half-sized CTAs per SM, one wave.
+    a.half_ctas = a.cluster == 1 && n > st->sm_count && st->nms_cluster_mode == 0 && st->h_dense_seen &&
+                  st->nms_seq - *static_cast<const volatile int*>(st->h_dense_seen) > kNmsClusterWindow;
+    st->nms_half_last = a.half_ctas;
     cudaError_t e;
     {
         ScopedKernelTimer t(st, OCTO_K_NMS, stream);
@@ -588,6 +592,7 @@ extern "C" int octo_stage_set_nms_cluster(octo_stage_t* st, int32_t cluster) {
 }
 
 extern "C" int32_t octo_stage_last_nms_cluster(const octo_stage_t* st) { return st ? st->nms_cluster_last : 0; }
+extern "C" int32_t octo_stage_last_nms_half_ctas(const octo_stage_t* st) { return st && st->nms_half_last ? 1 : 0; }
 
 extern "C" int octo_stage_set_timing(octo_stage_t* st, int32_t enable) {
     if (!st) return OCTO_E_INVALID_ARG;

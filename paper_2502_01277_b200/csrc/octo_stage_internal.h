@@ -37,6 +37,7 @@ struct octo_stage {
     int nms_max_cluster;
     int nms_cluster_mode;  // 0 automatic, else the caller's size
     int nms_cluster_last;  // size of the latest launch
+    bool nms_half_last;    // the latest launch ran two half-sized CTAs per SM
     int nms_seq;
     int* h_dense_seen;  // host view (volatile reads)
     int* d_dense_seen;  // device view of the same integer

@@ -87,3 +87,34 @@ def test_automatic_choice_follows_the_candidate_counts():
         assert st.last_nms_cluster() == 1
     finally:
         st.close()
+
+
+def test_more_images_than_sms_run_two_half_sized_ctas_per_sm():
+    """A batch of more images than the GPU has SMs is launched with two half-sized CTAs per SM while
+    no crowded image is known.  Such a CTA holds 4096 candidates on chip: in the first pass an image
+    with 5000 goes through the global-memory path and one with 700 through the general on-chip path
+    on half the threads; the crowded image is reported, so the second pass is full-sized again, and
+    after 64 sparse launches the half-sized form returns.  Every pass gives the oracle's detections."""
+    from test_gpu_parity import _check_dets
+    n = torch.cuda.get_device_properties(0).multi_processor_count + 2
+    sparse = _batch(150, 20, n, max_det=1000)
+    mixed = replace(sparse, head=sparse.head.copy())
+    mixed.head[3] = _batch(5000, 250, 1, seed=8, max_det=1000).head[0]
+    mixed.head[n // 2] = _batch(700, 60, 1, seed=9, max_det=1000).head[0]
+    ref_sparse, ref_mixed = _oracle_dets(sparse), _oracle_dets(mixed)
+    assert ref_mixed.n_cand[3] > 4096 and 256 < ref_mixed.n_cand[n // 2] <= 4096 and ref_sparse.n_cand.max() <= 256
+    st = make_stage(sparse.workload, n)
+    try:
+        res = run_stage_gpu(st, mixed.frames, mixed.sizes, mixed.head, max_items=[8])
+        assert st.last_nms_half_ctas() and st.last_nms_cluster() == 1
+        _check_dets(res, ref_mixed)
+        assert res.status & ~0x2 == 0  # 5000 candidates fit a full-sized CTA: no BIG_NMS report
+        res = run_stage_gpu(st, mixed.frames, mixed.sizes, mixed.head, max_items=[8])
+        assert not st.last_nms_half_ctas()
+        _check_dets(res, ref_mixed)
+        for i in range(66):
+            res = run_stage_gpu(st, sparse.frames, sparse.sizes, sparse.head, max_items=[8])
+            assert st.last_nms_half_ctas() == (i >= 64)
+        _check_dets(res, ref_sparse)
+    finally:
+        st.close()
