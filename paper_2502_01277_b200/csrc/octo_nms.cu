@@ -391,9 +391,23 @@ nms_kernel(const __grid_constant__ FrameTable<CAP> tab, const FrameDesc* __restr
             } else if (m > 1 && m <= kWarpSortMax) {
                 bitonic_range<false>(keys + s, m, lane, 32);
             }
-            for (int p = s + lane; p < e; p += 32) {
-                const int anchor = (int)(keys[p] & ((1ull << kKeyAnchorBits) - 1));
-                boxes[p] = gather_box(hbase + (size_t)anchor * as, es);
+            // boxes of the class from the head, four per lane in flight (a lone warp pays the full
+            // round trip for every load it waits on)
+            for (int p0 = s + lane; p0 < e; p0 += 128) {
+                float4 b4[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int p = p0 + 32 * u;
+                    if (p < e) {
+                        const int anchor = (int)(keys[p] & ((1ull << kKeyAnchorBits) - 1));
+                        b4[u] = gather_box(hbase + (size_t)anchor * as, es);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int p = p0 + 32 * u;
+                    if (p < e) boxes[p] = b4[u];
+                }
             }
             __syncwarp();
             int nk = 0;  // survivors of this class, compacted at [s, s + nk)
