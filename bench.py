@@ -47,9 +47,9 @@ NCU_TRAFFIC = {
     "letterbox": (("paper_2502_01277_b200/csrc/octo_letterbox.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
                   "82ba43ca31895b9a", 3706404.0, "frame"),
     "decode": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-               "47f0eeeadf72fd19", 1741824.0, "frame"),
+               "5ec9cd6b248b8101", 1740516.0, "frame"),
     "decode_planes": (("paper_2502_01277_b200/csrc/octo_decode.cu", "paper_2502_01277_b200/csrc/octo_common.cuh"),
-                      "47f0eeeadf72fd19", 2812296.0, "frame"),
+                      "5ec9cd6b248b8101", 2810668.0, "frame"),
 }
 # Warp instructions the crop kernel executes per crop (ncu smsp__inst_executed.sum of the same capture):
 # the kernel is bound by instruction issue, so its issue rate is reported beside the byte rates.

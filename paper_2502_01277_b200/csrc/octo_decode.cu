@@ -99,8 +99,9 @@ decode_kernel(const float* __restrict__ head, int A, int C, int mode, float conf
             if (have) {
                 // the row is requested in batches of kPieces 32-byte pieces (48 values per group), so
                 // a row of 85 values takes two round trips and the kernel stays at 32-40 registers
-                // (the obj scan of large batches lives on occupancy)
-                constexpr int kPieces = 6;
+                // (the obj scan of large batches lives on occupancy); the small-grid form asks for
+                // the whole row at once (any row of up to 5 + 128 values): one round trip less
+                constexpr int kPieces = kDecPerThread == 1 ? 17 : 6;
                 for (int e00 = 0; e00 < row_len; e00 += 8 * kPieces) {
                     float v[kPieces];
 #pragma unroll
