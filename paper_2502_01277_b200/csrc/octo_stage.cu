@@ -464,7 +464,8 @@ extern "C" int octo_postprocess_batch(octo_stage_t* st, const float* d_head, int
     }
     st->nms_cluster_last = a.cluster;
     // More images than SMs and no crowded image lately: two half-sized CTAs per SM, one wave.
-    a.half_ctas = a.cluster == 1 && n > st->sm_count && st->nms_cluster_mode == 0 && st->h_dense_seen &&
+    // (the half-sized kernel exists for the largest frame-table size only, i.e. for more than 64 images)
+    a.half_ctas = a.cluster == 1 && n > st->sm_count && n > 64 && st->nms_cluster_mode == 0 && st->h_dense_seen &&
                   st->nms_seq - *static_cast<const volatile int*>(st->h_dense_seen) > kNmsClusterWindow;
     st->nms_half_last = a.half_ctas;
     cudaError_t e;
