@@ -150,3 +150,11 @@ def test_crowded_image_under_the_checked_build(checked, cluster):
         _check_dets(res, ref)
     finally:
         st.close()
+
+
+def test_half_sized_nms_ctas_under_the_checked_build(checked):
+    """More images than SMs: two half-sized NMS CTAs per SM, with an image on the general on-chip path
+    and one that exceeds the smaller on-chip capacity, every index range-checked (the case of the
+    NMS module; it asserts the launch forms and parity, the status word is checked there too)."""
+    from test_gpu_nms_cluster import test_more_images_than_sms_run_two_half_sized_ctas_per_sm as case
+    case()

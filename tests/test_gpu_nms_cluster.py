@@ -116,5 +116,6 @@ def test_more_images_than_sms_run_two_half_sized_ctas_per_sm():
             res = run_stage_gpu(st, sparse.frames, sparse.sizes, sparse.head, max_items=[8])
             assert st.last_nms_half_ctas() == (i >= 64)
         _check_dets(res, ref_sparse)
+        assert res.status & ~0x2 == 0
     finally:
         st.close()
